@@ -1,0 +1,691 @@
+// Beam-search kernels: fused log-softmax + validity mask + beam top-k (one level of Algorithm 1 / Algorithm 3),
+// the draft head's glue (Eq. 1-3 inputs), the verify pass's token list, and accept / roll-back (Algorithm 2
+// lines 5-7).  Every kernel here runs one thread block per request; requests never interact.
+#include <math.h>
+
+#include "engine_state.cuh"
+
+namespace nz {
+
+// ====================================================================================================
+// fused log-softmax + mask + top-k
+// ====================================================================================================
+// Per request: each warp takes beams r = warp, warp + n_warps, ...  For a beam it loads the T logits of the
+// level's codebook (VPL per lane), computes log-softmax with warp shuffles, and extracts the beam's best
+// candidates in order (repeated warp arg-max; ties to the smaller code):
+//   per_beam <  T : the per_beam most probable codes, THEN the hash-set filter on those       (Algorithm 3 l.19, 23-26)
+//   per_beam >= T : the filter on all T codes, THEN the K best by cumulative log-probability  (top-k restricted to V)
+// The sorted per-beam lists go to shared memory and warp 0 merges them into the K best of the request
+// (ties to the smaller parent rank, then the smaller code).
+namespace {
+
+struct Cand { float s; int r; int t; };
+
+__device__ __forceinline__ bool cand_better(float s, int r, int t, float s2, int r2, int t2) {
+  if (s != s2) return s > s2;
+  if (r != r2) return r < r2;
+  return t < t2;
+}
+
+template <int VPL>
+__global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
+  const int b = blockIdx.x;
+  if (a.gate_mode == 1 && a.gate[b] != a.gate_value) return;
+  if (a.gate_mode == 2 && !(a.gate[b] < a.gate_value)) return;
+  extern __shared__ unsigned char smem_raw[];
+  const int nb_cap = a.in_stride;
+  float* l_score = reinterpret_cast<float*>(smem_raw);              // [nb_cap][K]
+  int* l_tok = reinterpret_cast<int*>(l_score + (size_t)nb_cap * a.K);   // [nb_cap][K]
+  int* l_cnt = l_tok + (size_t)nb_cap * a.K;                         // [nb_cap]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  const int nb = min(a.in_count[b], nb_cap);
+  const bool all_codes = a.per_beam >= a.T;
+  const int want = all_codes ? min(a.K, a.T) : min(a.per_beam, a.K);
+
+  for (int r = warp; r < nb; r += n_warps) {
+    const long long row = a.src_row ? a.src_row[(long long)b * a.in_stride + r] : (long long)b * a.src_mul + r;
+    const float* z = a.logits + row * a.row_stride + a.col_off;
+    float key[VPL];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int t = lane + 32 * j;
+      key[j] = (t < a.T) ? z[t] : -INFINITY;
+      mx = fmaxf(mx, key[j]);
+    }
+    mx = warp_max(mx);
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) sum += (lane + 32 * j < a.T) ? expf(key[j] - mx) : 0.f;
+    sum = warp_sum(sum);
+    const float lse = mx + logf(sum);
+    const float base = a.in_score[(long long)b * a.in_stride + r];
+    unsigned long long prefix_key = 0;
+    for (int l = 0; l < a.n; ++l)
+      prefix_key += (unsigned long long)a.in_codes[((long long)b * a.in_stride + r) * a.tuple_len + l] * a.li.mult[l];
+    const unsigned long long mult_n = a.li.mult[a.n];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int t = lane + 32 * j;
+      if (t < a.T) {
+        key[j] -= lse;                                   // log-probability
+        if (all_codes) {
+          key[j] += base;                                // rank by cumulative log-probability
+          if (a.filter && !hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n)) key[j] = -INFINITY;
+        }
+      }
+    }
+    // ordered extraction
+    int cnt = 0;
+    for (int it = 0; it < want; ++it) {
+      float bv = -INFINITY; int bt = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < VPL; ++j)
+        if (key[j] > bv) { bv = key[j]; bt = lane + 32 * j; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
+        if (ov > bv || (ov == bv && ot < bt)) { bv = ov; bt = ot; }
+      }
+      if (bv == -INFINITY) break;
+      if ((bt & 31) == lane) {
+#pragma unroll
+        for (int j = 0; j < VPL; ++j)
+          if (j == (bt >> 5)) key[j] = -INFINITY;
+      }
+      if (lane == 0) {
+        l_score[(size_t)r * a.K + cnt] = all_codes ? bv : base + bv;
+        l_tok[(size_t)r * a.K + cnt] = bt;
+      }
+      ++cnt;
+    }
+    __syncwarp();
+    if (!all_codes && a.filter) {                        // filter the chosen codes, keep their order
+      int kept = 0;
+      for (int c0 = 0; c0 < cnt; c0 += 32) {
+        const int c = c0 + lane;
+        bool ok = false; float s = 0.f; int t = 0;
+        if (c < cnt) {
+          s = l_score[(size_t)r * a.K + c]; t = l_tok[(size_t)r * a.K + c];
+          ok = hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, ok);
+        __syncwarp();
+        if (ok) {
+          const int dst = kept + __popc(m & ((1u << lane) - 1u));
+          l_score[(size_t)r * a.K + dst] = s; l_tok[(size_t)r * a.K + dst] = t;
+        }
+        kept += __popc(m);
+        __syncwarp();
+      }
+      cnt = kept;
+    }
+    if (lane == 0) l_cnt[r] = cnt;
+  }
+  __syncthreads();
+  if (warp != 0) return;
+
+  // merge the sorted lists
+  constexpr int RPL = 4;                                 // lists per lane: in_stride <= 128
+  int ptr[RPL];
+#pragma unroll
+  for (int q = 0; q < RPL; ++q) ptr[q] = 0;
+  int n_out = 0;
+  for (int k = 0; k < a.K; ++k) {
+    float bs = -INFINITY; int br = 0x7fffffff, bt = 0x7fffffff;
+#pragma unroll
+    for (int q = 0; q < RPL; ++q) {
+      const int r = lane + 32 * q;
+      if (r < nb && ptr[q] < l_cnt[r]) {
+        const float s = l_score[(size_t)r * a.K + ptr[q]];
+        const int t = l_tok[(size_t)r * a.K + ptr[q]];
+        if (br == 0x7fffffff || cand_better(s, r, t, bs, br, bt)) { bs = s; br = r; bt = t; }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float os = __shfl_xor_sync(0xffffffffu, bs, o);
+      const int orr = __shfl_xor_sync(0xffffffffu, br, o);
+      const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
+      if (orr != 0x7fffffff && (br == 0x7fffffff || cand_better(os, orr, ot, bs, br, bt))) { bs = os; br = orr; bt = ot; }
+    }
+    if (br == 0x7fffffff) break;
+#pragma unroll
+    for (int q = 0; q < RPL; ++q)
+      if (lane + 32 * q == br) ++ptr[q];
+    const long long o = (long long)b * a.out_stride + k;
+    if (lane == 0) {
+      a.out_score[o] = bs;
+      if (a.out_parent) a.out_parent[o] = br;
+      if (a.out_token) a.out_token[o] = bt;
+    }
+    if (a.out_codes) {
+      for (int l = lane; l < a.tuple_len; l += 32) {
+        int c = -1;
+        if (l < a.n) c = a.in_codes[((long long)b * a.in_stride + br) * a.tuple_len + l];
+        else if (l == a.n) c = bt;
+        a.out_codes[o * a.tuple_len + l] = c;
+      }
+    }
+    ++n_out;
+  }
+  for (int k = n_out + lane; k < a.K; k += 32) {
+    const long long o = (long long)b * a.out_stride + k;
+    a.out_score[o] = -INFINITY;
+    if (a.out_parent) a.out_parent[o] = -1;
+    if (a.out_token) a.out_token[o] = -1;
+    if (a.out_codes)
+      for (int l = 0; l < a.tuple_len; ++l) a.out_codes[o * a.tuple_len + l] = -1;
+  }
+  if (lane == 0) a.out_count[b] = n_out;
+}
+
+}  // namespace
+
+size_t select_smem_bytes(int in_stride, int K) {
+  return (size_t)in_stride * K * (sizeof(float) + sizeof(int)) + (size_t)in_stride * sizeof(int);
+}
+
+cudaError_t select_configure(int max_beam) {
+  const int bytes = (int)select_smem_bytes(max_beam, max_beam);
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(select_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  return cudaFuncSetAttribute(select_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+void launch_select(const SelectArgs& a, cudaStream_t st) {
+  if (a.batch <= 0) return;
+  const size_t smem = select_smem_bytes(a.in_stride, a.K);
+  if (a.T <= 32) select_kernel<1><<<a.batch, 256, smem, st>>>(a);
+  else if (a.T <= 256) select_kernel<8><<<a.batch, 256, smem, st>>>(a);
+  else if (a.T <= 512) select_kernel<16><<<a.batch, 256, smem, st>>>(a);
+  else select_kernel<32><<<a.batch, 256, smem, st>>>(a);
+}
+
+// ====================================================================================================
+// small state kernels
+// ====================================================================================================
+namespace {
+
+__global__ void fill_i32_kernel(int* p, long long n, int v) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    p[i] = v;
+}
+__global__ void fill_f32_kernel(float* p, long long n, float v) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    p[i] = v;
+}
+
+// B_0 = { empty beam, score 0 } for every request; nothing settled.
+__global__ void init_decode_kernel(EngineState e, int batch) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b == 0)
+    for (int i = 0; i < 8; ++i) e.counters[i] = 0;
+  if (b >= batch) return;
+  e.tb_count[0 * e.Bmax + b] = 1;
+  e.tb_score[lvl_bk(e, 0, b, 0)] = 0.f;
+  e.tb_parent[lvl_bk(e, 0, b, 0)] = -1;
+  e.tb_src[lvl_bk(e, 0, b, 0)] = -1;
+  e.row_m[b] = 0;
+  e.row_cur[b] = -1;
+  e.d_m[b] = e.L;
+  e.dw_count[(long long)e.L * e.Bmax + b] = 0;
+}
+
+// Start of a round's drafting (Algorithm 2 line 3): the draft head continues from the true beams B_m, or from
+// the empty beam in the first round (Algorithm 3 line 14).
+__global__ void draft_init_kernel(EngineState e, int batch, int from_scratch) {
+  const int b = blockIdx.x;
+  if (b >= batch) return;
+  const int m = e.row_m[b];
+  if (m >= e.L) { if (threadIdx.x == 0) { e.d_m[b] = e.L; e.dw_count[(long long)e.L * e.Bmax + b] = 0; } return; }
+  const int mm = from_scratch ? 0 : m;
+  const int cnt = e.tb_count[mm * e.Bmax + b];
+  for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
+    const long long s = lvl_bk(e, mm, b, k);
+    const bool live = k < cnt;
+    e.dw_score[s] = live ? e.tb_score[s] : -INFINITY;
+    e.dw_parent[s] = live ? k : -1;
+    for (int l = 0; l < e.L; ++l) e.dw_codes[s * e.L + l] = live ? e.tb_codes[s * e.L + l] : -1;
+  }
+  if (threadIdx.x == 0) { e.dw_count[mm * e.Bmax + b] = cnt; e.d_m[b] = mm; }
+}
+
+// Caller-supplied drafts for the round (or none: n_draft == nullptr and drafts == nullptr -> zero drafts).
+__global__ void draft_set_kernel(EngineState e, int batch, int K, const int* drafts, const int* n_draft) {
+  const int b = blockIdx.x;
+  if (b >= batch) return;
+  const int cnt = (drafts && e.row_m[b] < e.L) ? max(0, min(n_draft[b], K)) : 0;
+  for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
+    const long long s = lvl_bk(e, e.L, b, k);
+    bool ok = k < cnt;
+    for (int l = 0; l < e.L; ++l) {
+      int c = ok ? drafts[((long long)b * K + k) * e.L + l] : -1;
+      if (ok && (c < 0 || c >= e.li.T[l])) { atomicOr(e.status, kStBadCode); c = 0; }
+      e.dw_codes[s * e.L + l] = c;
+    }
+    e.dw_score[s] = ok ? 0.f : -INFINITY;
+    e.dw_parent[s] = -1;
+  }
+  if (threadIdx.x == 0) { e.dw_count[(long long)e.L * e.Bmax + b] = cnt; e.d_m[b] = e.L; }
+}
+
+// Eq. 2 input: x = h_l + s_l for every (request, beam); s_1 = h_0 (Eq. 1).
+template <typename T>
+__global__ void draft_x_kernel(EngineState e, int batch, int l, T* x) {
+  const int bk = blockIdx.x;                       // b * Kmax + k
+  const int b = bk / e.Kmax;
+  if (b >= batch) return;
+  const float* h = e.h_f32 + ((long long)b * (e.L + 1) + l) * e.d;
+  const float* s = (l == 1) ? e.h_f32 + (long long)b * (e.L + 1) * e.d
+                            : e.state_lv + ((long long)l * e.Bmax * e.Kmax + bk) * e.d;
+  for (int c = threadIdx.x; c < e.d; c += blockDim.x) x[(long long)bk * e.d + c] = from_f32<T>(h[c] + s[c]);
+}
+
+// Eq. 3 input rows [s_l ; e_l] for the step s_l -> s_{l+1}.
+//   requests still teacher-forcing (d_m >= l): beam k of the start set, its own state, its l-th code;
+//   requests drafting (d_m < l): survivor k of level l, its parent's state, the code just chosen.
+template <typename T>
+__global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* embed, T* A) {
+  const int bk = blockIdx.x;
+  const int b = bk / e.Kmax, k = bk - b * e.Kmax;
+  if (b >= batch) return;
+  T* dst = A + (long long)bk * 2 * e.d;
+  const int dm = e.d_m[b];
+  int src_level, parent;
+  bool live = dm < e.L || e.row_m[b] < e.L;
+  if (dm >= l) { src_level = min(dm, e.L); parent = k; }
+  else { src_level = l; parent = -2; }
+  const long long s_idx = lvl_bk(e, src_level, b, k);
+  live = live && k < e.dw_count[src_level * e.Bmax + b];
+  if (live && parent == -2) parent = e.dw_parent[s_idx];
+  const int code = live ? e.dw_codes[s_idx * e.L + (l - 1)] : -1;
+  live = live && code >= 0 && parent >= 0;
+  if (!live) {
+    for (int c = threadIdx.x; c < 2 * e.d; c += blockDim.x) dst[c] = from_f32<T>(0.f);
+    return;
+  }
+  const float* s = (l == 1) ? e.h_f32 + (long long)b * (e.L + 1) * e.d
+                            : e.state_lv + ((long long)l * e.Bmax * e.Kmax + (long long)b * e.Kmax + parent) * e.d;
+  const T* emb = embed + (long long)(e.li.off[l - 1] + code) * e.d;
+  for (int c = threadIdx.x; c < e.d; c += blockDim.x) {
+    dst[c] = from_f32<T>(s[c]);
+    dst[e.d + c] = emb[c];
+  }
+}
+
+// ----------------------------------------------------------------------------------------------------
+// verify-pass token list (the nodes M_p runs on this round)
+// ----------------------------------------------------------------------------------------------------
+// Request with m levels settled: nodes = the level-m code of every beam of B_m (slot = beam rank) and the codes
+// of levels m+1..L-1 of every alive draft (slot = draft index).  Tokens of a request are contiguous; requests
+// are laid out in order (each block sums the counts of the requests before it).
+__global__ void nodes_count_kernel(EngineState e, int batch) {
+  const int b = blockIdx.x;
+  const int m = e.row_m[b];
+  const int L = e.L;
+  __shared__ int n_alive;
+  if (threadIdx.x == 0) n_alive = 0;
+  __syncthreads();
+  if (m >= L) {
+    if (threadIdx.x == 0) { e.row_tok_count[b] = 0; e.row_cur[b] = -1; }
+    for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) e.d_alive[b * e.Kmax + k] = 0;
+    return;
+  }
+  const int nb = e.tb_count[m * e.Bmax + b];
+  const int nd = e.dw_count[(long long)L * e.Bmax + b];
+  for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
+    int beta = -1;
+    if (k < nd) {
+      const int* dc = e.dw_codes + lvl_bk(e, L, b, k) * L;
+      for (int r = 0; r < nb && beta < 0; ++r) {
+        const int* bc = e.tb_codes + lvl_bk(e, m, b, r) * L;
+        bool eq = true;
+        for (int l = 0; l < m; ++l) eq &= (dc[l] == bc[l]);
+        if (eq) beta = r;
+      }
+    }
+    e.d_alive[b * e.Kmax + k] = beta >= 0;
+    e.d_beam[b * e.Kmax + k] = beta;
+    if (beta >= 0) atomicAdd(&n_alive, 1);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    e.row_tok_count[b] = nb + n_alive * (L - 1 - m);
+    e.row_cur[b] = m;
+  }
+}
+
+__global__ void nodes_fill_kernel(EngineState e, int batch) {
+  const int b = blockIdx.x;
+  const int L = e.L, Kmax = e.Kmax;
+  __shared__ int s_off, s_alive_rank[128], s_n_alive;
+  if (threadIdx.x == 0) {
+    int off = 0;
+    for (int i = 0; i < b; ++i) off += e.row_tok_count[i];
+    s_off = off;
+    if (b == batch - 1) *e.n_tokens = off + e.row_tok_count[b];
+    int c = 0;
+    for (int k = 0; k < Kmax; ++k) { s_alive_rank[k] = c; c += e.d_alive[b * Kmax + k]; }
+    s_n_alive = c;
+  }
+  for (int i = threadIdx.x; i < L * Kmax; i += blockDim.x) e.node_index[(long long)b * L * Kmax + i] = -1;
+  __syncthreads();
+  const int m = e.row_m[b];
+  if (m >= L) return;
+  const int nb = e.tb_count[m * e.Bmax + b];
+  const int P = e.row_P[b];
+  const long long slab_elems = (long long)Kmax * e.Hkv * e.hd;       // one level slab of one request
+  const long long row_elems = (long long)(L - 1) * slab_elems;
+  auto kv_off = [&](int level, int slot) {                             // level 1..L-1
+    return (long long)b * row_elems + (long long)(level - 1) * slab_elems + (long long)slot * e.Hkv * e.hd;
+  };
+  // level-m nodes: the true beams
+  for (int r = threadIdx.x; r < nb; r += blockDim.x) {
+    const int t = s_off + r;
+    const long long bi = lvl_bk(e, m, b, r);
+    e.tok_row[t] = b; e.tok_pos[t] = P + m - 1; e.tok_ctx_len[t] = P;
+    e.tok_id[t] = e.li.off[m - 1] + e.tb_codes[bi * L + (m - 1)];
+    e.tok_kv_dst[t] = kv_off(m, r);
+    for (int i = 1; i <= L; ++i) {
+      long long o = -1;
+      if (i < m) o = kv_off(i, e.tb_anc[bi * L + (i - 1)]);
+      else if (i == m) o = kv_off(m, r);
+      e.tok_ext[(long long)t * L + (i - 1)] = o;
+    }
+    e.tb_src[bi] = t;
+    e.tb_self[bi] = r;
+    e.node_index[((long long)b * L + m) * Kmax + r] = t;
+  }
+  // levels m+1 .. L-1 of alive drafts
+  const int n_lv = L - 1 - m;
+  for (int idx = threadIdx.x; idx < n_lv * Kmax; idx += blockDim.x) {
+    const int j = m + 1 + idx / Kmax, k = idx % Kmax;
+    if (!e.d_alive[b * Kmax + k]) continue;
+    const int t = s_off + nb + (j - m - 1) * s_n_alive + s_alive_rank[k];
+    const int beta = e.d_beam[b * Kmax + k];
+    const long long bi = lvl_bk(e, m, b, beta);
+    const long long di = lvl_bk(e, L, b, k);
+    e.tok_row[t] = b; e.tok_pos[t] = P + j - 1; e.tok_ctx_len[t] = P;
+    e.tok_id[t] = e.li.off[j - 1] + e.dw_codes[di * L + (j - 1)];
+    e.tok_kv_dst[t] = kv_off(j, k);
+    for (int i = 1; i <= L; ++i) {
+      long long o = -1;
+      if (i < m) o = kv_off(i, e.tb_anc[bi * L + (i - 1)]);
+      else if (i == m) o = kv_off(m, beta);
+      else if (i <= j) o = kv_off(i, k);
+      e.tok_ext[(long long)t * L + (i - 1)] = o;
+    }
+    e.node_index[((long long)b * L + j) * Kmax + k] = t;
+  }
+}
+
+// Teacher-forced nodes: beams given by the caller, every beam processes all of its `level` codes.
+__global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams, int level, const int* prefixes) {
+  const int b = blockIdx.x;
+  const int L = e.L, Kmax = e.Kmax;
+  const int per_row = n_beams * level;
+  const int P = e.row_P[b];
+  const long long slab_elems = (long long)Kmax * e.Hkv * e.hd;
+  const long long row_elems = (long long)(L - 1) * slab_elems;
+  if (b == 0 && threadIdx.x == 0) *e.n_tokens = batch * per_row;
+  for (int i = threadIdx.x; i < L * Kmax; i += blockDim.x) e.node_index[(long long)b * L * Kmax + i] = -1;
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < per_row; idx += blockDim.x) {
+    const int j = 1 + idx / n_beams, r = idx % n_beams;
+    const int t = b * per_row + idx;
+    int code = prefixes[((long long)b * n_beams + r) * level + (j - 1)];
+    if (code < 0 || code >= e.li.T[j - 1]) { atomicOr(e.status, kStBadCode); code = 0; }
+    e.tok_row[t] = b; e.tok_pos[t] = P + j - 1; e.tok_ctx_len[t] = P;
+    e.tok_id[t] = e.li.off[j - 1] + code;
+    const long long self = (long long)b * row_elems + (long long)(j - 1) * slab_elems + (long long)r * e.Hkv * e.hd;
+    e.tok_kv_dst[t] = self;
+    for (int i = 1; i <= L; ++i)
+      e.tok_ext[(long long)t * L + (i - 1)] =
+          (i <= j) ? (long long)b * row_elems + (long long)(i - 1) * slab_elems + (long long)r * e.Hkv * e.hd : -1;
+    e.node_index[((long long)b * L + j) * Kmax + r] = t;
+  }
+}
+
+// ----------------------------------------------------------------------------------------------------
+// accept / roll back (Algorithm 2 lines 5-7)
+// ----------------------------------------------------------------------------------------------------
+// After B_{n+1} has been selected for a request whose beams B_n had logits in this pass:
+//   n + 1 == L : the request is finished; B_L is the result.
+//   otherwise  : every beam of B_{n+1} inherits its parent's KV slots (a slot-table rewrite: rejected drafts'
+//                KV rows simply become unreachable) and is matched against the alive drafts.  If every beam is
+//                the (n+1)-prefix of a draft, its hidden state is already in the pass and selection goes on;
+//                else level n+1 is the rejection level and the request waits for the next round.
+__global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count) {
+  const int b = blockIdx.x;
+  if (e.row_cur[b] != n) return;
+  const int L = e.L, Kmax = e.Kmax;
+  const int n1 = n + 1;
+  const int cnt = e.tb_count[n1 * e.Bmax + b];
+  if (n1 == L) {
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+      const long long s = lvl_bk(e, L, b, k);
+      out_score[(long long)b * K + k] = k < cnt ? e.tb_score[s] : -INFINITY;
+      for (int l = 0; l < L; ++l) out_codes[((long long)b * K + k) * L + l] = k < cnt ? e.tb_codes[s * L + l] : -1;
+    }
+    if (threadIdx.x == 0) { out_count[b] = cnt; e.row_m[b] = L; e.row_cur[b] = -1; }
+    return;
+  }
+  __shared__ int all_matched;
+  if (threadIdx.x == 0) all_matched = 1;
+  __syncthreads();
+  const int nd = e.dw_count[(long long)L * e.Bmax + b];
+  for (int r = threadIdx.x; r < cnt; r += blockDim.x) {
+    const long long bi = lvl_bk(e, n1, b, r);
+    const int parent = e.tb_parent[bi];
+    const long long pi = lvl_bk(e, n, b, parent);
+    for (int i = 0; i + 1 < n; ++i) e.tb_anc[bi * L + i] = e.tb_anc[pi * L + i];
+    if (n >= 1) e.tb_anc[bi * L + (n - 1)] = e.tb_self[pi];
+    const int* bc = e.tb_codes + bi * L;
+    int match = -1;
+    for (int k = 0; k < nd && match < 0; ++k) {
+      if (!e.d_alive[b * Kmax + k]) continue;
+      const int* dc = e.dw_codes + lvl_bk(e, L, b, k) * L;
+      bool eq = true;
+      for (int l = 0; l < n1; ++l) eq &= (dc[l] == bc[l]);
+      if (eq) match = k;
+    }
+    if (match >= 0) {
+      e.tb_src[bi] = e.node_index[((long long)b * L + n1) * Kmax + match];
+      e.tb_self[bi] = match;
+    } else {
+      e.tb_src[bi] = -1;
+      e.tb_self[bi] = -1;
+      all_matched = 0;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    e.row_m[b] = n1;
+    e.row_cur[b] = (all_matched && cnt > 0) ? n1 : -1;
+    if (cnt == 0) {               // no beam survived (possible only with an empty codebook): finish empty
+      e.row_m[b] = L;
+      out_count[b] = 0;
+    }
+  }
+}
+
+// End of a round: accepted length of every draft = the largest i <= (level reached) with D[k][0..i) in B_i;
+// trace outputs; counters for the host (unfinished requests, primary tokens, accepted levels).
+__global__ void round_end_kernel(EngineState e, int batch, int K, int round, nezha_trace tr, int m_before_unused) {
+  const int b = blockIdx.x;
+  const int L = e.L, Kmax = e.Kmax;
+  const int took_part = e.row_tok_count[b] > 0;
+  const int m_now = e.row_m[b];
+  const int nd = took_part ? e.dw_count[(long long)L * e.Bmax + b] : 0;
+  const long long tro = ((long long)(round - 1) * batch + b);
+  __shared__ int acc_sum;
+  if (threadIdx.x == 0) acc_sum = 0;
+  __syncthreads();
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    int acc = -1;
+    if (k < nd) {
+      const int* dc = e.dw_codes + lvl_bk(e, L, b, k) * L;
+      acc = 0;
+      for (int i = 1; i <= m_now; ++i) {
+        const int nbi = e.tb_count[i * e.Bmax + b];
+        bool in = false;
+        for (int r = 0; r < nbi && !in; ++r) {
+          const int* bc = e.tb_codes + lvl_bk(e, i, b, r) * L;
+          bool eq = true;
+          for (int l = 0; l < i; ++l) eq &= (dc[l] == bc[l]);
+          in = eq;
+        }
+        if (in) acc = i; else break;
+      }
+      atomicAdd(&acc_sum, acc);
+    }
+    if (tr.accepted_len) tr.accepted_len[tro * K + k] = acc;
+    if (tr.drafts)
+      for (int l = 0; l < L; ++l)
+        tr.drafts[(tro * K + k) * L + l] = (k < nd) ? e.dw_codes[lvl_bk(e, L, b, k) * L + l] : -1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (tr.n_draft) tr.n_draft[tro] = took_part ? nd : -1;
+    if (tr.level_reached) tr.level_reached[tro] = took_part ? m_now : -1;
+    if (m_now < L) atomicAdd(&e.counters[0], 1);
+    atomicAdd(&e.counters[1], e.row_tok_count[b]);
+    atomicAdd(&e.counters[2], acc_sum);
+    if (round == 1) atomicAdd(&e.counters[3], nd);
+  }
+}
+
+__global__ void write_out_kernel(const int* codes, const float* score, const int* count, int stride, int L, int K,
+                                 int* out_codes, float* out_score, int* out_count) {
+  const int b = blockIdx.x;
+  const int cnt = min(count[b], K);
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    const long long s = (long long)b * stride + k;
+    out_score[(long long)b * K + k] = k < cnt ? score[s] : -INFINITY;
+    for (int l = 0; l < L; ++l) out_codes[((long long)b * K + k) * L + l] = k < cnt ? codes[s * L + l] : -1;
+  }
+  if (threadIdx.x == 0) out_count[b] = cnt;
+}
+
+// dst[b, r, :] = src[row(b, r), col_off : col_off + T],
+// row = row_index ? row_index[b*idx_stride + r] : b*row_mul + r*beam_mul
+__global__ void copy_logits_kernel(const float* src, long long row_stride, int col_off, const int* row_index, int row_mul,
+                                   int beam_mul, int n_beams, int idx_stride, int T, float* dst) {
+  const int b = blockIdx.x / n_beams, r = blockIdx.x % n_beams;
+  const long long row = row_index ? row_index[(long long)b * idx_stride + r] : (long long)b * row_mul + (long long)r * beam_mul;
+  if (row < 0) return;
+  for (int t = threadIdx.x; t < T; t += blockDim.x)
+    dst[(long long)blockIdx.x * T + t] = src[row * row_stride + col_off + t];
+}
+
+__global__ void trace_beams_kernel(EngineState e, int batch, int K, nezha_trace tr) {
+  const int b = blockIdx.x;
+  const int L = e.L;
+  for (int n = 1; n <= L; ++n) {
+    const int cnt = e.tb_count[n * e.Bmax + b];
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+      const long long s = lvl_bk(e, n, b, k);
+      const long long o = ((long long)(n - 1) * batch + b) * K + k;
+      if (tr.beam_scores) tr.beam_scores[o] = k < cnt ? e.tb_score[s] : -INFINITY;
+      if (tr.beams)
+        for (int l = 0; l < L; ++l) tr.beams[o * L + l] = (k < cnt && l < n) ? e.tb_codes[s * L + l] : -1;
+    }
+  }
+}
+
+}  // namespace
+
+void launch_fill_i32(int* p, long long n, int v, cudaStream_t st) {
+  if (n <= 0) return;
+  fill_i32_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, st>>>(p, n, v);
+}
+void launch_fill_f32(float* p, long long n, float v, cudaStream_t st) {
+  if (n <= 0) return;
+  fill_f32_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, st>>>(p, n, v);
+}
+void launch_init_decode(const EngineState& e, int batch, cudaStream_t st) {
+  init_decode_kernel<<<(batch + 127) / 128, 128, 0, st>>>(e, batch);
+}
+void launch_draft_init(const EngineState& e, int batch, int from_scratch, cudaStream_t st) {
+  draft_init_kernel<<<batch, 64, 0, st>>>(e, batch, from_scratch);
+}
+void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st) {
+  draft_set_kernel<<<batch, 64, 0, st>>>(e, batch, K, drafts, n_draft);
+}
+void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st) {
+  if (bf16) draft_x_kernel<__nv_bfloat16><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (__nv_bfloat16*)x);
+  else draft_x_kernel<float><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (float*)x);
+}
+void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
+                         cudaStream_t st) {
+  if (bf16)
+    trans_gather_kernel<__nv_bfloat16><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (const __nv_bfloat16*)embed,
+                                                                      (__nv_bfloat16*)A);
+  else trans_gather_kernel<float><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (const float*)embed, (float*)A);
+}
+void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st) {
+  nodes_count_kernel<<<batch, 64, 0, st>>>(e, batch);
+  nodes_fill_kernel<<<batch, 128, 0, st>>>(e, batch);
+}
+void launch_nodes_from_prefixes(const EngineState& e, int batch, int n_beams, int level, const int* prefixes,
+                                cudaStream_t st) {
+  nodes_from_prefixes_kernel<<<batch, 128, 0, st>>>(e, batch, n_beams, level, prefixes);
+}
+void launch_advance(const EngineState& e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count,
+                    cudaStream_t st) {
+  advance_kernel<<<batch, 64, 0, st>>>(e, batch, n, K, out_codes, out_score, out_count);
+}
+void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, cudaStream_t st) {
+  round_end_kernel<<<batch, 64, 0, st>>>(e, batch, K, round, tr, 0);
+}
+void launch_write_out(const int* codes, const float* score, const int* count, int stride, int L, int batch, int K,
+                      int* out_codes, float* out_score, int* out_count, cudaStream_t st) {
+  write_out_kernel<<<batch, 64, 0, st>>>(codes, score, count, stride, L, K, out_codes, out_score, out_count);
+}
+void launch_copy_logits(const float* src, long long row_stride, int col_off, const int* row_index, int row_mul,
+                        int beam_mul, int batch, int n_beams, int idx_stride, int T, float* dst, cudaStream_t st) {
+  copy_logits_kernel<<<batch * n_beams, 128, 0, st>>>(src, row_stride, col_off, row_index, row_mul, beam_mul, n_beams,
+                                                      idx_stride, T, dst);
+}
+
+// Prompt tokens of a chunk of requests: [BOS, history codes item by item, SP_1..SP_L], padded with BOS up to
+// S_call positions (padding sits after the real tokens, so causal attention never shows it to them).
+__global__ void prefill_tokens_kernel(EngineState e, const int* hist, const int* n_hist, int b0, int rows, int max_n,
+                                      int S_call, int S_cap, int* h_rows) {
+  const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (idx >= (long long)rows * S_call) return;
+  const int lb = (int)(idx / S_call), p = (int)(idx % S_call), b = b0 + lb;
+  const int L = e.L;
+  int nh = n_hist[b];
+  if (nh < 0 || nh > max_n) { atomicOr(e.status, kStBadCode); nh = nh < 0 ? 0 : max_n; }
+  const int P = 1 + nh * L;
+  const int bos = e.li.vocab_codes + L;
+  int tok = bos;
+  if (p > 0 && p < P) {
+    const int item = (p - 1) / L, lv = (p - 1) % L;
+    int code = hist[((long long)b * max_n + item) * L + lv];
+    if (code < 0 || code >= e.li.T[lv]) { atomicOr(e.status, kStBadCode); code = 0; }
+    tok = e.li.off[lv] + code;
+  } else if (p >= P && p < P + L) {
+    tok = e.li.vocab_codes + (p - P);
+  }
+  e.tok_id[idx] = tok; e.tok_pos[idx] = p; e.tok_row[idx] = b; e.tok_ctx_len[idx] = p + 1;
+  e.tok_kv_dst[idx] = ((long long)b * e.Hkv * S_cap + p) * e.hd;
+  if (p == 0) e.row_P[b] = P;
+  if (p >= P - 1 && p <= P - 1 + L) h_rows[lb * (L + 1) + (p - (P - 1))] = (int)idx;
+}
+
+void launch_prefill_tokens(const EngineState& e, const int* hist, const int* n_hist, int b0, int rows, int max_n,
+                           int S_call, int S_cap, int* h_rows, cudaStream_t st) {
+  const long long n = (long long)rows * S_call;
+  prefill_tokens_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(e, hist, n_hist, b0, rows, max_n, S_call, S_cap, h_rows);
+}
+void launch_trace_beams(const EngineState& e, int batch, int K, const nezha_trace& tr, cudaStream_t st) {
+  trace_beams_kernel<<<batch, 64, 0, st>>>(e, batch, K, tr);
+}
+
+}  // namespace nz

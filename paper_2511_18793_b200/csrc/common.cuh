@@ -1,0 +1,157 @@
+// Shared declarations of the decode library's translation units (device helpers, argument structs,
+// kernel launchers).  Everything here is internal; the public surface is include/nezha.h.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "nezha.h"
+
+namespace nz {
+
+constexpr int kMaxLevels = NEZHA_MAX_LEVELS;
+constexpr int kBucketSlots = 4;                  // 4 x 8 B = one 32-byte sector per bucket
+constexpr unsigned long long kEmptyKey = ~0ull;  // never a packed key: prod(T) < 2^64 - 1
+constexpr int kMaxProbeBuckets = 4096;           // bound of every probe / insert walk
+
+// bits of the device status word
+enum : int { kStHashFull = 1, kStBadCode = 2, kStInternal = 4 };
+
+// --------------------------------------------------------------------------------------------------
+// small device helpers
+// --------------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// --------------------------------------------------------------------------------------------------
+// hash set (Eq. 5): open addressing over 4-slot buckets, linear probing over buckets
+// --------------------------------------------------------------------------------------------------
+struct HashSetView {
+  unsigned long long* slots;       // [n_buckets * kBucketSlots]
+  unsigned long long n_buckets;
+};
+
+// 64-bit finalizer (the published murmur3 fmix64 constants), then multiply-shift range reduction so that
+// any bucket count works (no power-of-two requirement).
+__device__ __forceinline__ unsigned long long hs_mix(unsigned long long k) {
+  k ^= k >> 33; k *= 0xff51afd7ed558ccdull; k ^= k >> 33; k *= 0xc4ceb9fe1a85ec53ull; k ^= k >> 33;
+  return k;
+}
+__device__ __forceinline__ unsigned long long hs_bucket(unsigned long long key, unsigned long long n_buckets) {
+  return __umul64hi(hs_mix(key), n_buckets);
+}
+
+// One thread walks the probe sequence alone, a whole bucket (one sector) per step.
+__device__ __forceinline__ bool hs_contains_thread(const HashSetView& hs, unsigned long long key) {
+  unsigned long long b = hs_bucket(key, hs.n_buckets);
+  for (int step = 0; step < kMaxProbeBuckets; ++step) {
+    const ulonglong2* p = reinterpret_cast<const ulonglong2*>(hs.slots + b * kBucketSlots);
+    ulonglong2 lo = __ldg(p), hi = __ldg(p + 1);
+    if (lo.x == key || lo.y == key || hi.x == key || hi.y == key) return true;
+    if (lo.x == kEmptyKey || lo.y == kEmptyKey || hi.x == kEmptyKey || hi.y == kEmptyKey) return false;
+    if (++b == hs.n_buckets) b = 0;
+  }
+  return false;
+}
+
+// --------------------------------------------------------------------------------------------------
+// model / engine description shared by the host code and the kernels
+// --------------------------------------------------------------------------------------------------
+struct LevelInfo {
+  int L;
+  int T[kMaxLevels];
+  int off[kMaxLevels];             // vocabulary offset of each level's codes
+  unsigned long long mult[kMaxLevels];   // Eq. 4 positional multipliers
+  int vocab_codes;                 // sum(T)
+};
+
+// Eq. 4 on a code tuple held in registers / local memory.
+__device__ __forceinline__ unsigned long long pack_key(const LevelInfo& li, const int* codes) {
+  unsigned long long k = 0;
+  for (int l = 0; l < li.L; ++l) k += (unsigned long long)codes[l] * li.mult[l];
+  return k;
+}
+
+// --------------------------------------------------------------------------------------------------
+// GEMM:  C[M,N] (op)= A[M,K] * W[N,K]^T   (both operands K-major)
+// --------------------------------------------------------------------------------------------------
+enum GemmEpilogue : int {
+  kEpiStoreAct = 0,     // C (activation type) = acc
+  kEpiStoreF32 = 1,     // C (float) = acc
+  kEpiAddF32 = 2,       // C (float) += acc                    (residual stream)
+  kEpiBiasTanhF32 = 3,  // C (float) = tanh(acc + bias[n])     (Eq. 3)
+  kEpiSwiGLU = 4        // C (activation type)[m, n/2] = silu(acc[m, n]) * acc[m, n+1] on interleaved columns
+};
+
+struct GemmArgs {
+  const void* A; long long lda;
+  const void* W; long long ldw;
+  void* C; long long ldc;
+  int M;                 // upper bound of rows (grid is sized for it)
+  const int* M_dev;      // optional: actual row count on the device (<= M); rows beyond are skipped
+  int N, K;
+  int epilogue;
+  const float* bias;
+};
+
+void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);
+
+// --------------------------------------------------------------------------------------------------
+// element-wise / glue kernels
+// --------------------------------------------------------------------------------------------------
+void launch_embed(const void* table, bool bf16, const int* tokens, int M, const int* M_dev, int d, float* resid,
+                  cudaStream_t st);
+void launch_rmsnorm(const float* x, long long x_stride, const int* row_index, const void* gain, bool bf16, void* out,
+                    float* out_f32, int M, const int* M_dev, int d, float eps, cudaStream_t st);
+
+struct RopeAppendArgs {
+  void* qkv;                       // [M, (Hq + 2 Hkv) * hd], activation type; q and k rotated in place
+  const int* tok_pos;              // [M] rotary position
+  const long long* kv_dst;         // [M] element offset of the token's K (and V) row group in the layer's cache:
+                                   //     token's head h row starts at kv_dst[i] + h * kv_head_stride
+  long long kv_head_stride;
+  void* k_cache; void* v_cache;    // layer base pointers
+  const float* cos_tab; const float* sin_tab;   // [positions, hd/2]
+  int M; const int* M_dev;
+  int Hq, Hkv, hd;
+};
+void launch_rope_append(const RopeAppendArgs& a, bool bf16, cudaStream_t st);
+void launch_swiglu(const void* gu, void* act, int M, const int* M_dev, int F, bool bf16, cudaStream_t st);
+
+// --------------------------------------------------------------------------------------------------
+// attention over (context KV prefix) + (a few extra KV rows per token)
+// --------------------------------------------------------------------------------------------------
+struct AttnArgs {
+  const void* q; long long q_stride;        // token i, head h at q + i*q_stride + h*hd
+  void* out; long long out_stride;          // [M, Hq*hd]
+  const void* k_ctx; const void* v_ctx;     // layer base of the context cache [rows][Hkv][S][hd]
+  long long ctx_row_stride, ctx_head_stride;// element strides (row = request, head = kv head)
+  const void* k_ext; const void* v_ext;     // layer base of the draft-token cache
+  long long ext_head_stride;                // element stride between kv heads inside one extra entry
+  const int* tok_row;                       // [M] request (cache row) of the token
+  const int* tok_ctx_len;                   // [M] number of context positions visible
+  const long long* tok_ext;                 // [M, n_ext_max] element offsets of extra KV entries, -1 = unused
+  int n_ext_max;
+  int M; const int* M_dev;
+  int Hq, Hkv, hd;
+  float scale;
+};
+void launch_attention_simt(const AttnArgs& a, bool bf16, cudaStream_t st);
+
+}  // namespace nz

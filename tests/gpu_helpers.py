@@ -1,0 +1,86 @@
+"""Helpers of the GPU parity tests: build an engine and the oracle objects from the same seeded inputs."""
+import numpy as np
+import torch
+
+from oracle import nezha_oracle as O
+from paper_2511_18793_b200 import synth
+from helpers import oracle_bundle
+
+
+def tolerance(w):
+    """Absolute tolerance on logits: 1e-4 for the fp32 configuration, 2e-2 for bf16 storage."""
+    return 1e-4 if w.dtype == "fp32" else 2e-2
+
+
+class Case:
+    """Engine + oracle on one workload.  Weights are drawn once and handed to both sides as the same bytes."""
+
+    def __init__(self, w, device="cuda", max_beam=None, catalog=None, hist=None, weights=None, oracle_rows=None):
+        from paper_2511_18793_b200 import binding
+        self.binding = binding
+        self.w = w
+        self.dev = device
+        self.weights = weights if weights is not None else synth.make_weights(w, device=device)
+        self.catalog = synth.make_catalog(w) if catalog is None else catalog
+        self.hist = synth.make_histories(w, self.catalog) if hist is None else hist
+        self.cat_dev = torch.from_numpy(self.catalog).to(device)
+        cfg = binding.make_config(w, max_batch=self.hist.shape[0], max_beam=max_beam or w.beam,
+                                  max_hist_items=self.hist.shape[1])
+        self.eng = binding.Engine(cfg, self.weights, self.cat_dev, load_factor=w.load_factor)
+        self.n_unique = self.eng.build_hashset()
+        self.hist_dev = torch.from_numpy(self.hist).to(device)
+        self.n_hist = torch.full((self.hist.shape[0],), self.hist.shape[1], dtype=torch.int32, device=device)
+        self._oracle = None
+        self._reqs = {}
+
+    def prefill(self):
+        self.eng.prefill(self.hist_dev, self.n_hist)
+        return self
+
+    @property
+    def oracle(self):
+        if self._oracle is None:
+            Wn = synth.weights_to_numpy(self.weights)
+            big = self.w.d_model * self.w.d_ffn * self.w.n_layers > 2e8
+            self._oracle = oracle_bundle(self.w, Wn, self.catalog, cache_f64=not big)
+        return self._oracle
+
+    def req(self, b, n_items=None):
+        key = (b, n_items)
+        if key not in self._reqs:
+            model = self.oracle[0]
+            h = self.hist[b] if n_items is None else self.hist[b, :n_items]
+            self._reqs[key] = model.prefill(h)
+        return self._reqs[key]
+
+
+def assert_topk_matches(gpu_codes, gpu_scores, gpu_count, oracle_beams, K, tol, all_scored=None):
+    """Top-k comparison with the tie rule: identical when scores are separated by more than `tol`; where the
+    oracle's scores tie within tol around the K-th place, either choice is accepted.
+    Returns True if the two lists are identical item for item."""
+    o_codes = [b.codes for b in oracle_beams]
+    o_scores = np.asarray([float(b.score) for b in oracle_beams], dtype=np.float64)
+    g_codes = [tuple(int(c) for c in gpu_codes[k] if c >= 0) for k in range(int(gpu_count))]
+    assert int(gpu_count) == len(o_codes), (int(gpu_count), len(o_codes))
+    assert all(np.all(gpu_codes[k] == -1) for k in range(int(gpu_count), K))
+    assert all(np.isneginf(gpu_scores[k]) for k in range(int(gpu_count), K))
+    if g_codes == o_codes:
+        assert np.allclose(gpu_scores[: len(o_codes)], o_scores, atol=tol * max(1, len(o_codes[0]) if o_codes else 1))
+        return True
+    # not identical: every disagreement must be explained by near-ties
+    g_set, o_set = set(g_codes), set(o_codes)
+    kth = o_scores[-1] if len(o_scores) else -np.inf
+    L = len(o_codes[0]) if o_codes else 1
+    slack = tol * L
+    o_map = dict(zip(o_codes, o_scores))
+    for t in o_set - g_set:            # oracle members the GPU dropped: must be within slack of the K-th score
+        assert o_map[t] <= kth + 2 * slack, ("dropped a clear winner", t, o_map[t], kth)
+    g_map = dict(zip(g_codes, [float(s) for s in gpu_scores[: len(g_codes)]]))
+    for t in g_set - o_set:            # GPU members the oracle did not keep: their GPU score must be near the K-th
+        assert g_map[t] >= kth - 2 * slack, ("kept a clear loser", t, g_map[t], kth)
+    for t in g_set & o_set:
+        assert abs(g_map[t] - o_map[t]) <= slack, (t, g_map[t], o_map[t])
+    # order: GPU scores non-increasing
+    gs = np.asarray([g_map[t] for t in g_codes])
+    assert np.all(gs[:-1] >= gs[1:] - 1e-6)
+    return False

@@ -1,0 +1,259 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nezha_oracle as O
+from paper_2511_18793_b200 import synth
+from helpers import codes_of
+from gpu_helpers import Case, assert_topk_matches, tolerance
+
+pytestmark = pytest.mark.gpu
+
+
+def _as_u64(t):
+    return t.cpu().numpy().view(np.uint64)
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    return Case(synth.WORKLOADS["tiny"]).prefill()
+
+
+# ---------------------------------------------------------------------------------------- hash set
+@pytest.mark.parametrize("name,n_items", [("tiny", None), ("small", 200_000)])
+def test_hashset_build_and_probe_bit_exact(name, n_items):
+    w = synth.WORKLOADS[name]
+    if n_items:
+        w = synth.scaled(w, n_items=n_items, n_layers=1, batch=2, n_hist=2)
+    cat = synth.make_catalog(w)
+    cat_dup = np.concatenate([cat, cat[: len(cat) // 10]])            # duplicated tuples are counted once
+    case = Case(w, catalog=cat_dup)
+    V = O.ValidSet(cat, w.T)
+    assert case.n_unique == len(V) == len(cat)
+    dev = case.dev
+    # Eq. 4: keys bit-identical
+    probe_codes = synth.probe_keys_mix(w, cat, 100_000)
+    keys = case.eng.pack(torch.from_numpy(probe_codes).to(dev))
+    assert np.array_equal(_as_u64(keys), O.pack_keys(probe_codes, w.T))
+    # Eq. 5: (i) every catalogue key, (ii) a hit/miss mix, (iii) siblings of catalogue prefixes
+    found = case.eng.probe(case.eng.pack(torch.from_numpy(cat).to(dev)))
+    assert bool(found.all())
+    found = case.eng.probe(keys).cpu().numpy().astype(bool)
+    assert np.array_equal(found, V.contains(probe_codes))
+    pre = cat[np.random.default_rng(0).integers(0, len(cat), 500)]
+    sib = np.repeat(pre, w.T[-1], axis=0)
+    sib[:, -1] = np.tile(np.arange(w.T[-1]), len(pre))
+    found = case.eng.probe(case.eng.pack(torch.from_numpy(sib.astype(np.int32)).to(dev))).cpu().numpy().astype(bool)
+    assert np.array_equal(found, V.contains(sib))
+    assert found.sum() >= len(pre)
+    # empty probe is a no-op
+    assert case.eng.probe(torch.empty(0, dtype=torch.int64, device=dev)).numel() == 0
+
+
+def test_error_paths(tiny):
+    b = tiny.binding
+    w = tiny.w
+    # out-of-range catalogue code
+    bad = tiny.catalog.copy(); bad[7, 1] = w.T[1]
+    c2 = None
+    with pytest.raises(b.NezhaError) as ei:
+        c2 = Case(w, catalog=bad)
+    assert ei.value.status == 6
+    # decode before prefill, wrong batch, beam too wide
+    c3 = Case(w)
+    with pytest.raises(b.NezhaError) as ei:
+        c3.eng.batch = w.batch
+        c3.eng.decode(w.beam)
+    assert ei.value.status == 2
+    with pytest.raises(b.NezhaError) as ei:
+        tiny.eng.decode(w.beam + 1)
+    assert ei.value.status == 1
+    # arena too small
+    import ctypes as C
+    cfg = b.make_config(w)
+    h = C.c_void_p()
+    wts = b.NezhaWeights()
+    arena = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    st = b.lib.nezha_create(C.byref(cfg), C.byref(wts), tiny.cat_dev.data_ptr(), 5000, 0.5, arena.data_ptr(), 1024, None,
+                            C.byref(h))
+    assert st == 3
+    # a history code out of range is reported by the next synchronising call
+    hist = tiny.hist.copy(); hist[0, 0, 0] = 99
+    c3.eng.prefill(torch.from_numpy(hist).cuda(), c3.n_hist)
+    with pytest.raises(b.NezhaError) as ei:
+        c3.eng.sync()
+    assert ei.value.status == 6
+
+
+# ---------------------------------------------------------------------------------------- stage-wise FP parity
+def test_prefill_hidden_states(tiny):
+    h = tiny.eng.get_hidden().cpu().numpy()
+    for b in range(tiny.w.batch):
+        assert np.abs(h[b] - tiny.req(b).h).max() < 2e-5
+
+
+def test_primary_logits_teacher_forced(tiny):
+    w = tiny.w
+    model = tiny.oracle[0]
+    rng = np.random.default_rng(3)
+    for level in range(w.L):
+        nb = w.beam
+        pre = np.stack([rng.integers(0, w.T[l], size=(w.batch, nb)) for l in range(level)], axis=2).astype(np.int32) \
+            if level else None
+        got = tiny.eng.primary_logits(nb, level, None if pre is None else torch.from_numpy(pre).cuda()).cpu().numpy()
+        for b in range(w.batch):
+            ref = model.next_level_logits_many(tiny.req(b), [tuple(pre[b, r]) if level else () for r in range(nb)])
+            assert np.abs(got[b] - np.stack(ref)).max() < tolerance(w)
+
+
+def test_draft_logits_teacher_forced(tiny):
+    w = tiny.w
+    head = tiny.oracle[1]
+    rng = np.random.default_rng(4)
+    for level in range(w.L):
+        nb = w.beam
+        pre = np.stack([rng.integers(0, w.T[l], size=(w.batch, nb)) for l in range(level)], axis=2).astype(np.int32) \
+            if level else None
+        got = tiny.eng.draft_logits(nb, level, None if pre is None else torch.from_numpy(pre).cuda()).cpu().numpy()
+        for b in range(w.batch):
+            req = tiny.req(b)
+            for r in range(nb):
+                st = O.teacher_forced_state(head, req, tuple(pre[b, r]) if level else ())
+                ref = head.logits(level, req.h[level + 1], st)
+                assert np.abs(got[b, r] - ref).max() < tolerance(w)
+
+
+# ---------------------------------------------------------------------------------------- select (integer stage)
+@pytest.mark.parametrize("level,per_beam_all,filt", [(0, True, False), (1, True, False), (2, True, True), (2, False, True),
+                                                     (1, False, False)])
+def test_select_on_identical_logits(tiny, level, per_beam_all, filt):
+    w = tiny.w
+    V = tiny.oracle[2]
+    rng = np.random.default_rng(10 + level)
+    K = w.beam
+    nb = 1 if level == 0 else K
+    logits = rng.standard_normal((w.batch, nb, w.T[level])).astype(np.float32) * 2
+    scores = (-rng.random((w.batch, nb)) * 3).astype(np.float32)
+    if level == 2:                                   # prefixes that have valid completions
+        idx = rng.integers(0, len(tiny.catalog), size=(w.batch, nb))
+        codes = tiny.catalog[idx][:, :, :level].astype(np.int32)
+    else:
+        codes = np.stack([rng.integers(0, w.T[l], size=(w.batch, nb)) for l in range(level)], axis=2).astype(np.int32) \
+            if level else None
+    n_live = np.full((w.batch,), nb, dtype=np.int32); n_live[-1] = max(1, nb - 2)
+    per_beam = w.T[level] if per_beam_all else min(K, w.T[level])
+    parent, code, score, count = tiny.eng.select(
+        torch.from_numpy(logits).cuda(), torch.from_numpy(scores).cuda(),
+        None if codes is None else torch.from_numpy(codes).cuda(), torch.from_numpy(n_live).cuda(), K, level, per_beam, filt)
+    parent, code, score, count = [t.cpu().numpy() for t in (parent, code, score, count)]
+    for b in range(w.batch):
+        beams = [O.Beam(tuple(codes[b, r]) if level else (), np.float32(scores[b, r])) for r in range(n_live[b])]
+        ref = O.expand_level(beams, [logits[b, r].astype(np.float64) for r in range(n_live[b])], K, per_beam,
+                             V if filt else None)
+        assert count[b] == len(ref)
+        got = [(int(parent[b, k]), int(code[b, k])) for k in range(count[b])]
+        want = [(bm.parent, bm.codes[-1]) for bm in ref]
+        if got != want:       # only near-ties (fp32 vs fp64 log-softmax) may differ
+            gs, ws = score[b, : count[b]], np.asarray([float(x.score) for x in ref])
+            assert np.abs(np.sort(gs) - np.sort(ws)).max() < 1e-5
+            assert len(set(got) ^ set(want)) <= 2
+        else:
+            assert np.allclose(score[b, : count[b]], [float(x.score) for x in ref], atol=2e-6)
+        assert np.all(parent[b, count[b]:] == -1) and np.all(np.isneginf(score[b, count[b]:]))
+
+
+# ---------------------------------------------------------------------------------------- end to end, tiny (fp32)
+def test_mode_draft_equals_algorithm3(tiny):
+    w = tiny.w
+    head, V = tiny.oracle[1], tiny.oracle[2]
+    out = tiny.eng.decode(w.beam, mode=0)
+    codes, scores, count = [out[k].cpu().numpy() for k in ("codes", "scores", "count")]
+    for b in range(w.batch):
+        ref = O.nezha_draft(head, tiny.req(b), w.beam, V)[-1]
+        assert assert_topk_matches(codes[b], scores[b], count[b], ref, w.beam, tolerance(w))
+        assert V.contains(codes[b, : count[b]]).all()                      # zero hallucinations
+
+
+def test_mode_ar_equals_algorithm1(tiny):
+    w = tiny.w
+    model, _, V = tiny.oracle
+    out = tiny.eng.decode(w.beam, mode=2, trace=True)
+    codes, scores, count = [out[k].cpu().numpy() for k in ("codes", "scores", "count")]
+    beams = out["trace"]["beams"].cpu().numpy()
+    assert out["stats"].rounds == w.L - 1
+    for b in range(w.batch):
+        ref = O.ar_beam_search(model, tiny.req(b), w.beam, V)
+        assert assert_topk_matches(codes[b], scores[b], count[b], ref[-1], w.beam, tolerance(w))
+        for n in range(w.L):                                                # every intermediate beam set too
+            got = [tuple(int(c) for c in beams[n, b, k, : n + 1]) for k in range(len(ref[n]))]
+            assert got == codes_of(ref[n])
+        assert V.contains(codes[b, : count[b]]).all()
+
+
+def test_mode_verified_equals_ar_and_matches_oracle_trace(tiny):
+    w = tiny.w
+    model, head, V = tiny.oracle
+    out = tiny.eng.decode(w.beam, mode=1, trace=True)
+    ar = tiny.eng.decode(w.beam, mode=2)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])      # zero sacrifice
+    assert torch.allclose(out["scores"], ar["scores"], atol=1e-5)
+    codes, scores, count = [out[k].cpu().numpy() for k in ("codes", "scores", "count")]
+    tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+    tot_tokens, max_rounds = 0, 0
+    for b in range(w.batch):
+        sets, st = O.speculative_decode(model, head, tiny.req(b), w.beam, V)
+        assert assert_topk_matches(codes[b], scores[b], count[b], sets[-1], w.beam, tolerance(w))
+        for r in range(st.rounds):
+            nd = tr["n_draft"][r, b]
+            assert list(tr["accepted_len"][r, b, :nd]) == st.accepted_len[r]
+            assert tr["level_reached"][r, b] == st.reject_level[r]
+        assert np.all(tr["level_reached"][st.rounds:, b] == -1)
+        tot_tokens += st.primary_tokens
+        max_rounds = max(max_rounds, st.rounds)
+    assert out["stats"].primary_tokens == tot_tokens and out["stats"].rounds == max_rounds
+
+
+def test_decode_with_drafts_acceptance_regimes(tiny):
+    w = tiny.w
+    model, head, V = tiny.oracle
+    K = w.beam
+    ar = tiny.eng.decode(K, mode=2)
+    ar_codes = ar["codes"].cpu().numpy()
+    rng = np.random.default_rng(5)
+    for rho in (0.0, 0.5, 1.0):
+        drafts = ar_codes.copy()
+        n_draft = ar["count"].cpu().numpy().copy()
+        for b in range(w.batch):
+            for k in range(n_draft[b]):
+                if rng.random() < rho:
+                    lvl = int(rng.integers(0, w.L))
+                    drafts[b, k, lvl] = (drafts[b, k, lvl] + 1 + rng.integers(0, w.T[lvl] - 1)) % w.T[lvl]
+        out = tiny.eng.decode_with_drafts(K, torch.from_numpy(drafts).cuda(), torch.from_numpy(n_draft).cuda(), trace=True)
+        assert torch.equal(out["codes"], ar["codes"])                        # result never depends on the drafts
+        tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+        for b in range(w.batch):
+            D = [tuple(int(c) for c in drafts[b, k]) for k in range(n_draft[b])]
+            sets, st = O.speculative_decode(model, head, tiny.req(b), K, V, drafts_round1=D)
+            assert codes_of(sets[-1]) == [tuple(int(c) for c in ar_codes[b, k]) for k in range(len(sets[-1]))]
+            assert list(tr["accepted_len"][0, b, : n_draft[b]]) == st.accepted_len[0]
+            assert tr["level_reached"][0, b] == st.reject_level[0]
+            if rho == 0.0 and st.rounds == 1:
+                assert st.accepted_len[0] == [w.L] * n_draft[b]
+    # decode is repeatable from the same prefilled state
+    again = tiny.eng.decode(K, mode=1)
+    assert torch.equal(again["codes"], ar["codes"])
+
+
+def test_ragged_histories_and_small_beams():
+    w = synth.scaled(synth.WORKLOADS["tiny"], n_kv_heads=2, batch=3)
+    case = Case(w)
+    n_hist = torch.tensor([w.n_hist, 7, 0], dtype=torch.int32, device="cuda")
+    case.eng.prefill(case.hist_dev, n_hist)
+    model, head, V = case.oracle
+    for K in (1, 3):
+        out = case.eng.decode(K, mode=1)
+        codes, scores, count = [out[k].cpu().numpy() for k in ("codes", "scores", "count")]
+        for b, n in enumerate([w.n_hist, 7, 0]):
+            ref = O.ar_beam_search(model, case.req(b, n), K, V)[-1]
+            assert assert_topk_matches(codes[b], scores[b], count[b], ref, K, tolerance(w))
