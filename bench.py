@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative semantic-ID decode step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload small] [--mode 1] [--impl ours|reference]
+
+One step = one nezha_decode call (draft head -> hash-set filter -> primary verify pass -> masked log-softmax /
+beam top-k -> accept / roll back, all rounds) over the whole batch, always from the same prefilled state.
+Prints ONE JSON line.  `value` = items (batch x beam) decoded per second with all inputs resident in HBM;
+`e2e` = the same through the C ABI starting from pinned HOST histories (H2D copy + prefill + decode + D2H of
+the results inside the timed region).  With N > 1 (torchrun) every rank runs an independent replica on its own
+GPU -- requests are independent, so there is no collective on the data path -- and `value` sums the replicas.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+METRIC, UNIT = "items_per_s_decoded", "items/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of one GPU, sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, weights_np, catalog, hist, mode, budget_s=20.0, max_rows=None):
+    """The CPU oracle, as it stands, on the first rows of the workload until ~budget_s of work is done."""
+    import numpy as np
+    from oracle import nezha_oracle as O
+    shape = O.ModelShape(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.d_ffn, w.L, tuple(w.T), w.rope_theta, w.rms_eps)
+    big = w.d_model * w.d_ffn * w.n_layers > 2e8
+    model = O.PrimaryModel(shape, weights_np, cache_f64=not big)
+    head, valid = O.DraftHead(shape, weights_np), O.ValidSet(catalog, w.T)
+    rows, t_decode, t_prefill = 0, 0.0, 0.0
+    limit = hist.shape[0] if max_rows is None else min(max_rows, hist.shape[0])
+    while rows < limit and (t_decode + t_prefill) < budget_s:
+        t0 = time.perf_counter()
+        req = model.prefill(hist[rows])
+        t1 = time.perf_counter()
+        if mode == 0:
+            O.nezha_draft(head, req, w.beam, valid)
+        elif mode == 2:
+            O.ar_beam_search(model, req, w.beam, valid)
+        else:
+            O.speculative_decode(model, head, req, w.beam, valid)
+        t2 = time.perf_counter()
+        t_prefill += t1 - t0
+        t_decode += t2 - t1
+        rows += 1
+    return {"rows": rows, "decode_s": t_decode, "prefill_s": t_prefill,
+            "items_per_s": rows * w.beam / t_decode if t_decode > 0 else 0.0}
+
+
+def algorithmic_work(w, stats_tokens_per_step, rounds):
+    """Algorithmic flops / bytes of one decode step, per kernel class (the per-unit figures are in the design doc)."""
+    esz = 4 if w.dtype == "fp32" else 2
+    d, hd, Hq, Hkv, F, nl = w.d_model, w.head_dim, w.n_q_heads, w.n_kv_heads, w.d_ffn, w.n_layers
+    per_tok_params = nl * ((Hq + 2 * Hkv) * hd * d + d * Hq * hd + 3 * F * d)
+    lm = sum(w.T[1:]) * d
+    gemm_flops = 2.0 * stats_tokens_per_step * (per_tok_params + lm)
+    P = w.ctx_tokens
+    # attention: the context KV of a request is read once per (request, layer, pass); queries and outputs once
+    attn_bytes = rounds * nl * w.batch * (2 * Hkv * P * hd * esz) + stats_tokens_per_step * nl * 2 * Hq * hd * esz
+    attn_flops = 4.0 * stats_tokens_per_step * nl * Hq * hd * (P + 2)
+    return {"gemm_flops": gemm_flops, "attention_bytes": attn_bytes, "attention_flops": attn_flops}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="small")
+    ap.add_argument("--mode", type=int, default=1, help="0 draft-only, 1 verified (default), 2 plain autoregressive")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget-s", type=float, default=20.0)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import numpy as np
+    import torch
+    from paper_2511_18793_b200 import synth
+
+    w = synth.WORKLOADS[args.workload]
+    config = {"workload": f"{w.name}: {w.n_layers}L d{w.d_model} {w.n_q_heads}q/{w.n_kv_heads}kv ffn{w.d_ffn}, "
+                          f"L={w.L} T={w.T[0]}, catalogue {w.n_items} ({w.catalog}), history {w.n_hist} items, "
+                          f"batch {w.batch} x beam {w.beam}, seed {w.seed}",
+              "mode": {0: "draft-only (Algorithm 3)", 1: "verified (Algorithm 2)", 2: "autoregressive (Algorithm 1)"}[args.mode],
+              "batch": w.batch, "beam": w.beam, "l2": "flushed between steps (256 MB write, outside the timed events)",
+              "drafts": "natural (random-init draft head)"}
+
+    # ------------------------------------------------------------------ reference arm: the oracle on host cores
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        weights = synth.make_weights(w, device="cpu")
+        catalog = synth.make_catalog(w)
+        hist = synth.make_histories(w, catalog)
+        Wn = synth.weights_to_numpy(weights)
+        per_step = max(2.0, min(args.cpu_budget_s, 120.0 / max(1, args.steps + args.warmup)))
+        vals, rows = [], 0
+        for i in range(args.warmup + args.steps):
+            r = oracle_sample(w, Wn, catalog, hist, args.mode, budget_s=per_step, max_rows=4)
+            if i >= args.warmup:
+                vals.append(r["items_per_s"]); rows = r["rows"]
+        v = statistics.mean(vals)
+        cores = os.cpu_count()
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * rows * w.beam / v if v else None,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic", "config": config,
+                          "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                           "sample": f"decode of the first {rows} request(s) of the batch per step, prefill excluded"},
+                          "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    # ------------------------------------------------------------------ our arm
+    from paper_2511_18793_b200 import binding
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    weights = synth.make_weights(w, device=dev)
+    catalog = synth.make_catalog(w)
+    hist = synth.make_histories(w, catalog)
+    cat_dev = torch.from_numpy(catalog).to(dev)
+    eng = binding.Engine(binding.make_config(w), weights, cat_dev, w.load_factor, stream=torch.cuda.current_stream())
+    n_unique = eng.build_hashset()
+    assert n_unique == w.n_items
+    hist_pinned = torch.from_numpy(hist).pin_memory()
+    nh_pinned = torch.full((w.batch,), w.n_hist, dtype=torch.int32).pin_memory()
+    hist_dev = hist_pinned.to(dev, non_blocking=True)
+    nh_dev = nh_pinned.to(dev, non_blocking=True)
+    eng.prefill(hist_dev, nh_dev)
+    out = eng.alloc_outputs(w.batch, w.beam)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    items = w.batch * w.beam
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        return eng.decode(w.beam, mode=args.mode, out=out)
+
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = binding.lib.nezha_launch_count()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    tokens = rounds = 0
+    for a, b in evs:
+        flush.fill_(1)
+        a.record()
+        r = step()
+        b.record()
+        tokens += r["stats"].primary_tokens
+        rounds += r["stats"].rounds
+    barrier()
+    launches = binding.lib.nezha_launch_count() - launches0
+    clocks = sampler.stop()
+    per_step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = sum(per_step_ms)
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    value = world * items * args.steps / (total_ms_max / 1e3)
+
+    # ---- end to end from pinned host memory: H2D histories, prefill, decode, D2H results
+    host_codes = torch.empty(w.batch, w.beam, w.L, dtype=torch.int32).pin_memory()
+    host_scores = torch.empty(w.batch, w.beam, dtype=torch.float32).pin_memory()
+    host_count = torch.empty(w.batch, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        hd = hist_pinned.to(dev, non_blocking=True)
+        nd = nh_pinned.to(dev, non_blocking=True)
+        eng.prefill(hd, nd)
+        step()
+        host_codes.copy_(out["codes"], non_blocking=True)
+        host_scores.copy_(out["scores"], non_blocking=True)
+        host_count.copy_(out["count"], non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record()
+    barrier()
+    e2e_ms = max(ea.elapsed_time(eb), 0.0)
+    te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * items * e2e_steps / (float(te.item()) / 1e3)
+    h2d = hist_pinned.numel() * 4 + nh_pinned.numel() * 4
+    d2h = host_codes.numel() * 4 + host_scores.numel() * 4 + host_count.numel() * 4
+
+    # ---- per-kernel-class CUDA-event timing (separate pass: two event records per launch perturb throughput)
+    eng.prefill(hist_dev, nh_dev)
+    eng.profile_enable(True)
+    eng.profile_read()
+    prof_steps = max(3, min(args.steps, 10))
+    ptok = prd = 0
+    for _ in range(prof_steps):
+        flush.fill_(1)
+        r = step()
+        ptok += r["stats"].primary_tokens
+        prd += r["stats"].rounds
+    prof = eng.profile_read()
+    eng.profile_enable(False)
+    peaks = load_peaks()
+    work = algorithmic_work(w, ptok / prof_steps, prd / prof_steps)
+    tot_prof_ms = sum(v["ms"] for v in prof.values()) or 1.0
+    shares = {k: {"launches_per_step": v["launches"] / prof_steps, "ms_per_step": v["ms"] / prof_steps,
+                  "share": v["ms"] / tot_prof_ms} for k, v in prof.items() if v["launches"]}
+    dom = max(shares, key=lambda k: shares[k]["ms_per_step"])
+    roof = {"kernel": dom, "bound": None, "achieved": None, "peak": None, "unit": None, "frac": None, "traffic": None,
+            "of": peaks["source"]}
+    dom_s = shares[dom]["ms_per_step"] / 1e3
+    if dom == "gemm":
+        ach = work["gemm_flops"] / dom_s / 1e12
+        peak = peaks["bf16_tflops_sustained"] if w.dtype == "bf16" else 75.0
+        roof.update(bound="tensor" if w.dtype == "bf16" else "alu", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
+    elif dom == "attention":
+        ach = work["attention_bytes"] / dom_s / 1e9
+        roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+    else:
+        roof.update(bound="latency", note="dominant class is neither GEMM nor attention")
+    roof["classes"] = shares
+    roof["attention_gbs"] = work["attention_bytes"] / (shares["attention"]["ms_per_step"] / 1e3) / 1e9 if "attention" in shares else None
+    roof["gemm_tflops"] = work["gemm_flops"] / (shares["gemm"]["ms_per_step"] / 1e3) / 1e12 if "gemm" in shares else None
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms_max / args.steps, "p50_ms": statistics.median(per_step_ms),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
+            "clocks": clocks, "gpu_launches": int(launches),
+            "rounds_per_step": rounds / args.steps, "primary_tokens_per_step": tokens / args.steps,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "includes": "H2D histories + prefill + decode + D2H results", "steps": e2e_steps},
+            "roofline": roof}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        Wn = synth.weights_to_numpy(weights)
+        r = oracle_sample(w, Wn, catalog, hist, args.mode, budget_s=args.cpu_budget_s)
+        line["cpu_baseline"] = {"value": r["items_per_s"], "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"decode of the first {r['rows']} request(s) of the batch "
+                                          f"({r['decode_s']:.1f} s; their prefill, {r['prefill_s']:.1f} s, excluded)"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

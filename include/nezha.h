@@ -196,6 +196,26 @@ nezha_status nezha_select(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_
                           const int32_t* n_live,
                           int32_t* out_parent, int32_t* out_code, float* out_score, int32_t* out_count);
 
+/* ---- instrumentation (the paper has no counterpart: these only measure the library itself) -------------- */
+
+#define NEZHA_PROFILE_CLASSES 16
+/* Kernel classes, in index order: gemm, attention, select, norm, rope_append, embed, swiglu, draft_glue, nodes,
+ * accept, hash, misc. */
+typedef struct {
+  int64_t launches[NEZHA_PROFILE_CLASSES];   /* kernels launched per class since the last read                 */
+  double  ms[NEZHA_PROFILE_CLASSES];         /* summed CUDA-event time per class (0 unless timing was enabled) */
+} nezha_profile;
+
+/* Total kernels this library has launched in the process (all contexts).  Never fails. */
+uint64_t nezha_launch_count(void);
+
+/* Turn per-launch CUDA-event timing on (1) or off (0).  Timing adds two event records per launch, so measure
+ * throughput with it off.  Synchronises. */
+nezha_status nezha_profile_enable(nezha_ctx* ctx, int32_t on);
+
+/* Synchronise, copy out and reset the per-class launch counts and event times (host struct). */
+nezha_status nezha_profile_read(nezha_ctx* ctx, nezha_profile* out);
+
 /* Wait for the context's stream and report any pending device-side error. */
 nezha_status nezha_sync(nezha_ctx* ctx);
 

@@ -78,6 +78,18 @@ lib.nezha_draft_logits.restype = C.c_int
 lib.nezha_draft_logits.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp]
 lib.nezha_select.restype = C.c_int
 lib.nezha_select.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+class NezhaProfile(C.Structure):
+    _fields_ = [("launches", C.c_int64 * 16), ("ms", C.c_double * 16)]
+
+
+PROFILE_CLASSES = ["gemm", "attention", "select", "norm", "rope_append", "embed", "swiglu", "draft_glue", "nodes",
+                   "accept", "hash", "misc"]
+lib.nezha_launch_count.restype = C.c_uint64
+lib.nezha_launch_count.argtypes = []
+lib.nezha_profile_enable.restype = C.c_int
+lib.nezha_profile_enable.argtypes = [_vp, _i32]
+lib.nezha_profile_read.restype = C.c_int
+lib.nezha_profile_read.argtypes = [_vp, C.POINTER(NezhaProfile)]
 lib.nezha_sync.restype = C.c_int
 lib.nezha_sync.argtypes = [_vp]
 lib.nezha_last_error.restype = C.c_char_p
@@ -87,7 +99,8 @@ lib.nezha_destroy.argtypes = [_vp]
 
 EXPORTS = ["nezha_arena_bytes", "nezha_create", "nezha_build_hashset", "nezha_pack", "nezha_probe", "nezha_prefill",
            "nezha_decode", "nezha_decode_with_drafts", "nezha_get_hidden", "nezha_primary_logits",
-           "nezha_draft_logits", "nezha_select", "nezha_sync", "nezha_last_error", "nezha_destroy"]
+           "nezha_draft_logits", "nezha_select", "nezha_launch_count", "nezha_profile_enable",
+           "nezha_profile_read", "nezha_sync", "nezha_last_error", "nezha_destroy"]
 
 
 class NezhaError(RuntimeError):
@@ -275,6 +288,14 @@ class Engine:
                                      _ptr(logits.contiguous()), _ptr(beam_scores.contiguous()), _ptr(bc),
                                      _ptr(n_live.contiguous()), _ptr(parent), _ptr(code), _ptr(score), _ptr(count)))
         return parent, code, score, count
+
+    def profile_enable(self, on: bool):
+        self._check(lib.nezha_profile_enable(self._h, 1 if on else 0))
+
+    def profile_read(self) -> Dict[str, Dict[str, float]]:
+        p = NezhaProfile()
+        self._check(lib.nezha_profile_read(self._h, C.byref(p)))
+        return {name: {"launches": int(p.launches[i]), "ms": float(p.ms[i])} for i, name in enumerate(PROFILE_CLASSES)}
 
     def sync(self):
         self._check(lib.nezha_sync(self._h))

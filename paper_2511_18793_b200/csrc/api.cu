@@ -20,6 +20,9 @@ void launch_hs_probe(HashSetView hs, const unsigned long long* keys, unsigned lo
                      cudaStream_t st);
 void launch_prefill_tokens(const EngineState& e, const int* hist, const int* n_hist, int b0, int rows, int max_n,
                            int S_call, int S_cap, int* h_rows, cudaStream_t st);
+unsigned long long profile_total_launches();
+void profile_enable(bool on);
+void profile_read(nezha_profile* out);
 bool gemm_tc_supported(const GemmArgs& a);
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
 bool attention_tc_supported(const AttnArgs& a);
@@ -633,6 +636,22 @@ nezha_status nezha_select(nezha_ctx* c, int32_t batch, int32_t n_beams, int32_t 
   s.out_stride = beam_width; s.tuple_len = level; s.batch = batch; s.li = c->es.li; s.hs = c->es.hs;
   launch_select(s, c->st);
   NZ_CUDA(c, cudaGetLastError());
+  return NEZHA_OK;
+}
+
+uint64_t nezha_launch_count(void) { return profile_total_launches(); }
+
+nezha_status nezha_profile_enable(nezha_ctx* c, int32_t on) {
+  if (!c) return NEZHA_ERR_ARG;
+  NZ_CUDA(c, cudaStreamSynchronize(c->st));
+  profile_enable(on != 0);
+  return NEZHA_OK;
+}
+
+nezha_status nezha_profile_read(nezha_ctx* c, nezha_profile* out) {
+  if (!c || !out) return NEZHA_ERR_ARG;
+  NZ_CUDA(c, cudaStreamSynchronize(c->st));
+  profile_read(out);
   return NEZHA_OK;
 }
 

@@ -107,6 +107,7 @@ void dispatch(const AttnArgs& a, cudaStream_t st) {
 
 void launch_attention_simt(const AttnArgs& a, bool bf16, cudaStream_t st) {
   if (a.M <= 0) return;
+  LaunchScope ls(kcAttention, st);
   if (bf16) dispatch<__nv_bfloat16>(a, st);
   else dispatch<float>(a, st);
 }

@@ -199,6 +199,7 @@ cudaError_t select_configure(int max_beam) {
 void launch_select(const SelectArgs& a, cudaStream_t st) {
   if (a.batch <= 0) return;
   const size_t smem = select_smem_bytes(a.in_stride, a.K);
+  LaunchScope ls(kcSelect, st);
   if (a.T <= 32) select_kernel<1><<<a.batch, 256, smem, st>>>(a);
   else if (a.T <= 256) select_kernel<8><<<a.batch, 256, smem, st>>>(a);
   else if (a.T <= 512) select_kernel<16><<<a.batch, 256, smem, st>>>(a);
@@ -601,53 +602,66 @@ __global__ void trace_beams_kernel(EngineState e, int batch, int K, nezha_trace 
 
 void launch_fill_i32(int* p, long long n, int v, cudaStream_t st) {
   if (n <= 0) return;
+  LaunchScope ls(kcMisc, st);
   fill_i32_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, st>>>(p, n, v);
 }
 void launch_fill_f32(float* p, long long n, float v, cudaStream_t st) {
   if (n <= 0) return;
+  LaunchScope ls(kcMisc, st);
   fill_f32_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, st>>>(p, n, v);
 }
 void launch_init_decode(const EngineState& e, int batch, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
   init_decode_kernel<<<(batch + 127) / 128, 128, 0, st>>>(e, batch);
 }
 void launch_draft_init(const EngineState& e, int batch, int from_scratch, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
   draft_init_kernel<<<batch, 64, 0, st>>>(e, batch, from_scratch);
 }
 void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
   draft_set_kernel<<<batch, 64, 0, st>>>(e, batch, K, drafts, n_draft);
 }
 void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
   if (bf16) draft_x_kernel<__nv_bfloat16><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (__nv_bfloat16*)x);
   else draft_x_kernel<float><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (float*)x);
 }
 void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
                          cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
   if (bf16)
     trans_gather_kernel<__nv_bfloat16><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (const __nv_bfloat16*)embed,
                                                                       (__nv_bfloat16*)A);
   else trans_gather_kernel<float><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (const float*)embed, (float*)A);
 }
 void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st) {
+  LaunchScope ls(kcNodes, st, 2);
   nodes_count_kernel<<<batch, 64, 0, st>>>(e, batch);
   nodes_fill_kernel<<<batch, 128, 0, st>>>(e, batch);
 }
 void launch_nodes_from_prefixes(const EngineState& e, int batch, int n_beams, int level, const int* prefixes,
                                 cudaStream_t st) {
+  LaunchScope ls(kcNodes, st);
   nodes_from_prefixes_kernel<<<batch, 128, 0, st>>>(e, batch, n_beams, level, prefixes);
 }
 void launch_advance(const EngineState& e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count,
                     cudaStream_t st) {
+  LaunchScope ls(kcAccept, st);
   advance_kernel<<<batch, 64, 0, st>>>(e, batch, n, K, out_codes, out_score, out_count);
 }
 void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, cudaStream_t st) {
+  LaunchScope ls(kcAccept, st);
   round_end_kernel<<<batch, 64, 0, st>>>(e, batch, K, round, tr, 0);
 }
 void launch_write_out(const int* codes, const float* score, const int* count, int stride, int L, int batch, int K,
                       int* out_codes, float* out_score, int* out_count, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
   write_out_kernel<<<batch, 64, 0, st>>>(codes, score, count, stride, L, K, out_codes, out_score, out_count);
 }
 void launch_copy_logits(const float* src, long long row_stride, int col_off, const int* row_index, int row_mul,
                         int beam_mul, int batch, int n_beams, int idx_stride, int T, float* dst, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
   copy_logits_kernel<<<batch * n_beams, 128, 0, st>>>(src, row_stride, col_off, row_index, row_mul, beam_mul, n_beams,
                                                       idx_stride, T, dst);
 }
@@ -682,9 +696,11 @@ __global__ void prefill_tokens_kernel(EngineState e, const int* hist, const int*
 void launch_prefill_tokens(const EngineState& e, const int* hist, const int* n_hist, int b0, int rows, int max_n,
                            int S_call, int S_cap, int* h_rows, cudaStream_t st) {
   const long long n = (long long)rows * S_call;
+  LaunchScope ls(kcNodes, st);
   prefill_tokens_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(e, hist, n_hist, b0, rows, max_n, S_call, S_cap, h_rows);
 }
 void launch_trace_beams(const EngineState& e, int batch, int K, const nezha_trace& tr, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
   trace_beams_kernel<<<batch, 64, 0, st>>>(e, batch, K, tr);
 }
 

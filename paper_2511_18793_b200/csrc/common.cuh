@@ -18,6 +18,19 @@ constexpr int kMaxProbeBuckets = 4096;           // bound of every probe / inser
 // bits of the device status word
 enum : int { kStHashFull = 1, kStBadCode = 2, kStInternal = 4 };
 
+// Kernel classes for the launch counter and the optional CUDA-event timing (see nezha_profile_*).
+enum KernelClass : int {
+  kcGemm = 0, kcAttention, kcSelect, kcNorm, kcRope, kcEmbed, kcSwiglu, kcDraftGlue, kcNodes, kcAccept, kcHash, kcMisc,
+  kcCount
+};
+static_assert(kcCount <= NEZHA_PROFILE_CLASSES, "profile classes");
+// Wrap the launch(es) of one kernel class: counts them and, when profiling is on, brackets them with events.
+struct LaunchScope {
+  LaunchScope(int cls, cudaStream_t st, int n_launches = 1);
+  ~LaunchScope();
+  int cls; cudaStream_t st; int slot;
+};
+
 // --------------------------------------------------------------------------------------------------
 // small device helpers
 // --------------------------------------------------------------------------------------------------

@@ -93,6 +93,7 @@ __global__ void swiglu_kernel(const T* __restrict__ gu, T* __restrict__ act, int
 void launch_embed(const void* table, bool bf16, const int* tokens, int M, const int* M_dev, int d, float* resid,
                   cudaStream_t st) {
   if (M <= 0) return;
+  LaunchScope ls(kcEmbed, st);
   if (bf16) embed_kernel<__nv_bfloat16><<<M, 128, 0, st>>>((const __nv_bfloat16*)table, tokens, M, M_dev, d, resid);
   else embed_kernel<float><<<M, 128, 0, st>>>((const float*)table, tokens, M, M_dev, d, resid);
 }
@@ -101,6 +102,7 @@ void launch_rmsnorm(const float* x, long long x_stride, const int* row_index, co
                     float* out_f32, int M, const int* M_dev, int d, float eps, cudaStream_t st) {
   if (M <= 0) return;
   const int wpb = 8;
+  LaunchScope ls(kcNorm, st);
   dim3 grid((M + wpb - 1) / wpb);
   if (bf16)
     rmsnorm_kernel<__nv_bfloat16><<<grid, wpb * 32, 0, st>>>(x, x_stride, row_index, (const __nv_bfloat16*)gain,
@@ -112,6 +114,7 @@ void launch_rmsnorm(const float* x, long long x_stride, const int* row_index, co
 
 void launch_rope_append(const RopeAppendArgs& a, bool bf16, cudaStream_t st) {
   if (a.M <= 0) return;
+  LaunchScope ls(kcRope, st);
   if (bf16) rope_append_kernel<__nv_bfloat16><<<a.M, 128, 0, st>>>(a);
   else rope_append_kernel<float><<<a.M, 128, 0, st>>>(a);
 }
@@ -119,6 +122,7 @@ void launch_rope_append(const RopeAppendArgs& a, bool bf16, cudaStream_t st) {
 void launch_swiglu(const void* gu, void* act, int M, const int* M_dev, int F, bool bf16, cudaStream_t st) {
   if (M <= 0) return;
   long long total = (long long)M * F;
+  LaunchScope ls(kcSwiglu, st);
   int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
   if (bf16) swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)gu, (__nv_bfloat16*)act, M, M_dev, F);
   else swiglu_kernel<float><<<blocks, 256, 0, st>>>((const float*)gu, (float*)act, M, M_dev, F);

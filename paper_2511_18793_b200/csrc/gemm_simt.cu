@@ -81,6 +81,7 @@ void dispatch(const GemmArgs& a, cudaStream_t st) {
 
 void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st) {
   if (a.M <= 0 || a.N <= 0) return;
+  LaunchScope ls(kcGemm, st);
   if (bf16) dispatch<__nv_bfloat16>(a, st);
   else dispatch<float>(a, st);
 }

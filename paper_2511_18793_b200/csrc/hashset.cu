@@ -88,22 +88,26 @@ __global__ void hs_probe_kernel(HashSetView hs, const unsigned long long* __rest
 }
 
 void launch_hs_clear(HashSetView hs, cudaStream_t st) {
+  LaunchScope ls(kcHash, st);
   hs_clear_kernel<<<148 * 8, 512, 0, st>>>(hs.slots, hs.n_buckets * kBucketSlots);
 }
 void launch_hs_pack(const LevelInfo& li, const int* codes, unsigned long long n, unsigned long long* keys, int* status,
                     cudaStream_t st) {
   if (!n) return;
+  LaunchScope ls(kcHash, st);
   hs_pack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(li, codes, n, keys, status);
 }
 void launch_hs_insert(const LevelInfo& li, HashSetView hs, const int* codes, unsigned long long n,
                       unsigned long long* n_unique, int* status, cudaStream_t st) {
   if (!n) return;
+  LaunchScope ls(kcHash, st);
   hs_insert_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(li, hs, codes, n, n_unique, status);
 }
 void launch_hs_probe(HashSetView hs, const unsigned long long* keys, unsigned long long n, uint8_t* found,
                      cudaStream_t st) {
   if (!n) return;
   unsigned long long threads = n * kBucketSlots;
+  LaunchScope ls(kcHash, st);
   hs_probe_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(hs, keys, n, found);
 }
 
