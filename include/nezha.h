@@ -196,6 +196,16 @@ nezha_status nezha_select(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_
                           const int32_t* n_live,
                           int32_t* out_parent, int32_t* out_code, float* out_score, int32_t* out_count);
 
+/* The projection GEMM by itself: C[M,N] (op)= A[M,K] * W[N,K]^T with fp32 accumulation, operands in the context's
+ * storage type (device pointers, row-major, leading dimensions = K for A and W, N for C).
+ *   epilogue 0: C (storage type) = acc;  1: C (float) = acc;  2: C (float) += acc;  3: C (float) = tanh(acc + bias[n])
+ *   path     0: the engine's own choice; 1: CUDA-core kernel; 2: tcgen05 kernel (NEZHA_ERR_UNSUPPORTED if the shape
+ *               is not covered: bf16 storage, K % 64 == 0, N % 128 == 0)
+ * Used by every projection of the primary model (Algorithm 1 line 4), the LM head (line 5) and the draft head
+ * (Eq. 2-3).  Asynchronous. */
+nezha_status nezha_gemm(nezha_ctx* ctx, const void* A, const void* W, void* C, int32_t M, int32_t N, int32_t K,
+                        int32_t epilogue, const float* bias, int32_t path);
+
 /* ---- instrumentation (the paper has no counterpart: these only measure the library itself) -------------- */
 
 #define NEZHA_PROFILE_CLASSES 16

@@ -84,6 +84,8 @@ class NezhaProfile(C.Structure):
 
 PROFILE_CLASSES = ["gemm", "attention", "select", "norm", "rope_append", "embed", "swiglu", "draft_glue", "nodes",
                    "accept", "hash", "misc"]
+lib.nezha_gemm.restype = C.c_int
+lib.nezha_gemm.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32]
 lib.nezha_launch_count.restype = C.c_uint64
 lib.nezha_launch_count.argtypes = []
 lib.nezha_profile_enable.restype = C.c_int
@@ -99,7 +101,7 @@ lib.nezha_destroy.argtypes = [_vp]
 
 EXPORTS = ["nezha_arena_bytes", "nezha_create", "nezha_build_hashset", "nezha_pack", "nezha_probe", "nezha_prefill",
            "nezha_decode", "nezha_decode_with_drafts", "nezha_get_hidden", "nezha_primary_logits",
-           "nezha_draft_logits", "nezha_select", "nezha_launch_count", "nezha_profile_enable",
+           "nezha_draft_logits", "nezha_select", "nezha_gemm", "nezha_launch_count", "nezha_profile_enable",
            "nezha_profile_read", "nezha_sync", "nezha_last_error", "nezha_destroy"]
 
 
@@ -288,6 +290,14 @@ class Engine:
                                      _ptr(logits.contiguous()), _ptr(beam_scores.contiguous()), _ptr(bc),
                                      _ptr(n_live.contiguous()), _ptr(parent), _ptr(code), _ptr(score), _ptr(count)))
         return parent, code, score, count
+
+    def gemm(self, A: torch.Tensor, W: torch.Tensor, C_out: torch.Tensor, epilogue: int = 0,
+             bias: Optional[torch.Tensor] = None, path: int = 0):
+        M, K = A.shape
+        N = W.shape[0]
+        assert W.shape[1] == K and tuple(C_out.shape) == (M, N)
+        self._check(lib.nezha_gemm(self._h, _ptr(A), _ptr(W), _ptr(C_out), M, N, K, epilogue, _ptr(bias), path))
+        return C_out
 
     def profile_enable(self, on: bool):
         self._check(lib.nezha_profile_enable(self._h, 1 if on else 0))

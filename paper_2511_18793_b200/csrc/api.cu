@@ -215,7 +215,7 @@ size_t carve(nezha_ctx* c) {
 
 void gemm(nezha_ctx* c, const void* A, long long lda, const void* W, long long ldw, void* C, long long ldc, long long M,
           const int* M_dev, int N, int K, int epi, const float* bias = nullptr) {
-  GemmArgs a{A, lda, W, ldw, C, ldc, (int)M, M_dev, N, K, epi, bias};
+  GemmArgs a{A, lda, W, ldw, C, ldc, (int)M, M_dev, N, K, epi, bias, c->es.status};
   if (c->bf16 && gemm_tc_supported(a)) launch_gemm_tc(a, c->st);
   else launch_gemm_simt(a, c->bf16, c->st);
 }
@@ -325,7 +325,7 @@ nezha_status pending_device_error(nezha_ctx* c) {
   if (st) NZ_CUDA(c, cudaMemsetAsync(c->es.status, 0, sizeof(int), c->st));
   if (st & kStHashFull) return fail(c, NEZHA_ERR_HASH_FULL, "hash set insertion exhausted its probe bound");
   if (st & kStBadCode) return fail(c, NEZHA_ERR_CATALOG, "a code outside [0, T_l) was given");
-  if (st) return fail(c, NEZHA_ERR_CUDA, "internal device-side check failed");
+  if (st) return fail(c, NEZHA_ERR_CUDA, "a bounded device-side wait expired (kernel gave up and returned)");
   return NEZHA_OK;
 }
 
@@ -635,6 +635,21 @@ nezha_status nezha_select(nezha_ctx* c, int32_t batch, int32_t n_beams, int32_t 
   s.out_codes = nullptr; s.out_token = out_code; s.out_score = out_score; s.out_parent = out_parent; s.out_count = out_count;
   s.out_stride = beam_width; s.tuple_len = level; s.batch = batch; s.li = c->es.li; s.hs = c->es.hs;
   launch_select(s, c->st);
+  NZ_CUDA(c, cudaGetLastError());
+  return NEZHA_OK;
+}
+
+nezha_status nezha_gemm(nezha_ctx* c, const void* A, const void* W, void* C, int32_t M, int32_t N, int32_t K,
+                        int32_t epilogue, const float* bias, int32_t path) {
+  if (!c) return NEZHA_ERR_ARG;
+  if (!A || !W || !C || M < 1 || N < 1 || K < 1 || epilogue < 0 || epilogue > 3 || (epilogue == 3 && !bias) || path < 0 ||
+      path > 2)
+    return fail(c, NEZHA_ERR_ARG, "nezha_gemm: bad argument");
+  GemmArgs a{A, K, W, K, C, N, M, nullptr, N, K, epilogue, bias, c->es.status};
+  const bool tc_ok = c->bf16 && gemm_tc_supported(a);
+  if (path == 2 && !tc_ok) return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: shape not covered by the tcgen05 kernel");
+  if (path != 1 && tc_ok) launch_gemm_tc(a, c->st);
+  else launch_gemm_simt(a, c->bf16, c->st);
   NZ_CUDA(c, cudaGetLastError());
   return NEZHA_OK;
 }

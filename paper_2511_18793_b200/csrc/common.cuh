@@ -121,6 +121,7 @@ struct GemmArgs {
   int N, K;
   int epilogue;
   const float* bias;
+  int* status;           // device status word (bounded waits report here)
 };
 
 void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);

@@ -1,0 +1,56 @@
+"""The projection GEMM kernels against a plain fp64 matrix product (numpy) on the same bf16 inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_18793_b200 import synth
+from gpu_helpers import Case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    w = synth.scaled(synth.WORKLOADS["small"], n_items=10_000, n_layers=1, batch=2, n_hist=2)
+    return Case(w)
+
+
+def _ref(A, W):
+    return A.double().cpu().numpy() @ W.double().cpu().numpy().T
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 512), (1920, 1536, 512), (77, 768, 2048), (640, 512, 1024),
+                                    (1, 128, 64), (129, 128, 4864)])
+@pytest.mark.parametrize("path", [1, 2])
+def test_gemm_epilogues(ctx, M, N, K, path):
+    g = torch.Generator(device="cuda"); g.manual_seed(M * 7 + N * 3 + K)
+    A = (torch.randn(M, K, generator=g, device="cuda") * 0.5).bfloat16()
+    W = (torch.randn(N, K, generator=g, device="cuda") * 0.05).bfloat16()
+    ref = _ref(A, W)
+    scale = np.abs(ref).max()
+    out = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    ctx.eng.gemm(A, W, out, epilogue=1, path=path)
+    assert np.abs(out.cpu().numpy() - ref).max() < 2e-5 * scale * np.sqrt(K / 64) + 1e-6      # fp32 accumulation only
+    outb = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    ctx.eng.gemm(A, W, outb, epilogue=0, path=path)
+    assert np.abs(outb.float().cpu().numpy() - ref).max() < scale * 2 ** -8
+    res = torch.randn(M, N, generator=g, device="cuda")
+    acc = res.clone()
+    ctx.eng.gemm(A, W, acc, epilogue=2, path=path)
+    assert np.abs(acc.cpu().numpy() - (res.double().cpu().numpy() + ref)).max() < 2e-5 * scale * np.sqrt(K / 64) + 1e-5
+    bias = torch.randn(N, generator=g, device="cuda")
+    th = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    ctx.eng.gemm(A, W, th, epilogue=3, bias=bias, path=path)
+    assert np.abs(th.cpu().numpy() - np.tanh(ref + bias.double().cpu().numpy())).max() < 1e-4
+    ctx.eng.sync()
+
+
+def test_gemm_tc_rejects_uncovered_shapes(ctx):
+    A = torch.zeros(8, 48, dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(128, 48, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(8, 128, dtype=torch.float32, device="cuda")
+    with pytest.raises(ctx.binding.NezhaError) as ei:
+        ctx.eng.gemm(A, W, out, epilogue=1, path=2)
+    assert ei.value.status == 7
+    ctx.eng.gemm(A, W, out, epilogue=1, path=0)          # falls back to the CUDA-core kernel
+    ctx.eng.sync()

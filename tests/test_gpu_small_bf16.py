@@ -77,8 +77,9 @@ def test_small_verified_decode_all_rows(small):
     # GPU-internal invariants on all rows: zero sacrifice and zero hallucinations
     assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
     codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
-    assert np.all(count == w.beam)
-    assert V.contains(codes.reshape(-1, w.L)).all()
+    # (with an untrained model most level-(L-1) beams have no valid completion: count < beam is expected)
+    live = np.arange(w.beam)[None, :] < count[:, None]
+    assert V.contains(codes[live]).all() and np.all(codes[~live] == -1)
     assert 1 <= out["stats"].rounds <= w.L - 1
     beams = out["trace"]["beams"].cpu().numpy()
     scores = out["trace"]["beam_scores"].cpu().numpy()
