@@ -209,6 +209,7 @@ size_t carve(nezha_ctx* c) {
   e.tok_ctx_len = cv.take<int>(c->Ms); e.tok_kv_dst = cv.take<long long>(c->Ms);
   e.tok_ext = cv.take<long long>((size_t)c->Mv_max * c->L);
   e.row_tok_count = cv.take<int>(c->Bmax); e.n_tokens = cv.take<int>(1);
+  e.row_tok_start = cv.take<int>(c->Bmax); e.pf_row_start = cv.take<int>(c->Bmax); e.pf_row_count = cv.take<int>(c->Bmax);
   e.h_f32 = c->h_f32;
   return (cv.off + 255) & ~(size_t)255;
 }
@@ -223,7 +224,7 @@ void gemm(nezha_ctx* c, const void* A, long long lda, const void* W, long long l
 // One pass of the primary model's layers over the tokens described by es.tok_* (resid already holds the
 // embeddings).  verify = false: prefill (KV goes to the context cache, tokens see a causal prefix of it);
 // verify = true: drafted codes (KV goes to the draft region, tokens see the whole context + their own tuple).
-void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify) {
+void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify, int n_rows, int max_tok_per_row) {
   const EngineState& e = c->es;
   const size_t esz = c->esz;
   for (int i = 0; i < c->nl; ++i) {
@@ -248,6 +249,9 @@ void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify) {
     t.k_ext = ke; t.v_ext = ve; t.ext_head_stride = c->hd;
     t.tok_row = e.tok_row; t.tok_ctx_len = e.tok_ctx_len; t.tok_ext = e.tok_ext; t.n_ext_max = verify ? c->L : 0;
     t.M = (int)M; t.M_dev = M_dev; t.Hq = c->Hq; t.Hkv = c->Hkv; t.hd = c->hd; t.scale = 1.f / sqrtf((float)c->hd);
+    t.row_start = verify ? e.row_tok_start : e.pf_row_start; t.row_count = verify ? e.row_tok_count : e.pf_row_count;
+    t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
+    t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
     if (c->bf16 && attention_tc_supported(t)) launch_attention_tc(t, c->st);
     else launch_attention_simt(t, c->bf16, c->st);
     gemm(c, c->attn, (long long)c->Hq * c->hd, w.wo, (long long)c->Hq * c->hd, c->resid, c->d, M, M_dev, c->d,
@@ -261,11 +265,11 @@ void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify) {
 }
 
 // The verify pass proper: embeddings of the node tokens, all layers, final norm, LM head of levels 2..L.
-void verify_pass(nezha_ctx* c, long long M_bound) {
+void verify_pass(nezha_ctx* c, long long M_bound, int n_rows, int max_tok_per_row) {
   const EngineState& e = c->es;
   if (M_bound <= 0 || c->L < 2) return;
   launch_embed(c->embed, c->bf16, e.tok_id, (int)M_bound, e.n_tokens, c->d, c->resid, c->st);
-  run_layers(c, M_bound, e.n_tokens, true);
+  run_layers(c, M_bound, e.n_tokens, true, n_rows, max_tok_per_row);
   launch_rmsnorm(c->resid, c->d, nullptr, c->final_norm, c->bf16, c->xn, nullptr, (int)M_bound, e.n_tokens, c->d,
                  c->cfg.rms_eps, c->st);
   const char* w = (const char*)c->lm_head + (size_t)e.li.off[1] * c->d * c->esz;
@@ -383,7 +387,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
     else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, true);
     launch_build_nodes(e, batch, c->st);
-    verify_pass(c, (long long)batch * K * (L - round));
+    verify_pass(c, (long long)batch * K * (L - round), batch, K * (L - round));
     for (int n = round; n < L; ++n) {
       SelectArgs s = select_base(c, batch, K);
       const size_t lv_in = (size_t)n * c->Bmax * c->Kmax, lv_out = (size_t)(n + 1) * c->Bmax * c->Kmax;
@@ -452,6 +456,11 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
     return src && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   };
   bool ok = cudaMemsetAsync(c->es.status, 0, 8 * sizeof(int), st) == cudaSuccess;
+  // the caches start as zeros: tiles may overhang into never-written rows, whose (masked) values must be finite
+  ok = ok && cudaMemsetAsync(c->k_ctx, 0, (size_t)c->nl * c->ctx_layer_elems * c->esz, st) == cudaSuccess &&
+       cudaMemsetAsync(c->v_ctx, 0, (size_t)c->nl * c->ctx_layer_elems * c->esz, st) == cudaSuccess &&
+       cudaMemsetAsync(c->k_ext, 0, (size_t)c->nl * c->ext_layer_elems * c->esz, st) == cudaSuccess &&
+       cudaMemsetAsync(c->v_ext, 0, (size_t)c->nl * c->ext_layer_elems * c->esz, st) == cudaSuccess;
   ok = ok && cp(c->embed, w->embed, (size_t)c->vocab * c->d * esz) && cp(c->lm_head, w->lm_head, (size_t)c->vocab * c->d * esz) &&
        cp(c->final_norm, w->final_norm, (size_t)c->d * esz);
   const size_t q_b = (size_t)c->Hq * c->hd * c->d * esz, kv_b = (size_t)c->Hkv * c->hd * c->d * esz, f_b = (size_t)c->F * c->d * esz;
@@ -537,7 +546,7 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
     const long long M = (long long)rows * S_call;
     launch_prefill_tokens(e, hist_codes, n_hist, b0, rows, max_n, S_call, c->S, c->h_rows, c->st);
     launch_embed(c->embed, c->bf16, e.tok_id, (int)M, nullptr, c->d, c->resid, c->st);
-    run_layers(c, M, nullptr, false);
+    run_layers(c, M, nullptr, false, rows, S_call);
     const size_t ho = (size_t)b0 * (c->L + 1) * c->d;
     launch_rmsnorm(c->resid, c->d, c->h_rows, c->final_norm, c->bf16, (char*)c->h_act + ho * c->esz, c->h_f32 + ho,
                    rows * (c->L + 1), nullptr, c->d, c->cfg.rms_eps, c->st);
@@ -583,7 +592,7 @@ nezha_status nezha_primary_logits(nezha_ctx* c, int32_t batch, int32_t n_beams, 
     launch_copy_logits(c->logits0, c->cfg.T[0], 0, nullptr, 1, 0, batch, n_beams, 0, c->cfg.T[0], logits, c->st);
   } else {
     launch_nodes_from_prefixes(e, batch, n_beams, level, prefixes, c->st);
-    verify_pass(c, (long long)batch * n_beams * level);
+    verify_pass(c, (long long)batch * n_beams * level, batch, n_beams * level);
     launch_copy_logits(c->logits_v, c->Nv, e.li.off[level] - e.li.off[1], e.node_index + (size_t)level * c->Kmax, 0, 0, batch,
                        n_beams, c->L * c->Kmax, c->cfg.T[level], logits, c->st);
   }

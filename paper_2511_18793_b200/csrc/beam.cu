@@ -368,6 +368,7 @@ __global__ void nodes_fill_kernel(EngineState e, int batch) {
     int off = 0;
     for (int i = 0; i < b; ++i) off += e.row_tok_count[i];
     s_off = off;
+    e.row_tok_start[b] = off;
     if (b == batch - 1) *e.n_tokens = off + e.row_tok_count[b];
     int c = 0;
     for (int k = 0; k < Kmax; ++k) { s_alive_rank[k] = c; c += e.d_alive[b * Kmax + k]; }
@@ -433,6 +434,7 @@ __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams
   const long long slab_elems = (long long)Kmax * e.Hkv * e.hd;
   const long long row_elems = (long long)(L - 1) * slab_elems;
   if (b == 0 && threadIdx.x == 0) *e.n_tokens = batch * per_row;
+  if (threadIdx.x == 0) { e.row_tok_start[b] = b * per_row; e.row_tok_count[b] = per_row; }
   for (int i = threadIdx.x; i < L * Kmax; i += blockDim.x) e.node_index[(long long)b * L * Kmax + i] = -1;
   __syncthreads();
   for (int idx = threadIdx.x; idx < per_row; idx += blockDim.x) {
@@ -689,7 +691,7 @@ __global__ void prefill_tokens_kernel(EngineState e, const int* hist, const int*
   }
   e.tok_id[idx] = tok; e.tok_pos[idx] = p; e.tok_row[idx] = b; e.tok_ctx_len[idx] = p + 1;
   e.tok_kv_dst[idx] = ((long long)b * e.Hkv * S_cap + p) * e.hd;
-  if (p == 0) e.row_P[b] = P;
+  if (p == 0) { e.row_P[b] = P; e.pf_row_start[lb] = lb * S_call; e.pf_row_count[lb] = S_call; }
   if (p >= P - 1 && p <= P - 1 + L) h_rows[lb * (L + 1) + (p - (P - 1))] = (int)idx;
 }
 

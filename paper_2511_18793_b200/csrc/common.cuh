@@ -165,6 +165,11 @@ struct AttnArgs {
   int M; const int* M_dev;
   int Hq, Hkv, hd;
   float scale;
+  // grouping of the token list by request (tokens of a request are contiguous), for the tensor-core kernel
+  const int* row_start; const int* row_count;   // [n_rows] first token / token count of each request in this pass
+  int n_rows, max_tokens_per_row;
+  long long ctx_rows_total;                     // requests * kv heads * positions of the layer's context cache
+  int* status;
 };
 void launch_attention_simt(const AttnArgs& a, bool bf16, cudaStream_t st);
 

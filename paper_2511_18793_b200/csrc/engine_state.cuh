@@ -35,6 +35,8 @@ struct EngineState {
   int* node_index;  // [Bmax][L][Kmax] token index of node (level n = 1..L-1 stored at n, slot), -1 if absent
   int* tok_row; int* tok_pos; int* tok_id; int* tok_ctx_len; long long* tok_kv_dst; long long* tok_ext;  // tok_ext [Mv][L]
   int* row_tok_count;   // [Bmax]
+  int* row_tok_start;   // [Bmax] first token of the request in the list
+  int* pf_row_start; int* pf_row_count;   // [Bmax] the same for a prefill chunk (indexed by row within the chunk)
   int* n_tokens;        // [1]
   int* counters;        // [8]: 0 unfinished rows, 1 primary tokens (round), 2 accepted levels (round), 3 drafted (round)
 

@@ -7,12 +7,7 @@
 // accumulator back with tcgen05.ld and apply the epilogue (store / residual add / bias+tanh).
 // Every mbarrier wait is bounded: on expiry the CTA records an error in the status word, drains what it has
 // in flight, frees its TMEM and returns.
-#include <cuda.h>
-
-#include <map>
-#include <tuple>
-
-#include "common.cuh"
+#include "tma.cuh"
 
 namespace nz {
 
@@ -23,35 +18,6 @@ constexpr int kTileBytesA = BM * BK * 2, kTileBytesB = BN * BK * 2;
 constexpr int kStageBytes = kTileBytesA + kTileBytesB;
 constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 192;
-constexpr long long kWaitCycles = 2000000000ll;     // about one second of SM clock: bound of every barrier wait
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait; false = gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  const long long t0 = clock64();
-  for (;;) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return true;
-    if (clock64() - t0 > kWaitCycles) return false;
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
-}
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -116,8 +82,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(accum_bar, 1);
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_fence_init();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(BN));
@@ -213,50 +178,6 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
 // ---------------------------------------------------------------------------------------------------
 // host side: tensor maps
 // ---------------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    cudaGetLastError();
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// 2-D bf16 row-major [rows, cols] with row pitch ld (elements); box = 64 columns x box_rows rows, 128B swizzle.
-bool make_map(CUtensorMap* tm, const void* ptr, long long rows, long long cols, long long ld, int box_rows) {
-  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return encode_fn()(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-using MapKey = std::tuple<const void*, long long, long long, long long, int>;
-std::map<MapKey, CUtensorMap>& map_cache() {
-  static std::map<MapKey, CUtensorMap> c;
-  return c;
-}
-const CUtensorMap* get_map(const void* ptr, long long rows, long long cols, long long ld, int box_rows) {
-  MapKey key{ptr, rows, cols, ld, box_rows};
-  auto& c = map_cache();
-  auto it = c.find(key);
-  if (it != c.end()) return &it->second;
-  CUtensorMap tm;
-  if (!make_map(&tm, ptr, rows, cols, ld, box_rows)) return nullptr;
-  if (c.size() > 4096) c.clear();
-  return &c.emplace(key, tm).first->second;
-}
-
 template <int EPI>
 void launch(const CUtensorMap* ta, const CUtensorMap* tb, const GemmArgs& a, cudaStream_t st) {
   static bool configured = false;
@@ -271,7 +192,7 @@ void launch(const CUtensorMap* ta, const CUtensorMap* tb, const GemmArgs& a, cud
 }  // namespace
 
 bool gemm_tc_supported(const GemmArgs& a) {
-  if (!a.status || !encode_fn()) return false;
+  if (!a.status || !tma_encode_fn()) return false;
   if (a.K % BK || a.N % BN || a.M <= 0) return false;
   if ((a.lda * 2) % 16 || (a.ldw * 2) % 16 || ((uintptr_t)a.A & 15) || ((uintptr_t)a.W & 15)) return false;
   if (a.epilogue == kEpiStoreAct && (((uintptr_t)a.C & 3) || (a.ldc & 1))) return false;
@@ -281,8 +202,8 @@ bool gemm_tc_supported(const GemmArgs& a) {
 }
 
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
-  const CUtensorMap* ta = get_map(a.A, a.M, a.K, a.lda, BM);
-  const CUtensorMap* tb = get_map(a.W, a.N, a.K, a.ldw, BN);
+  const CUtensorMap* ta = tma_map_bf16(a.A, a.M, a.K, a.lda, BM);
+  const CUtensorMap* tb = tma_map_bf16(a.W, a.N, a.K, a.ldw, BN);
   if (!ta || !tb) { launch_gemm_simt(a, true, st); return; }
   LaunchScope ls(kcGemm, st);
   switch (a.epilogue) {

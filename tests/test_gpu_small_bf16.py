@@ -104,3 +104,40 @@ def test_small_draft_mode(small):
             lp = O.joint_logprob_draft(head, small.req(b), tuple(int(c) for c in codes[b, k]))
             assert abs(lp - scores[b, k]) < w.L * tolerance(w)
     assert n_valid >= 0
+
+
+# ---------------------------------------------------------------------------------------- other bf16 shapes
+SHAPES = {
+    "hd128_gqa2": dict(d_model=512, n_q_heads=4, n_kv_heads=2, d_ffn=1024),      # head_dim 128, groups of 2
+    "hd64_gqa7": dict(d_model=448, n_q_heads=7, n_kv_heads=1, d_ffn=896),        # head_dim 64, 7 query heads on 1 KV head
+    "hd128_mha": dict(d_model=256, n_q_heads=2, n_kv_heads=2, d_ffn=512),
+}
+
+
+@pytest.mark.parametrize("shape", sorted(SHAPES))
+def test_bf16_shapes_ragged_histories(shape):
+    w = synth.scaled(synth.WORKLOADS["small"], n_layers=2, n_items=50_000, batch=5, beam=7, n_hist=40, seed=11,
+                     **SHAPES[shape])
+    case = Case(w)
+    lens = [40, 1, 17, 0, 33]
+    case.eng.prefill(case.hist_dev, torch.tensor(lens, dtype=torch.int32, device="cuda"))
+    model, head, V = case.oracle
+    reqs = [model.prefill(case.hist[b, :n]) for b, n in enumerate(lens)]
+    case._reqs = {(b, None): r for b, r in enumerate(reqs)}
+    h = case.eng.get_hidden().cpu().numpy()
+    for b in range(w.batch):
+        assert np.abs(h[b] - reqs[b].h).max() < 3e-2
+    rng = np.random.default_rng(1)
+    for level in (1, 3):
+        pre = np.stack([rng.integers(0, w.T[l], size=(w.batch, w.beam)) for l in range(level)], axis=2).astype(np.int32)
+        got = case.eng.primary_logits(w.beam, level, torch.from_numpy(pre).cuda()).cpu().numpy()
+        for b in range(w.batch):
+            ref = model.next_level_logits_many(reqs[b], [tuple(pre[b, r]) for r in range(w.beam)])
+            assert np.abs(got[b] - np.stack(ref)).max() < tolerance(w)
+    out = case.eng.decode(w.beam, mode=1, trace=True)
+    ar = case.eng.decode(w.beam, mode=2)
+    assert torch.equal(out["codes"], ar["codes"])
+    beams = out["trace"]["beams"].cpu().numpy()
+    scores = out["trace"]["beam_scores"].cpu().numpy()
+    for b in range(w.batch):
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam)
