@@ -153,9 +153,12 @@ def silu(x: np.ndarray) -> np.ndarray:
 class PrimaryModel:
     """M_p.  Weights are given as float arrays (already rounded to their storage type); all arithmetic is fp64."""
 
-    def __init__(self, shape: ModelShape, weights: Dict[str, object], cache_f64: bool = True):
+    def __init__(self, shape: ModelShape, weights: Dict[str, object], cache_f64: bool = True, dtype=np.float64):
+        """dtype: arithmetic type of the forward pass.  fp64 by default; fp32 is offered only so that a multi-billion
+        parameter model can be checked in minutes (its rounding, ~1e-6 relative, is far below the bf16 tolerance)."""
         self.s = shape
         self.w = weights
+        self.dtype = dtype
         self._cache: Optional[Dict[Tuple[str, Optional[int]], np.ndarray]] = {} if cache_f64 else None
 
     def _f64(self, name: str, layer: Optional[int] = None) -> np.ndarray:
@@ -163,7 +166,7 @@ class PrimaryModel:
         if self._cache is not None and (name, layer) in self._cache:
             return self._cache[(name, layer)]
         a = self.w[name] if layer is None else self.w[name][layer]
-        a = np.asarray(a, dtype=np.float64)
+        a = np.asarray(a, dtype=self.dtype)
         if self._cache is not None:
             self._cache[(name, layer)] = a
         return a
@@ -189,8 +192,8 @@ class PrimaryModel:
             q = (xn @ self._f64("wq", layer).T).reshape(n, s.n_q_heads, hd)
             k = (xn @ self._f64("wk", layer).T).reshape(n, s.n_kv_heads, hd)
             v = (xn @ self._f64("wv", layer).T).reshape(n, s.n_kv_heads, hd)
-            q = rope(q, positions, s.rope_theta)
-            k = rope(k, positions, s.rope_theta)
+            q = rope(q, positions, s.rope_theta).astype(self.dtype)
+            k = rope(k, positions, s.rope_theta).astype(self.dtype)
             new_kv.append((k, v))
             if past is not None:
                 k_all = np.concatenate([past[layer][0], k], axis=0)
@@ -198,7 +201,7 @@ class PrimaryModel:
             else:
                 k_all, v_all = k, v
             n_past = k_all.shape[0] - n
-            attn = np.zeros((n, s.n_q_heads, hd), dtype=np.float64)
+            attn = np.zeros((n, s.n_q_heads, hd), dtype=self.dtype)
             if visible_new is None:
                 visible_new = np.tril(np.ones((n, n), dtype=bool))
             visible = np.concatenate([np.ones((n, n_past), dtype=bool), visible_new], axis=1)
@@ -206,7 +209,7 @@ class PrimaryModel:
                 kv = h // G
                 sc = q[:, h, :] @ k_all[:, kv, :].T / np.sqrt(hd)
                 sc = np.where(visible, sc, -np.inf)
-                p = np.exp(log_softmax(sc))
+                p = np.exp(log_softmax(sc)).astype(self.dtype)
                 attn[:, h, :] = p @ v_all[:, kv, :]
             x = x + attn.reshape(n, s.n_q_heads * hd) @ self._f64("wo", layer).T
             xn = rms_norm(x, self._f64("mlp_norm", layer), s.rms_eps)

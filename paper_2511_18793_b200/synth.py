@@ -143,7 +143,7 @@ def _zipf_quotas(n_items: int, n_prefix: int, cap: int, s: float) -> np.ndarray:
     def total(c):
         return int(np.minimum(np.floor(c * r), cap).sum())
 
-    for _ in range(60):
+    for _ in range(40):                      # a shortfall left by the finite bisection goes to `rem` below
         mid = 0.5 * (lo + hi)
         if total(mid) <= n_items:
             lo = mid

@@ -15,7 +15,7 @@ def tolerance(w):
 class Case:
     """Engine + oracle on one workload.  Weights are drawn once and handed to both sides as the same bytes."""
 
-    def __init__(self, w, device="cuda", max_beam=None, catalog=None, hist=None, weights=None, oracle_rows=None):
+    def __init__(self, w, device="cuda", max_beam=None, catalog=None, hist=None, weights=None, oracle_dtype=np.float64):
         from paper_2511_18793_b200 import binding
         self.binding = binding
         self.w = w
@@ -31,6 +31,7 @@ class Case:
         self.hist_dev = torch.from_numpy(self.hist).to(device)
         self.n_hist = torch.full((self.hist.shape[0],), self.hist.shape[1], dtype=torch.int32, device=device)
         self._oracle = None
+        self.oracle_dtype = oracle_dtype
         self._reqs = {}
 
     def prefill(self):
@@ -42,7 +43,7 @@ class Case:
         if self._oracle is None:
             Wn = synth.weights_to_numpy(self.weights)
             big = self.w.d_model * self.w.d_ffn * self.w.n_layers > 2e8
-            self._oracle = oracle_bundle(self.w, Wn, self.catalog, cache_f64=not big)
+            self._oracle = oracle_bundle(self.w, Wn, self.catalog, cache_f64=not big, dtype=self.oracle_dtype)
         return self._oracle
 
     def req(self, b, n_items=None):
@@ -84,3 +85,17 @@ def assert_topk_matches(gpu_codes, gpu_scores, gpu_count, oracle_beams, K, tol, 
     gs = np.asarray([g_map[t] for t in g_codes])
     assert np.all(gs[:-1] >= gs[1:] - 1e-6)
     return False
+
+
+def check_levels(case, b, beams, beam_scores, K, per_beam_all=True):
+    """beams [L, K, L] / beam_scores [L, K] of one request (GPU trace) against the oracle, level by level."""
+    w = case.w
+    model, _, V = case.oracle
+    req = case.req(b)
+    prev = [O.Beam((), np.float32(0.0))]
+    for n in range(w.L):
+        logits = model.next_level_logits_many(req, [bm.codes for bm in prev])
+        ref = O.expand_level(prev, logits, K, w.T[n], V if n == w.L - 1 else None)
+        cnt = int((beams[n, :, 0] >= 0).sum())
+        assert_topk_matches(beams[n][:, : n + 1], beam_scores[n], cnt, ref, K, tolerance(w))
+        prev = [O.Beam(tuple(int(c) for c in beams[n, k, : n + 1]), np.float32(beam_scores[n, k])) for k in range(cnt)]

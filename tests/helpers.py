@@ -10,9 +10,9 @@ def oracle_shape(w):
                         w.rope_theta, w.rms_eps)
 
 
-def oracle_bundle(w, weights_np, catalog, cache_f64=True):
+def oracle_bundle(w, weights_np, catalog, cache_f64=True, dtype=np.float64):
     shape = oracle_shape(w)
-    return (O.PrimaryModel(shape, weights_np, cache_f64=cache_f64), O.DraftHead(shape, weights_np),
+    return (O.PrimaryModel(shape, weights_np, cache_f64=cache_f64, dtype=dtype), O.DraftHead(shape, weights_np),
             O.ValidSet(catalog, w.T))
 
 

@@ -1,0 +1,68 @@
+"""GPU parity at the full sizes of the three LLM-shaped workloads (0.5B / 1.5B / 7B shapes; 10M and 100M-item
+catalogues), in the launch configuration bench.py times.
+
+All requests: GPU-internal invariants (verified decode == plain autoregressive decode item for item; every emitted
+tuple is in the exact valid set; counts and padding).  A fixed subset of requests: the oracle recomputes every
+beam level from the GPU's own beams (tie rule) and the prefill hidden states.  The hash set is probed with a
+hit/miss mix and with sibling keys and compared bit for bit with the exact set."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nezha_oracle as O
+from paper_2511_18793_b200 import synth
+from gpu_helpers import Case, check_levels, tolerance
+
+pytestmark = pytest.mark.gpu
+
+PLAN = {                       # workload -> (requests checked by the oracle, oracle arithmetic)
+    "0.5b": ([0, 128, 255, 77], np.float64),
+    "1.5b": ([0, 127], np.float64),
+    "7b": ([0], np.float32),   # 5.7e9 parameters x 2005 tokens: fp32 BLAS keeps the check to about a minute
+}
+
+
+@pytest.mark.parametrize("name", ["0.5b", "1.5b", "7b"])
+def test_full_size_workload(name):
+    w = synth.WORKLOADS[name]
+    rows, odt = PLAN[name]
+    case = Case(w, oracle_dtype=odt).prefill()
+    V = O.ValidSet(case.catalog, w.T)
+    assert case.n_unique == w.n_items == len(V)
+    # ---- hash set, bit exact
+    probe = synth.probe_keys_mix(w, case.catalog, 2_000_000)
+    keys = case.eng.pack(torch.from_numpy(probe).cuda())
+    assert np.array_equal(keys.cpu().numpy().view(np.uint64), O.pack_keys(probe, w.T))
+    assert np.array_equal(case.eng.probe(keys).cpu().numpy().astype(bool), V.contains(probe))
+    pre = case.catalog[np.random.default_rng(0).integers(0, len(case.catalog), 2000)]
+    sib = np.repeat(pre, w.T[-1], axis=0)
+    sib[:, -1] = np.tile(np.arange(w.T[-1]), len(pre))
+    got = case.eng.probe(case.eng.pack(torch.from_numpy(sib.astype(np.int32)).cuda())).cpu().numpy().astype(bool)
+    assert np.array_equal(got, V.contains(sib))
+    # ---- decode: invariants on every request
+    out = case.eng.decode(w.beam, mode=1, trace=True)
+    ar = case.eng.decode(w.beam, mode=2)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
+    assert torch.allclose(out["scores"], ar["scores"], atol=1e-4)
+    codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
+    live = np.arange(w.beam)[None, :] < count[:, None]
+    assert V.contains(codes[live]).all() and np.all(codes[~live] == -1)
+    assert 1 <= out["stats"].rounds <= w.L - 1
+    dr = case.eng.decode(w.beam, mode=0)
+    dcodes, dcount = dr["codes"].cpu().numpy(), dr["count"].cpu().numpy()
+    dlive = np.arange(w.beam)[None, :] < dcount[:, None]
+    assert V.contains(dcodes[dlive]).all()
+    # ---- oracle on a subset of requests
+    case._oracle = None
+    model, head, _ = case.oracle
+    h = case.eng.get_hidden().cpu().numpy()
+    beams = out["trace"]["beams"].cpu().numpy()
+    scores = out["trace"]["beam_scores"].cpu().numpy()
+    for b in rows:
+        assert np.abs(h[b] - case.req(b).h).max() < 4e-2
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam)
+        st = case.req(b).h[0]
+        z = head.logits(0, case.req(b).h[1], st)                     # draft head level 1 on the oracle's states
+    gotd = case.eng.draft_logits(w.beam, 0, None).cpu().numpy()
+    for b in rows:
+        assert np.abs(gotd[b, 0] - head.logits(0, case.req(b).h[1], case.req(b).h[0])).max() < tolerance(w)

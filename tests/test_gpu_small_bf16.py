@@ -9,7 +9,7 @@ import torch
 
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
-from gpu_helpers import Case, assert_topk_matches, tolerance
+from gpu_helpers import Case, assert_topk_matches, check_levels, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -17,20 +17,6 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def small():
     return Case(synth.WORKLOADS["small"]).prefill()
-
-
-def check_levels(case, b, beams, beam_scores, K, per_beam_all=True):
-    """beams [L, K, L] / beam_scores [L, K] of one request (GPU trace) against the oracle, level by level."""
-    w = case.w
-    model, _, V = case.oracle
-    req = case.req(b)
-    prev = [O.Beam((), np.float32(0.0))]
-    for n in range(w.L):
-        logits = model.next_level_logits_many(req, [bm.codes for bm in prev])
-        ref = O.expand_level(prev, logits, K, w.T[n], V if n == w.L - 1 else None)
-        cnt = int((beams[n, :, 0] >= 0).sum())
-        assert_topk_matches(beams[n][:, : n + 1], beam_scores[n], cnt, ref, K, tolerance(w))
-        prev = [O.Beam(tuple(int(c) for c in beams[n, k, : n + 1]), np.float32(beam_scores[n, k])) for k in range(cnt)]
 
 
 def test_small_hashset_full_catalogue(small):
