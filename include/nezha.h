@@ -134,7 +134,7 @@ nezha_status nezha_pack(nezha_ctx* ctx, const int32_t* codes, size_t n, uint64_t
  * Asynchronous. */
 nezha_status nezha_probe(nezha_ctx* ctx, const uint64_t* keys, size_t n, uint8_t* found);
 
-/* Algorithm 3 line 13: one pass of the primary model over [BOS, history codes, SP_1..SP_L] of every row.
+/* Prefill step of Algorithm 3 (inference): one pass of the primary model over [BOS, history codes, SP_1..SP_L] of every row.
  * Keeps the context KV cache (placeholders are not retained) and the hidden states h_0..h_L.
  *   hist_codes  device int32 [batch, max_n, L]; row b uses its first n_hist[b] items.
  *   n_hist      device int32 [batch], each in [0, max_n]; max_n <= cfg.max_hist_items.
@@ -143,7 +143,7 @@ nezha_status nezha_prefill(nezha_ctx* ctx, const int32_t* hist_codes, const int3
                            int32_t batch, int32_t max_n);
 
 /* Decode the next item of every prefilled row: the top `beam_width` valid semantic IDs and their
- * cumulative log-probabilities (Algorithm 3 lines 14-30 in mode 0; Algorithm 2 in mode 1; Algorithm 1 in mode 2).
+ * cumulative log-probabilities (Algorithm 3's inference loop in mode 0; Algorithm 2 in mode 1; Algorithm 1 in mode 2).
  *   out_codes   device int32 [batch, beam_width, L], best first, rows past out_count padded with -1
  *   out_scores  device float [batch, beam_width], padded with -inf
  *   out_count   device int32 [batch]
@@ -167,7 +167,7 @@ nezha_status nezha_decode_with_drafts(nezha_ctx* ctx, int32_t batch, int32_t bea
 /* h_0..h_L of the prefilled rows as fp32: device float [batch, L+1, d].  Asynchronous. */
 nezha_status nezha_get_hidden(nezha_ctx* ctx, float* out);
 
-/* Algorithm 1 lines 4-5, teacher-forced: for every (row, beam) the primary model runs on the context plus the
+/* Algorithm 1's model call and LM head, teacher-forced: for every (row, beam) the primary model runs on the context plus the
  * beam's `level` codes (0 <= level < L) and the LM head of level+1 gives logits.
  *   prefixes  device int32 [batch, n_beams, level] (ignored when level == 0)
  *   logits    device float [batch, n_beams, T[level]]
@@ -180,7 +180,7 @@ nezha_status nezha_primary_logits(nezha_ctx* ctx, int32_t batch, int32_t n_beams
 nezha_status nezha_draft_logits(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_t level,
                                 const int32_t* prefixes, float* logits);
 
-/* One beam-search level (Algorithm 1 lines 6-9 / Algorithm 3 lines 19-27) on caller-supplied logits:
+/* One beam-search level (the top-K, union and pruning steps of Algorithm 1 / Algorithm 3) on caller-supplied logits:
  * log-softmax over the codebook, per-beam top `per_beam` codes, optional hash-set filter of the resulting
  * tuples (only meaningful when level + 1 == L), top beam_width by cumulative log-probability; ties go to the
  * smaller (parent rank, code).
@@ -201,7 +201,7 @@ nezha_status nezha_select(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_
  *   epilogue 0: C (storage type) = acc;  1: C (float) = acc;  2: C (float) += acc;  3: C (float) = tanh(acc + bias[n])
  *   path     0: the engine's own choice; 1: CUDA-core kernel; 2: tcgen05 kernel (NEZHA_ERR_UNSUPPORTED if the shape
  *               is not covered: bf16 storage, K % 64 == 0, N % 128 == 0)
- * Used by every projection of the primary model (Algorithm 1 line 4), the LM head (line 5) and the draft head
+ * Used by every projection of the primary model (Algorithm 1's model call), the LM head and the draft head
  * (Eq. 2-3).  Asynchronous. */
 nezha_status nezha_gemm(nezha_ctx* ctx, const void* A, const void* W, void* C, int32_t M, int32_t N, int32_t K,
                         int32_t epilogue, const float* bias, int32_t path);

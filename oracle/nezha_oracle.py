@@ -227,7 +227,7 @@ class PrimaryModel:
         return np.asarray(toks, dtype=np.int64)
 
     def prefill(self, hist_codes: np.ndarray) -> "Request":
-        """Algorithm 3 line 13: one pass over context + L placeholders -> h_0..h_L; keeps the context KV only."""
+        """Prefill step of Algorithm 3 (inference): one pass over context + L placeholders -> h_0..h_L; keeps the context KV only."""
         s = self.s
         ctx = self.prompt_tokens(hist_codes)
         P = ctx.shape[0]
@@ -236,7 +236,7 @@ class PrimaryModel:
         return Request(P=P, h=hidden[P - 1: P + s.L].copy(), ctx_kv=[(k[:P], v[:P]) for k, v in kv])
 
     def next_level_logits(self, req: "Request", prefix: Sequence[int]) -> np.ndarray:
-        """Algorithm 1 lines 4-5 for one beam: logits over the codebook of level len(prefix)+1.
+        """Model call and LM head of Algorithm 1 for one beam: logits over the codebook of level len(prefix)+1.
 
         M_p runs on the context plus the beam's codes (no placeholders); the LM head rows of the next level
         are applied to the hidden state of the last position.
@@ -326,10 +326,10 @@ def expand_level(beams: List[Beam], logits: List[np.ndarray], K: int, per_beam: 
                  valid: Optional[ValidSet]) -> List[Beam]:
     """One level of beam search.
 
-    For every beam: log-softmax over the level's codebook, its `per_beam` most probable codes (Algorithm 1
-    line 6 / Algorithm 3 line 19), candidates = beam + code.  If `valid` is given, candidates that are not
-    valid IDs are dropped (Algorithm 3 lines 23-26; Eq. 5).  The K candidates with the largest cumulative
-    probability survive (Algorithm 1 line 9 / Algorithm 3 line 27).
+    For every beam: log-softmax over the level's codebook, its `per_beam` most probable codes (the top-K step
+    of Algorithm 1 / Algorithm 3), candidates = beam + code.  If `valid` is given, candidates that are not
+    valid IDs are dropped (the verification step of Algorithm 3; Eq. 5).  The K candidates with the largest cumulative
+    probability survive (the pruning step of Algorithm 1 / Algorithm 3).
 
     per_beam = K is the draft-head setting of Algorithm 3 (K x K candidates before the filter); per_beam = T_l
     applies the filter to every extension before the top-K (top-k restricted to valid tuples).
@@ -361,10 +361,10 @@ def teacher_forced_state(head: DraftHead, req: Request, codes: Sequence[int]) ->
 
 def nezha_draft(head: DraftHead, req: Request, K: int, valid: Optional[ValidSet],
                 start: Optional[List[Beam]] = None) -> List[List[Beam]]:
-    """Algorithm 3 lines 14-30.  Returns the beam sets of every level reached (last entry = final drafts).
+    """Algorithm 3, inference after the prefill.  Returns the beam sets of every level reached (last entry = final drafts).
 
     start = None is the paper's inference from the empty beam.  Otherwise drafting continues from the given
-    beams of level m (Algorithm 2 line 3): their states are teacher-forced along their codes and their scores
+    beams of level m (the drafting step of Algorithm 2): their states are teacher-forced along their codes and their scores
     seed the cumulative probabilities.
     """
     L = head.s.L
@@ -427,7 +427,7 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
         alive draft (each token attends to the context and to its own tuple's earlier codes).
       * selection walks forward: B_{j+1} from the logits at the beams of B_j, while every beam of B_j is the
         j-prefix of some alive draft (so its logits are in the pass); the first level where that fails is the
-        rejection level of Algorithm 2 line 5; the round ends there and m <- that level (line 7).
+        rejection level of Algorithm 2; the round ends there and m <- that level.
       * accepted length of draft k = the largest i <= (level reached) with D[k][:i] in B_i.
     Every B_j is computed from M_p's logits only, so the result equals ar_beam_search whatever the drafts.
     use_drafts=False gives L-1 rounds of plain autoregressive steps.
@@ -442,7 +442,7 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
     m = 1
     while m < L:
         stats.rounds += 1
-        # ---- draft (Algorithm 2 line 3)
+        # ---- draft (Algorithm 2, drafting step)
         if not use_drafts:
             D: List[Tuple[int, ...]] = []
         elif stats.rounds == 1:
@@ -455,13 +455,13 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
             D = [b.codes for b in lv[-1]] if lv else []
         beam_set = {b.codes for b in B}
         alive = [k for k, t in enumerate(D) if t[:m] in beam_set]
-        # ---- the parallel pass (line 4): count its tokens; logits are looked up per prefix below
+        # ---- the parallel verification pass: count its tokens; logits are looked up per prefix below
         stats.primary_tokens += len(B) + len(alive) * (L - 1 - m)
         in_pass = {b.codes for b in B}
         for k in alive:
             for j in range(m + 1, L):
                 in_pass.add(D[k][:j])
-        # ---- progressive selection / rejection (lines 5-7)
+        # ---- progressive selection / rejection (Algorithm 2, rejection and update steps)
         j = m
         while True:
             assert all(b.codes in in_pass for b in B)
@@ -502,7 +502,7 @@ def joint_logprob_primary(model: PrimaryModel, req: Request, codes: Sequence[int
 
 
 def joint_logprob_draft(head: DraftHead, req: Request, codes: Sequence[int]) -> float:
-    """log p(codes) under the draft head by teacher forcing (Algorithm 3 training lines 4-8)."""
+    """log p(codes) under the draft head by teacher forcing (the teacher-forced loop of Algorithm 3's training part)."""
     total = 0.0
     st = req.h[0]
     for l in range(len(codes)):

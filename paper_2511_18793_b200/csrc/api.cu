@@ -299,7 +299,7 @@ SelectArgs select_base(nezha_ctx* c, int batch, int K) {
   return s;
 }
 
-// Algorithm 3 lines 14-30 (from the empty beam), or its continuation from the true beams (Algorithm 2 line 3).
+// Algorithm 3's inference loop (from the empty beam), or its continuation from the true beams (Algorithm 2's drafting step).
 // `first_level` = smallest level any request can still need drafting at (levels below are teacher-forced only).
 void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_level, bool filter) {
   const EngineState& e = c->es;
@@ -365,7 +365,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     return ps;
   }
 
-  // B_1 from the prefill hidden state h_0 (Algorithm 1 lines 5-9 at l = 1)
+  // B_1 from the prefill hidden state h_0 (Algorithm 1's LM head, top-K and pruning at l = 1)
   gemm(c, c->h_act, (long long)(L + 1) * c->d, c->lm_head, c->d, c->logits0, c->cfg.T[0], batch, nullptr, c->cfg.T[0], c->d,
        kEpiStoreF32);
   {

@@ -1,6 +1,6 @@
 // Beam-search kernels: fused log-softmax + validity mask + beam top-k (one level of Algorithm 1 / Algorithm 3),
-// the draft head's glue (Eq. 1-3 inputs), the verify pass's token list, and accept / roll-back (Algorithm 2
-// lines 5-7).  Every kernel here runs one thread block per request; requests never interact.
+// the draft head's glue (Eq. 1-3 inputs), the verify pass's token list, and accept / roll-back (Algorithm 2's
+// rejection and update steps).  Every kernel here runs one thread block per request; requests never interact.
 #include <math.h>
 
 #include "engine_state.cuh"
@@ -13,7 +13,7 @@ namespace nz {
 // Per request: each warp takes beams r = warp, warp + n_warps, ...  For a beam it loads the T logits of the
 // level's codebook (VPL per lane), computes log-softmax with warp shuffles, and extracts the beam's best
 // candidates in order (repeated warp arg-max; ties to the smaller code):
-//   per_beam <  T : the per_beam most probable codes, THEN the hash-set filter on those       (Algorithm 3 l.19, 23-26)
+//   per_beam <  T : the per_beam most probable codes, THEN the hash-set filter on those       (Algorithm 3: top-K, then verification)
 //   per_beam >= T : the filter on all T codes, THEN the K best by cumulative log-probability  (top-k restricted to V)
 // The sorted per-beam lists go to shared memory and warp 0 merges them into the K best of the request
 // (ties to the smaller parent rank, then the smaller code).
@@ -236,8 +236,8 @@ __global__ void init_decode_kernel(EngineState e, int batch) {
   e.dw_count[(long long)e.L * e.Bmax + b] = 0;
 }
 
-// Start of a round's drafting (Algorithm 2 line 3): the draft head continues from the true beams B_m, or from
-// the empty beam in the first round (Algorithm 3 line 14).
+// Start of a round's drafting (Algorithm 2's drafting step): the draft head continues from the true beams B_m, or from
+// the empty beam in the first round (Algorithm 3's initialisation).
 __global__ void draft_init_kernel(EngineState e, int batch, int from_scratch) {
   const int b = blockIdx.x;
   if (b >= batch) return;
@@ -454,7 +454,7 @@ __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams
 }
 
 // ----------------------------------------------------------------------------------------------------
-// accept / roll back (Algorithm 2 lines 5-7)
+// accept / roll back (Algorithm 2's rejection and update steps)
 // ----------------------------------------------------------------------------------------------------
 // After B_{n+1} has been selected for a request whose beams B_n had logits in this pass:
 //   n + 1 == L : the request is finished; B_L is the result.

@@ -3,7 +3,7 @@ catalogues), in the launch configuration bench.py times.
 
 All requests: GPU-internal invariants (verified decode == plain autoregressive decode item for item; every emitted
 tuple is in the exact valid set; counts and padding).  A fixed subset of requests: the oracle recomputes every
-beam level from the GPU's own beams (tie rule) and the prefill hidden states.  The hash set is probed with a
+beam level from the GPU's own beams (tie rule), the prefill hidden states and the draft head's first-level logits.  The hash set is probed with a
 hit/miss mix and with sibling keys and compared bit for bit with the exact set."""
 import numpy as np
 import pytest
@@ -11,7 +11,7 @@ import torch
 
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
-from gpu_helpers import Case, check_levels, tolerance
+from gpu_helpers import Case, check_levels, e2e_tolerance, hidden_rms_bound, hidden_tolerance, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -59,10 +59,15 @@ def test_full_size_workload(name):
     beams = out["trace"]["beams"].cpu().numpy()
     scores = out["trace"]["beam_scores"].cpu().numpy()
     for b in rows:
-        assert np.abs(h[b] - case.req(b).h).max() < 4e-2
-        check_levels(case, b, beams[:, b], scores[:, b], w.beam)
-        st = case.req(b).h[0]
-        z = head.logits(0, case.req(b).h[1], st)                     # draft head level 1 on the oracle's states
+        dh = h[b] - case.req(b).h
+        assert np.abs(dh).max() < hidden_tolerance(w) and np.sqrt((dh ** 2).mean()) < hidden_rms_bound(w)
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam, tol=e2e_tolerance(w))
+    # draft head, stage-wise: the oracle's Eq. 1-2 on the hidden states the GPU's prefill produced (float64 copies of
+    # the same numbers), so that the 2e-2 budget is spent by the draft head alone and not by 24-32 layers of bf16
+    # activations upstream; end to end (oracle hidden states) the same logits stay within the depth-scaled bound
+    # (h_l + s_1 carries two hidden-state errors, hence the factor)
     gotd = case.eng.draft_logits(w.beam, 0, None).cpu().numpy()
     for b in rows:
-        assert np.abs(gotd[b, 0] - head.logits(0, case.req(b).h[1], case.req(b).h[0])).max() < tolerance(w)
+        hg = h[b].astype(np.float64)
+        assert np.abs(gotd[b, 0] - head.logits(0, hg[1], hg[0])).max() < tolerance(w)
+        assert np.abs(gotd[b, 0] - head.logits(0, case.req(b).h[1], case.req(b).h[0])).max() < 1.5 * e2e_tolerance(w)
