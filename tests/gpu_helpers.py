@@ -27,6 +27,16 @@ def hidden_tolerance(w):
     return 1e-4 if w.dtype == "fp32" else 5.0 * hidden_rms_bound(w)
 
 
+def stage_tolerance(w, w_std, x_rms):
+    """One stage on identical inputs whose d-vector (rms x_rms) is rounded once to bf16 before a [T, d] matmul with
+    weights of the given std: each logit is off by ||row|| * x_rms * 1.6e-3 rms; 4 sigma over a codebook, never below
+    the 2e-2 budget (which it exceeds only for the noise-perturbed draft head of the 7B-shaped workload, whose
+    logits are several times larger than everyone else's)."""
+    if w.dtype == "fp32":
+        return tolerance(w)
+    return max(tolerance(w), 4.0 * w_std * np.sqrt(w.d_model) * x_rms * 1.6e-3)
+
+
 def e2e_tolerance(w, std=0.02):
     """Largest logit deviation of the whole pipeline: a logit is a dot product of a weight row (d entries of the given
     std) with the hidden state, so it inherits ||row|| * rms(hidden error), 4 sigma of which over a codebook; never
