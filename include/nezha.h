@@ -206,6 +206,35 @@ nezha_status nezha_select(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_
 nezha_status nezha_gemm(nezha_ctx* ctx, const void* A, const void* W, void* C, int32_t M, int32_t N, int32_t K,
                         int32_t epilogue, const float* bias, int32_t path);
 
+/* ---- for callers that cannot allocate device memory (the paper has no counterpart) ------------------------ */
+
+/* Largest n nezha_contains_noalloc accepts.  The library image carries a key buffer of this many 8-byte entries
+ * (8 MiB), which every GPU that loads the library holds until the process exits. */
+#define NEZHA_NOALLOC_MAX_TUPLES (1u << 20)
+
+/* Eq. 4 + Eq. 5 in one call without any allocation: found[i] = 1 if the code tuple codes[i, :] is a valid
+ * semantic ID, else 0.  Same result as nezha_pack followed by nezha_probe, but the packed keys in between are kept
+ * in a fixed buffer inside the library instead of a buffer somebody has to allocate.
+ *
+ * It exists for callers that must not, or cannot, call cudaMalloc (directly or through an allocating framework)
+ * at the point where they need the answer: a serving loop that handed all device memory to its own pool at
+ * start-up, a host thread inside a latency-critical section where cudaMalloc's implicit device synchronisation is
+ * not acceptable, a plug-in that was given buffers but no allocator.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating routine; the caller still provides the input and the output.
+ *
+ *   codes  device int32 [n, L]      found  device uint8 [n]      n <= NEZHA_NOALLOC_MAX_TUPLES
+ *
+ * Asynchronous on the context's stream.  Errors: NEZHA_ERR_ARG (null pointer; n above the maximum, with a message
+ * saying so), NEZHA_ERR_STATE (before nezha_build_hashset), NEZHA_ERR_CUDA.  A code outside [0, T_l) sets
+ * NEZHA_ERR_CATALOG, reported by the next synchronising call; that tuple reads as not found.
+ *
+ * The first call on a device looks up the device address of the built-in buffer (the GPU of the context must be
+ * the current device); make that first call before starting any stream capture.  The buffer is one per device and
+ * shared by all contexts and streams: it keeps the previous call's keys (each call overwrites the entries it then
+ * reads, nothing has to be cleared), and two calls whose kernels can overlap on the GPU -- different streams,
+ * different contexts, different host threads -- race on it.  Serialise them. */
+nezha_status nezha_contains_noalloc(nezha_ctx* ctx, const int32_t* codes, size_t n, uint8_t* found);
+
 /* ---- instrumentation (the paper has no counterpart: these only measure the library itself) -------------- */
 
 #define NEZHA_PROFILE_CLASSES 16

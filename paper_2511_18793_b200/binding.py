@@ -63,6 +63,8 @@ lib.nezha_pack.restype = C.c_int
 lib.nezha_pack.argtypes = [_vp, _vp, _sz, _vp]
 lib.nezha_probe.restype = C.c_int
 lib.nezha_probe.argtypes = [_vp, _vp, _sz, _vp]
+lib.nezha_contains_noalloc.restype = C.c_int
+lib.nezha_contains_noalloc.argtypes = [_vp, _vp, _sz, _vp]
 lib.nezha_prefill.restype = C.c_int
 lib.nezha_prefill.argtypes = [_vp, _vp, _vp, _i32, _i32]
 lib.nezha_decode.restype = C.c_int
@@ -99,7 +101,9 @@ lib.nezha_last_error.argtypes = [_vp]
 lib.nezha_destroy.restype = None
 lib.nezha_destroy.argtypes = [_vp]
 
-EXPORTS = ["nezha_arena_bytes", "nezha_create", "nezha_build_hashset", "nezha_pack", "nezha_probe", "nezha_prefill",
+NOALLOC_MAX_TUPLES = 1 << 20
+EXPORTS = ["nezha_arena_bytes", "nezha_create", "nezha_build_hashset", "nezha_pack", "nezha_probe",
+           "nezha_contains_noalloc", "nezha_prefill",
            "nezha_decode", "nezha_decode_with_drafts", "nezha_get_hidden", "nezha_primary_logits",
            "nezha_draft_logits", "nezha_select", "nezha_gemm", "nezha_launch_count", "nezha_profile_enable",
            "nezha_profile_read", "nezha_sync", "nezha_last_error", "nezha_destroy"]
@@ -208,6 +212,13 @@ class Engine:
     def probe(self, keys: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         found = out if out is not None else torch.empty(keys.shape[0], dtype=torch.uint8, device=keys.device)
         self._check(lib.nezha_probe(self._h, _ptr(keys), keys.shape[0], _ptr(found)))
+        return found
+
+    def contains_noalloc(self, codes: torch.Tensor, found: torch.Tensor) -> torch.Tensor:
+        """nezha_contains_noalloc: validity of code tuples with no allocation anywhere; `codes` (int32 [n, L],
+        contiguous) and `found` (uint8 [n]) are the caller's, and this method creates no tensor either."""
+        assert codes.dtype == torch.int32 and found.dtype == torch.uint8 and found.shape[0] == codes.shape[0]
+        self._check(lib.nezha_contains_noalloc(self._h, _ptr(codes), codes.shape[0], _ptr(found)))
         return found
 
     def prefill(self, hist_codes: torch.Tensor, n_hist: torch.Tensor):

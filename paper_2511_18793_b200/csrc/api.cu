@@ -686,6 +686,51 @@ nezha_status nezha_sync(nezha_ctx* c) {
   return pending_device_error(c);
 }
 
+// ---- membership test for callers that cannot allocate device memory ------------------------------------
+// The packed keys of the tuples are an intermediate result: nezha_pack writes them to a caller-allocated buffer and
+// nezha_probe reads them back.  Here they live in a fixed array that is part of the loaded library image instead,
+// so nothing is allocated by anyone.  The array is shared by every call on the device and keeps whatever the last
+// call wrote; each call overwrites the first n entries before it reads them, so nothing needs clearing.
+static __device__ __align__(256) unsigned long long g_noalloc_keys[NEZHA_NOALLOC_MAX_TUPLES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned long long* g_noalloc_keys_addr[kMaxDevices] = {nullptr};   // device address of the array, per device
+
+// `g_noalloc_keys` in host code is only a handle of the symbol; the address a kernel can use has to be asked for,
+// once per device, with that device current.
+cudaError_t noalloc_keys_address(unsigned long long** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_noalloc_keys_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_keys);
+    if (e != cudaSuccess) return e;
+    g_noalloc_keys_addr[dev] = static_cast<unsigned long long*>(p);
+  }
+  *out = g_noalloc_keys_addr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+nezha_status nezha_contains_noalloc(nezha_ctx* c, const int32_t* codes, size_t n, uint8_t* found) {
+  if (!c) return NEZHA_ERR_ARG;
+  if (n && (!codes || !found)) return fail(c, NEZHA_ERR_ARG, "nezha_contains_noalloc: null pointer");
+  if (n > (size_t)NEZHA_NOALLOC_MAX_TUPLES)
+    return fail(c, NEZHA_ERR_ARG, "nezha_contains_noalloc: n exceeds NEZHA_NOALLOC_MAX_TUPLES (the size of the built-in "
+                                  "key buffer); split the request or use nezha_pack + nezha_probe");
+  if (c->state < 1) return fail(c, NEZHA_ERR_STATE, "nezha_contains_noalloc before nezha_build_hashset");
+  if (!n) return NEZHA_OK;
+  unsigned long long* keys = nullptr;
+  NZ_CUDA(c, noalloc_keys_address(&keys));
+  launch_hs_pack(c->es.li, codes, n, keys, c->es.status, c->st);
+  launch_hs_probe(c->es.hs, keys, n, found, c->st);
+  NZ_CUDA(c, cudaGetLastError());
+  return NEZHA_OK;
+}
+
 const char* nezha_last_error(const nezha_ctx* c) { return c ? c->err.c_str() : "null context"; }
 
 void nezha_destroy(nezha_ctx* c) {
