@@ -25,6 +25,7 @@ void profile_enable(bool on);
 void profile_read(nezha_profile* out);
 bool gemm_tc_supported(const GemmArgs& a);
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
+int gemm_tc_norm_parts(int M, int N);
 bool attention_tc_supported(const AttnArgs& a);
 void launch_attention_tc(const AttnArgs& a, cudaStream_t st);
 }  // namespace nz
@@ -67,6 +68,9 @@ struct nezha_ctx {
   // scratch
   float* resid; void *xn, *qkv, *attn, *gu, *act, *xd, *a_se, *h_act;
   float *h_f32, *logits_v, *logits0, *logits_d;
+  // fused tensor-core path: RMSNorm split around the GEMMs (partial sums of squares per output tile), SwiGLU and
+  // rotary embedding + KV append in GEMM epilogues; weights of q/k heads and gate/up re-laid-out to match
+  bool fused; float *ss_a, *ss_b, *ss_e;
   int* h_rows; unsigned long long* n_unique_dev;
   EngineState es;
   int* host_counters;       // pinned
@@ -193,6 +197,13 @@ size_t carve(nezha_ctx* c) {
   c->logits0 = cv.take<float>((size_t)c->Bmax * g.T[0]);
   c->logits_d = cv.take<float>((size_t)c->Bmax * c->Kmax * c->Tmax);
   c->h_rows = cv.take<int>((size_t)c->Bmax * (c->L + 1));
+  c->fused = c->bf16 && (c->hd == 64 || c->hd == 128) && c->d % 64 == 0 && c->F % 64 == 0;
+  c->ss_a = c->ss_b = c->ss_e = nullptr;
+  if (c->fused) {
+    c->ss_a = cv.take<float>((size_t)(c->d / 16) * c->Ms);      // up to two partial sums per 32-column tile
+    c->ss_b = cv.take<float>((size_t)(c->d / 16) * c->Ms);
+    c->ss_e = cv.take<float>((size_t)c->Ms);
+  }
   // engine state
   const size_t lbk = (size_t)(c->L + 1) * c->Bmax * c->Kmax;
   e.tb_codes = cv.take<int>(lbk * c->L); e.tb_score = cv.take<float>(lbk); e.tb_parent = cv.take<int>(lbk);
@@ -219,6 +230,63 @@ void gemm(nezha_ctx* c, const void* A, long long lda, const void* W, long long l
   GemmArgs a{A, lda, W, ldw, C, ldc, (int)M, M_dev, N, K, epi, bias, c->es.status};
   if (c->bf16 && gemm_tc_supported(a)) launch_gemm_tc(a, c->st);
   else launch_gemm_simt(a, c->bf16, c->st);
+}
+
+// A projection of the fused tensor-core path.  ss_in / parts: partial sums of squares of the A operand's rows (its
+// RMSNorm scale is applied in the epilogue), or null.  Returns the number of column tiles (= partial sums written
+// by a kEpiAddNorm epilogue) of such a launch.
+int gemm_fused(nezha_ctx* c, const void* A, long long lda, const void* W, void* C, long long ldc, long long M,
+               const int* M_dev, int N, int K, int epi, const float* ss_in, int ss_parts, const GemmFuse* extra) {
+  GemmArgs a{A, lda, W, (long long)K, C, ldc, (int)M, M_dev, N, K, epi, nullptr, c->es.status};
+  if (extra) a.f = *extra;
+  a.f.ss_in = ss_in; a.f.ss_in_parts = ss_parts; a.f.ss_ld = c->Ms; a.f.inv_dim = 1.f / (float)c->d; a.f.eps = c->cfg.rms_eps;
+  launch_gemm_tc(a, c->st);
+  return gemm_tc_norm_parts((int)M, N);
+}
+
+// The layers of the primary model on the fused path.  On entry resid holds the embeddings, xn = embedding * gain of
+// the first attention norm and ss_e the rows' sums of squares (launch_embed_norm).  Five kernels per layer:
+// QKV projection (+ norm scale, rotary embedding, KV append) -> attention -> output projection (+ residual, next
+// norm input) -> gate/up projection (+ norm scale, SwiGLU) -> down projection (+ residual, next norm input).
+// On exit xn = resid * final-norm gain and *ss_out / *parts_out describe its row scale.
+void run_layers_fused(nezha_ctx* c, long long M, const int* M_dev, bool verify, int n_rows, int max_tok_per_row,
+                      const float** ss_out, int* parts_out) {
+  const EngineState& e = c->es;
+  const size_t esz = c->esz;
+  const float* ss_cur = c->ss_e; int parts_cur = 1;
+  for (int i = 0; i < c->nl; ++i) {
+    const LayerW& w = c->layers[i];
+    char* kc = (char*)c->k_ctx + (size_t)i * c->ctx_layer_elems * esz;
+    char* vc = (char*)c->v_ctx + (size_t)i * c->ctx_layer_elems * esz;
+    char* ke = (char*)c->k_ext + (size_t)i * c->ext_layer_elems * esz;
+    char* ve = (char*)c->v_ext + (size_t)i * c->ext_layer_elems * esz;
+    GemmFuse fr{};
+    fr.tok_pos = e.tok_pos; fr.kv_dst = e.tok_kv_dst; fr.kv_head_stride = verify ? c->hd : (long long)c->S * c->hd;
+    fr.k_cache = verify ? ke : kc; fr.v_cache = verify ? ve : vc; fr.cos_tab = c->rope_cos; fr.sin_tab = c->rope_sin;
+    fr.Hq = c->Hq; fr.Hkv = c->Hkv; fr.hd = c->hd;
+    gemm_fused(c, c->xn, c->d, w.wqkv, c->qkv, c->qkv_dim, M, M_dev, c->qkv_dim, c->d, kEpiRopeKV, ss_cur, parts_cur, &fr);
+    AttnArgs t{};
+    t.q = c->qkv; t.q_stride = c->qkv_dim; t.out = c->attn; t.out_stride = (long long)c->Hq * c->hd;
+    t.k_ctx = kc; t.v_ctx = vc; t.ctx_row_stride = (long long)c->Hkv * c->S * c->hd; t.ctx_head_stride = (long long)c->S * c->hd;
+    t.k_ext = ke; t.v_ext = ve; t.ext_head_stride = c->hd;
+    t.tok_row = e.tok_row; t.tok_ctx_len = e.tok_ctx_len; t.tok_ext = e.tok_ext; t.n_ext_max = verify ? c->L : 0;
+    t.M = (int)M; t.M_dev = M_dev; t.Hq = c->Hq; t.Hkv = c->Hkv; t.hd = c->hd; t.scale = 1.f / sqrtf((float)c->hd);
+    t.row_start = verify ? e.row_tok_start : e.pf_row_start; t.row_count = verify ? e.row_tok_count : e.pf_row_count;
+    t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
+    t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
+    if (attention_tc_supported(t)) launch_attention_tc(t, c->st);
+    else launch_attention_simt(t, true, c->st);
+    GemmFuse fo{};
+    fo.xg = c->xn; fo.gain = w.mlp_norm; fo.ss_out = c->ss_a;
+    const int parts_a = gemm_fused(c, c->attn, (long long)c->Hq * c->hd, w.wo, c->resid, c->d, M, M_dev, c->d, c->Hq * c->hd,
+                                   kEpiAddNorm, nullptr, 0, &fo);
+    gemm_fused(c, c->xn, c->d, w.w_gu, c->act, c->F, M, M_dev, 2 * c->F, c->d, kEpiSwiGLU, c->ss_a, parts_a, nullptr);
+    GemmFuse fd{};
+    fd.xg = c->xn; fd.gain = (i + 1 < c->nl) ? c->layers[i + 1].attn_norm : c->final_norm; fd.ss_out = c->ss_b;
+    parts_cur = gemm_fused(c, c->act, c->F, w.w_down, c->resid, c->d, M, M_dev, c->d, c->F, kEpiAddNorm, nullptr, 0, &fd);
+    ss_cur = c->ss_b;
+  }
+  *ss_out = ss_cur; *parts_out = parts_cur;
 }
 
 // One pass of the primary model's layers over the tokens described by es.tok_* (resid already holds the
@@ -268,11 +336,19 @@ void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify, int n_
 void verify_pass(nezha_ctx* c, long long M_bound, int n_rows, int max_tok_per_row) {
   const EngineState& e = c->es;
   if (M_bound <= 0 || c->L < 2) return;
+  const char* w = (const char*)c->lm_head + (size_t)e.li.off[1] * c->d * c->esz;
+  if (c->fused) {
+    launch_embed_norm(c->embed, e.tok_id, (int)M_bound, e.n_tokens, c->d, c->resid, c->layers[0].attn_norm, c->xn, c->ss_e,
+                      c->st);
+    const float* ss; int parts;
+    run_layers_fused(c, M_bound, e.n_tokens, true, n_rows, max_tok_per_row, &ss, &parts);
+    gemm_fused(c, c->xn, c->d, w, c->logits_v, c->Nv, M_bound, e.n_tokens, c->Nv, c->d, kEpiStoreF32, ss, parts, nullptr);
+    return;
+  }
   launch_embed(c->embed, c->bf16, e.tok_id, (int)M_bound, e.n_tokens, c->d, c->resid, c->st);
   run_layers(c, M_bound, e.n_tokens, true, n_rows, max_tok_per_row);
   launch_rmsnorm(c->resid, c->d, nullptr, c->final_norm, c->bf16, c->xn, nullptr, (int)M_bound, e.n_tokens, c->d,
                  c->cfg.rms_eps, c->st);
-  const char* w = (const char*)c->lm_head + (size_t)e.li.off[1] * c->d * c->esz;
   gemm(c, c->xn, c->d, w, c->d, c->logits_v, c->Nv, M_bound, e.n_tokens, c->Nv, c->d, kEpiStoreF32);
 }
 
@@ -450,6 +526,11 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   c->host_counters = nullptr;
   if (cudaMallocHost((void**)&c->host_counters, 16 * sizeof(int)) != cudaSuccess) return bail(NEZHA_ERR_CUDA);
   if (select_configure(c->Kmax) != cudaSuccess) return bail(NEZHA_ERR_CUDA);
+  if (c->fused) {                  // needs the tensor-core GEMM (TMA descriptors) for every projection
+    GemmArgs probe{c->xn, c->d, c->layers[0].wqkv, c->d, c->qkv, c->qkv_dim, 128, nullptr, c->qkv_dim, c->d, kEpiStoreAct, nullptr,
+                   c->es.status};
+    if (!gemm_tc_supported(probe)) c->fused = false;
+  }
   const size_t esz = c->esz;
   cudaStream_t st = c->st;
   auto cp = [&](void* dst, const void* src, size_t bytes) {
@@ -469,8 +550,14 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
     ok = ok && w->attn_norm && w->wq && w->wk && w->wv && w->wo && w->mlp_norm && w->w_gate && w->w_up && w->w_down;
     ok = ok && cp(lw.attn_norm, w->attn_norm[i], (size_t)c->d * esz) && cp(lw.wqkv, w->wq[i], q_b) &&
          cp((char*)lw.wqkv + q_b, w->wk[i], kv_b) && cp((char*)lw.wqkv + q_b + kv_b, w->wv[i], kv_b) &&
-         cp(lw.wo, w->wo[i], q_b) && cp(lw.mlp_norm, w->mlp_norm[i], (size_t)c->d * esz) &&
-         cp(lw.w_gu, w->w_gate[i], f_b) && cp((char*)lw.w_gu + f_b, w->w_up[i], f_b) && cp(lw.w_down, w->w_down[i], f_b);
+         cp(lw.wo, w->wo[i], q_b) && cp(lw.mlp_norm, w->mlp_norm[i], (size_t)c->d * esz) && cp(lw.w_down, w->w_down[i], f_b);
+    if (ok && c->fused) {          // rows of the q / k heads grouped into rotary pairs; gate and up rows interleaved
+      launch_permute_rotary_rows(w->wq[i], lw.wqkv, c->Hq * c->hd, c->hd, c->d, st);
+      launch_permute_rotary_rows(w->wk[i], (char*)lw.wqkv + q_b, c->Hkv * c->hd, c->hd, c->d, st);
+      launch_interleave_gate_up(w->w_gate[i], w->w_up[i], lw.w_gu, c->F, c->d, st);
+    } else {
+      ok = ok && cp(lw.w_gu, w->w_gate[i], f_b) && cp((char*)lw.w_gu + f_b, w->w_up[i], f_b);
+    }
   }
   for (int l = 0; ok && l < c->L; ++l)
     ok = ok && w->draft_logit && cp(c->draft_logit[l], w->draft_logit[l], (size_t)cfg->T[l] * c->d * esz);
@@ -545,8 +632,14 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
     const int rows = (batch - b0 < c->chunk_rows) ? batch - b0 : c->chunk_rows;
     const long long M = (long long)rows * S_call;
     launch_prefill_tokens(e, hist_codes, n_hist, b0, rows, max_n, S_call, c->S, c->h_rows, c->st);
-    launch_embed(c->embed, c->bf16, e.tok_id, (int)M, nullptr, c->d, c->resid, c->st);
-    run_layers(c, M, nullptr, false, rows, S_call);
+    if (c->fused) {
+      launch_embed_norm(c->embed, e.tok_id, (int)M, nullptr, c->d, c->resid, c->layers[0].attn_norm, c->xn, c->ss_e, c->st);
+      const float* ss; int parts;
+      run_layers_fused(c, M, nullptr, false, rows, S_call, &ss, &parts);
+    } else {
+      launch_embed(c->embed, c->bf16, e.tok_id, (int)M, nullptr, c->d, c->resid, c->st);
+      run_layers(c, M, nullptr, false, rows, S_call);
+    }
     const size_t ho = (size_t)b0 * (c->L + 1) * c->d;
     launch_rmsnorm(c->resid, c->d, c->h_rows, c->final_norm, c->bf16, (char*)c->h_act + ho * c->esz, c->h_f32 + ho,
                    rows * (c->L + 1), nullptr, c->d, c->cfg.rms_eps, c->st);

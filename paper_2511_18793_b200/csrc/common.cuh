@@ -109,7 +109,23 @@ enum GemmEpilogue : int {
   kEpiStoreF32 = 1,     // C (float) = acc
   kEpiAddF32 = 2,       // C (float) += acc                    (residual stream)
   kEpiBiasTanhF32 = 3,  // C (float) = tanh(acc + bias[n])     (Eq. 3)
-  kEpiSwiGLU = 4        // C (activation type)[m, n/2] = silu(acc[m, n]) * acc[m, n+1] on interleaved columns
+  // ---- fused epilogues of the tensor-core kernel only -------------------------------------------------------
+  kEpiSwiGLU = 4,       // weight rows interleaved [16 gate, 16 up]: C (act)[m, n/2 ..] = silu(gate) * up
+  kEpiAddNorm = 5,      // C (float) += acc; xg (act)[m, n] = C * gain[n]; ss_out[tile_n][m] = sum_n C^2 (this tile)
+  kEpiRopeKV = 6        // fused QKV projection: rotary embedding on q and k, q to C, k and v to the KV cache
+};
+
+// Extras of the fused epilogues.  RMSNorm is split around the GEMMs: the producer of the residual stream
+// (kEpiAddNorm) leaves x * gain as the next GEMM's A operand and per-tile partial sums of x^2; the consumer GEMM
+// multiplies its accumulator rows by rsqrt(mean(x^2) + eps), summing the partials in a fixed order.
+struct GemmFuse {
+  const float* ss_in; int ss_in_parts; long long ss_ld; float inv_dim, eps;   // row scale of the A operand (or null)
+  float* ss_out;                     // [N / tile_n][ss_ld]
+  void* xg; const void* gain;        // kEpiAddNorm: next A operand [M, N] (activation type) and its norm gain [N]
+  // kEpiRopeKV: weight rows of every q / k head permuted so that each 32-column group holds 16 rotary pairs
+  const int* tok_pos; const long long* kv_dst; long long kv_head_stride;
+  void* k_cache; void* v_cache; const float* cos_tab; const float* sin_tab;
+  int Hq, Hkv, hd;
 };
 
 struct GemmArgs {
@@ -122,6 +138,7 @@ struct GemmArgs {
   int epilogue;
   const float* bias;
   int* status;           // device status word (bounded waits report here)
+  GemmFuse f;            // zero-initialised unless a fused epilogue is asked for
 };
 
 void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);
@@ -131,6 +148,10 @@ void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);
 // --------------------------------------------------------------------------------------------------
 void launch_embed(const void* table, bool bf16, const int* tokens, int M, const int* M_dev, int d, float* resid,
                   cudaStream_t st);
+void launch_embed_norm(const void* table, const int* tokens, int M, const int* M_dev, int d, float* resid,
+                       const void* gain, void* xg, float* ss, cudaStream_t st);
+void launch_permute_rotary_rows(const void* src, void* dst, int rows, int hd, int cols, cudaStream_t st);
+void launch_interleave_gate_up(const void* gate, const void* up, void* dst, int F, int cols, cudaStream_t st);
 void launch_rmsnorm(const float* x, long long x_stride, const int* row_index, const void* gain, bool bf16, void* out,
                     float* out_f32, int M, const int* M_dev, int d, float eps, cudaStream_t st);
 

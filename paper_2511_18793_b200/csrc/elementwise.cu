@@ -90,6 +90,66 @@ __global__ void swiglu_kernel(const T* __restrict__ gu, T* __restrict__ act, int
   }
 }
 
+// Embedding gather fused with the first layer's RMSNorm input: resid = e (fp32), xg = e * gain (bf16, the first
+// GEMM's A operand) and ss[i] = sum(e^2) (the row scale is applied in that GEMM's epilogue).  One block per token.
+__global__ void embed_norm_kernel(const __nv_bfloat16* __restrict__ table, const int* __restrict__ tokens, int M,
+                                  const int* M_dev, int d, float* __restrict__ resid,
+                                  const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xg,
+                                  float* __restrict__ ss) {
+  const int m = M_dev ? min(M, *M_dev) : M;
+  const int i = blockIdx.x;
+  if (i >= m) return;
+  const __nv_bfloat16* src = table + (long long)tokens[i] * d;
+  float part = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = __bfloat162float(src[c]);
+    resid[(long long)i * d + c] = v;
+    xg[(long long)i * d + c] = __float2bfloat16_rn(v * __bfloat162float(gain[c]));
+    part += v * v;
+  }
+  __shared__ float red[4];
+  part = warp_sum(part);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = part;
+  __syncthreads();
+  if (threadIdx.x == 0) ss[i] = red[0] + red[1] + red[2] + red[3];
+}
+
+// Weight re-layouts of the fused tensor-core path (run once, at context creation).
+//   rotary: inside every head of hd rows, output rows [32 g, 32 g + 16) are input rows [16 g, 16 g + 16) and output
+//           rows [32 g + 16, 32 g + 32) are input rows [hd/2 + 16 g, ...): every 32-row group holds 16 rotary pairs.
+//   gate/up: output rows [32 t, 32 t + 16) are gate rows [16 t, ...), rows [32 t + 16, 32 t + 32) the matching up rows.
+__global__ void permute_rotary_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
+                                           int hd, int cols) {
+  const int r = blockIdx.x;
+  const int h = r / hd, w = r % hd, g = w >> 5, j = w & 31;
+  const int sr = h * hd + (j < 16 ? 16 * g + j : (hd >> 1) + 16 * g + (j - 16));
+  for (int c = threadIdx.x; c < cols; c += blockDim.x) dst[(long long)r * cols + c] = src[(long long)sr * cols + c];
+}
+__global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ gate, const __nv_bfloat16* __restrict__ up,
+                                          __nv_bfloat16* __restrict__ dst, int cols) {
+  const int r = blockIdx.x;
+  const int t = r >> 5, j = r & 31;
+  const __nv_bfloat16* src = (j < 16 ? gate + (long long)(16 * t + j) * cols : up + (long long)(16 * t + j - 16) * cols);
+  for (int c = threadIdx.x; c < cols; c += blockDim.x) dst[(long long)r * cols + c] = src[c];
+}
+
+void launch_embed_norm(const void* table, const int* tokens, int M, const int* M_dev, int d, float* resid,
+                       const void* gain, void* xg, float* ss, cudaStream_t st) {
+  if (M <= 0) return;
+  LaunchScope ls(kcEmbed, st);
+  embed_norm_kernel<<<M, 128, 0, st>>>((const __nv_bfloat16*)table, tokens, M, M_dev, d, resid,
+                                       (const __nv_bfloat16*)gain, (__nv_bfloat16*)xg, ss);
+}
+void launch_permute_rotary_rows(const void* src, void* dst, int rows, int hd, int cols, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
+  permute_rotary_rows_kernel<<<rows, 128, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, hd, cols);
+}
+void launch_interleave_gate_up(const void* gate, const void* up, void* dst, int F, int cols, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
+  interleave_gate_up_kernel<<<2 * F, 128, 0, st>>>((const __nv_bfloat16*)gate, (const __nv_bfloat16*)up,
+                                                   (__nv_bfloat16*)dst, cols);
+}
+
 void launch_embed(const void* table, bool bf16, const int* tokens, int M, const int* M_dev, int d, float* resid,
                   cudaStream_t st) {
   if (M <= 0) return;

@@ -1,23 +1,40 @@
 // Blackwell tensor-core GEMM:  C[M,N] (op)= A[M,K] * W[N,K]^T,  bf16 operands, fp32 accumulation in TMEM.
 //
-// One CTA computes one 128 x 128 output tile.  Warp 0 streams 128x64 (A) and 128x64 (W) bf16 tiles into a
-// shared-memory ring with TMA (128-byte swizzle; K-major on both sides, which is exactly how activations
-// [tokens, features] and weights [out, in] are stored), warp 1 issues tcgen05.mma (M128 N128 K16, four per
-// stage) into a 128-column TMEM accumulator and releases ring slots with tcgen05.commit, warps 2-5 read the
-// accumulator back with tcgen05.ld and apply the epilogue (store / residual add / bias+tanh).
-// Every mbarrier wait is bounded: on expiry the CTA records an error in the status word, drains what it has
-// in flight, frees its TMEM and returns.
+// Persistent kernel: each CTA walks the 128 x BN output tiles assigned to it (BN = 32 ... 256, chosen so that small
+// problems still spread over the SMs and large ones use the widest tile).  Warp 0 streams 128x64 (A) and BNx64 (W)
+// bf16 tiles into a shared-memory ring with TMA (128-byte swizzle; K-major on both sides, which is exactly how
+// activations [tokens, features] and weights [out, in] are stored).  Warp 1 issues tcgen05.mma (M128 N=BN K16, four per
+// stage) into one of TWO BN-column TMEM accumulators and releases ring slots with tcgen05.commit.  Warps 2-9 (two per
+// TMEM lane quarter) read a finished accumulator back with tcgen05.ld, 32 columns at a time, transpose the 32 x 32
+// block through shared memory so that a warp writes whole row segments, and apply the epilogue -- while the MMA warp
+// is already filling the other accumulator with the next tile.  Besides plain stores the epilogue can finish the
+// surrounding element-wise work of a transformer layer: the RMSNorm row scale of the A operand, SwiGLU, rotary
+// embedding + KV-cache append, residual add + next layer's norm input (see GemmFuse).
+// Every mbarrier wait is bounded: on expiry the CTA raises an abort flag that ends every role's loop, records an error
+// in the status word, drains the copies it has in flight, frees its TMEM and returns.
 #include "tma.cuh"
 
 namespace nz {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4;
-constexpr int kTileBytesA = BM * BK * 2, kTileBytesB = BN * BK * 2;
-constexpr int kStageBytes = kTileBytesA + kTileBytesB;
-constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kThreads = 192;
+constexpr int BM = 128, BK = 64;
+constexpr int kTileBytesA = BM * BK * 2;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kTransposeBytes = kEpiWarps * 32 * 33 * 4;   // per epilogue warp: a 32 x 32 fp32 block, rows padded to 33
+template <int BN> struct Cfg {
+  static constexpr int kTileBytesB = BN * BK * 2;
+  static constexpr int kStageBytes = kTileBytesA + kTileBytesB;
+  static constexpr int kStages = BN >= 128 ? 4 : 6;
+  static constexpr int kSmemBytes =
+      kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTransposeBytes;
+  static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;       // two accumulators; a power of two >= 32
+  // kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128.
+  static constexpr uint32_t kInstrDesc =
+      (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+};
+
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -29,15 +46,13 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
-// kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N = 128, M = 128.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(kInstrDesc), "r"(accumulate) : "memory");
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
@@ -56,23 +71,103 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// The epilogue works in the "lane = column" domain: the 32 lanes of a warp hold 32 consecutive columns of one row, so
+// every global access is one contiguous segment per row.  It is split in two so that the loads of several rows are in
+// flight before the first dependent store:
+//   epi_prefetch  what the row needs from memory (old C for the accumulating epilogues, cos/sin for the rotary one);
+//   epi_apply     x = accumulator (already multiplied by the A operand's RMSNorm row scale where one applies), col =
+//                 this lane's per-column constant (norm gain / bias); returns what kEpiAddNorm sums squares of.
+struct EpiAux { float a, b; };
+
 template <int EPI>
+__device__ __forceinline__ EpiAux epi_prefetch(const GemmArgs& g, int row, int n_chunk, int lane, int pos) {
+  EpiAux r{0.f, 0.f};
+  if (EPI == kEpiAddF32 || EPI == kEpiAddNorm) {
+    r.a = reinterpret_cast<const float*>(g.C)[(long long)row * g.ldc + n_chunk + lane];
+  } else if (EPI == kEpiRopeKV) {
+    const GemmFuse& f = g.f;
+    const int q_cols = f.Hq * f.hd;
+    if (n_chunk < q_cols + f.Hkv * f.hd) {
+      const int in_head = (n_chunk < q_cols ? n_chunk : n_chunk - q_cols) % f.hd;
+      const long long t = (long long)pos * (f.hd >> 1) + ((in_head >> 5) << 4) + (lane & 15);
+      r.a = f.cos_tab[t]; r.b = f.sin_tab[t];
+    }
+  }
+  return r;
+}
+
+template <int EPI>
+__device__ __forceinline__ float epi_apply(const GemmArgs& g, int row, int n_chunk, int lane, float x, float col, EpiAux aux,
+                                          long long kv_dst) {
+  const int n = n_chunk + lane;
+  const long long o = (long long)row * g.ldc + n;
+  if (EPI == kEpiStoreAct) {
+    reinterpret_cast<__nv_bfloat16*>(g.C)[o] = __float2bfloat16_rn(x);
+  } else if (EPI == kEpiStoreF32) {
+    reinterpret_cast<float*>(g.C)[o] = x;
+  } else if (EPI == kEpiAddF32) {
+    reinterpret_cast<float*>(g.C)[o] = aux.a + x;
+  } else if (EPI == kEpiBiasTanhF32) {
+    reinterpret_cast<float*>(g.C)[o] = tanhf(x + col);
+  } else if (EPI == kEpiSwiGLU) {
+    // lanes 0-15 hold gate columns, lanes 16-31 the matching up projections; output feature index n_chunk / 2 + lane
+    const float up = __shfl_down_sync(0xffffffffu, x, 16);
+    if (lane < 16)
+      reinterpret_cast<__nv_bfloat16*>(g.C)[(long long)row * g.ldc + (n_chunk >> 1) + lane] =
+          __float2bfloat16_rn(x / (1.f + __expf(-x)) * up);
+  } else if (EPI == kEpiAddNorm) {
+    const float cn = aux.a + x;
+    reinterpret_cast<float*>(g.C)[o] = cn;
+    reinterpret_cast<__nv_bfloat16*>(g.f.xg)[(long long)row * g.N + n] = __float2bfloat16_rn(cn * col);
+    return cn;
+  } else if (EPI == kEpiRopeKV) {
+    const GemmFuse& f = g.f;
+    const int q_cols = f.Hq * f.hd, k_cols = f.Hkv * f.hd;
+    const int half = f.hd >> 1;
+    const float partner = __shfl_xor_sync(0xffffffffu, x, 16);
+    if (n_chunk < q_cols + k_cols) {
+      // lanes e and 16 + e hold the rotary pair (x_i, x_{i + hd/2}), i = 16 * group + e
+      const int in_head = (n_chunk < q_cols ? n_chunk : n_chunk - q_cols) % f.hd;
+      const int i = ((in_head >> 5) << 4) + (lane & 15);
+      const float y = lane < 16 ? x * aux.a - partner * aux.b : x * aux.a + partner * aux.b;
+      const int d = lane < 16 ? i : half + i;
+      if (n_chunk < q_cols) {
+        reinterpret_cast<__nv_bfloat16*>(g.C)[(long long)row * g.ldc + (n_chunk - in_head) + d] = __float2bfloat16_rn(y);
+      } else if (kv_dst >= 0) {
+        reinterpret_cast<__nv_bfloat16*>(f.k_cache)[kv_dst + (long long)((n_chunk - q_cols) / f.hd) * f.kv_head_stride + d] =
+            __float2bfloat16_rn(y);
+      }
+    } else if (kv_dst >= 0) {
+      const int nv = n - q_cols - k_cols;
+      reinterpret_cast<__nv_bfloat16*>(f.v_cache)[kv_dst + (long long)(nv / f.hd) * f.kv_head_stride + nv % f.hd] =
+          __float2bfloat16_rn(x);
+    }
+  }
+  return 0.f;
+}
+
+template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
                                                            const __grid_constant__ CUtensorMap tmB, GemmArgs a,
                                                            int* status) {
+  using C = Cfg<BN>;
+  constexpr int STAGES = C::kStages;
   const int M = a.M_dev ? min(a.M, *a.M_dev) : a.M;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  if (m0 >= M) return;
+  const int tiles_m = (M + BM - 1) / BM, tiles_n = (a.N + BN - 1) / BN;
+  const int n_tiles = tiles_m * tiles_n;
+  if ((int)blockIdx.x >= n_tiles) return;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = base + STAGES * kStageBytes;
-  // barriers: full[STAGES], empty[STAGES], accum; then tmem slot and abort flag
+  const uint32_t bar_base = base + STAGES * C::kStageBytes;
+  // barriers: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]; then the TMEM slot and the abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  const uint32_t accum_bar = bar_base + 8u * (2 * STAGES);
+  auto acc_full = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto acc_empty = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * kStageBytes + 8 * (2 * STAGES + 1));
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * C::kStageBytes + 8 * (2 * STAGES + 4));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -80,138 +175,235 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(accum_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kEpiWarps); }
     *abort_flag = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(BN));
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(C::kTmemCols));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_acc = *tmem_slot;
+  const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int issued = 0;
-      for (int k = 0; k < k_iters; ++k) {
-        const int s = k % STAGES;
-        if (k >= STAGES && !mbar_wait(empty_bar(s), ((k / STAGES) - 1) & 1)) { *abort_flag = 1; break; }
-        if (*abort_flag) break;
-        mbar_expect_tx(full_bar(s), kStageBytes);
-        tma_load_2d(base + s * kStageBytes, &tmA, k * BK, m0, full_bar(s));
-        tma_load_2d(base + s * kStageBytes + kTileBytesA, &tmB, k * BK, n0, full_bar(s));
-        issued = k + 1;
+      int it = 0;                                // k-iterations issued so far, over all tiles
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        for (int k = 0; k < k_iters; ++k, ++it) {
+          const int s = it % STAGES;
+          if (it >= STAGES && !mbar_wait_or_abort(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), C::kStageBytes);
+          tma_load_2d(base + s * C::kStageBytes, &tmA, k * BK, m0, full_bar(s));
+          tma_load_2d(base + s * C::kStageBytes + kTileBytesA, &tmB, k * BK, n0, full_bar(s));
+        }
       }
-      if (*abort_flag) {                       // drain: wait (bounded) for the copies still in flight
-        for (int k = max(0, issued - STAGES); k < issued; ++k) mbar_wait(full_bar(k % STAGES), (k / STAGES) & 1);
+      if (!ok) {                                 // drain: wait (bounded) for the copies still in flight
+        *abort_flag = 1;
+        for (int j = max(0, it - STAGES); j < it; ++j) mbar_wait(full_bar(j % STAGES), (j / STAGES) & 1);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      int it = 0, t_local = 0;
       bool ok = true;
-      for (int k = 0; k < k_iters && ok; ++k) {
-        const int s = k % STAGES;
-        if (!mbar_wait(full_bar(s), (k / STAGES) & 1) || *abort_flag) { *abort_flag = 1; ok = false; break; }
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
+        const int b = t_local & 1;
+        if (t_local >= 2 && !mbar_wait_or_abort(acc_empty(b), ((t_local >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = base + s * kStageBytes, sb = sa + kTileBytesA;
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(b * BN);
+        for (int k = 0; k < k_iters; ++k, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait_or_abort(full_bar(s), (it / STAGES) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + s * C::kStageBytes, sb = sa + kTileBytesA;
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk)
-          tc_mma(tmem_acc, smem_desc(sa + kk * 32), smem_desc(sb + kk * 32), (k > 0 || kk > 0) ? 1u : 0u);
-        tc_commit(empty_bar(s));               // slot free once these MMAs have read it
+          for (int kk = 0; kk < BK / 16; ++kk)
+            tc_mma(tmem_acc, smem_desc(sa + kk * 32), smem_desc(sb + kk * 32), C::kInstrDesc, (k > 0 || kk > 0) ? 1u : 0u);
+          tc_commit(empty_bar(s));               // slot free once these MMAs have read it
+        }
+        if (ok) tc_commit(acc_full(b));          // accumulator complete
       }
-      tc_commit(accum_bar);                    // accumulator complete (also arrives after an abort)
+      if (!ok) *abort_flag = 1;
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
-    const int q = warp & 3;                    // TMEM lane quarter this warp may access
-    const bool ok = __all_sync(0xffffffffu, mbar_wait(accum_bar, 0) && !*abort_flag);   // warp-uniform
-    tc_fence_after();
-    if (ok) {
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    const int q = warp & 3;                      // TMEM lane quarter this warp may access
+    const int half = (warp - 2) >> 2;            // which half of the tile's 32-column groups this warp takes
+    float* stg = reinterpret_cast<float*>(gen_base + STAGES * C::kStageBytes + 256) + (warp - 2) * (32 * 33);
+    int t_local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
+      const int tn = tile / tiles_m;
+      const int m0 = (tile % tiles_m) * BM, n0 = tn * BN;
+      const int b = t_local & 1;
       const int row = m0 + q * 32 + lane;
+      float rs = 1.f;                            // RMSNorm scale of the A operand's row (overlaps the main loop)
+      if (a.f.ss_in && row < M) {
+        float ss = 0.f;
+        for (int p = 0; p < a.f.ss_in_parts; ++p) ss += a.f.ss_in[(long long)p * a.f.ss_ld + row];
+        rs = rsqrtf(ss * a.f.inv_dim + a.f.eps);
+      }
+      int pos = 0; long long kvd = -1;
+      if (EPI == kEpiRopeKV && row < M) { pos = a.f.tok_pos[row]; kvd = a.f.kv_dst[row]; }
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(acc_full(b), (t_local >> 1) & 1, abort_flag));   // warp-uniform
+      if (!ok) break;
+      tc_fence_after();
+      const int rows_here = min(32, M - (m0 + q * 32));          // rows of this quarter that exist (may be <= 0)
+      float ssq = 0.f;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = half; c < BN / 32; c += 2) {
+        const int n_chunk = n0 + c * 32;
+        if (n_chunk >= a.N) break;                               // ragged last tile (N is a multiple of 32)
         float v[32];
-        tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
-        if (row < M) {
-          const int n = n0 + c * 32;
-          const long long o = (long long)row * a.ldc + n;
-          if (EPI == kEpiStoreAct) {
-            __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(a.C) + o);
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * 32), v);
+        // transpose through shared memory: from lane = row (how TMEM hands the block out) to lane = column
 #pragma unroll
-            for (int i = 0; i < 16; ++i) dst[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-          } else if (EPI == kEpiStoreF32) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + o);
+        for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j] * rs;
+        __syncwarp();
+        float col = 0.f;
+        if (EPI == kEpiAddNorm) col = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.f.gain)[n_chunk + lane]);
+        if (EPI == kEpiBiasTanhF32) col = a.bias[n_chunk + lane];
+        for (int rr0 = 0; rr0 < rows_here; rr0 += 8) {
+          EpiAux aux[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          } else if (EPI == kEpiAddF32) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + o);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float4 c4 = dst[i];
-              c4.x += v[4 * i]; c4.y += v[4 * i + 1]; c4.z += v[4 * i + 2]; c4.w += v[4 * i + 3];
-              dst[i] = c4;
+          for (int u = 0; u < 8; ++u) {
+            const int rr = rr0 + u;
+            if (rr < rows_here) {
+              const int p_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, pos, rr) : 0;
+              aux[u] = epi_prefetch<EPI>(a, m0 + q * 32 + rr, n_chunk, lane, p_r);
             }
-          } else if (EPI == kEpiBiasTanhF32) {
-            float* dst = reinterpret_cast<float*>(a.C) + o;
+          }
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[i] = tanhf(v[i] + a.bias[n + i]);
+          for (int u = 0; u < 8; ++u) {
+            const int rr = rr0 + u;
+            if (rr < rows_here) {
+              const long long kv_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, kvd, rr) : -1;
+              const float back = epi_apply<EPI>(a, m0 + q * 32 + rr, n_chunk, lane, stg[rr * 33 + lane], col, aux[u], kv_r);
+              if (EPI == kEpiAddNorm) stg[rr * 33 + lane] = back;
+            }
           }
         }
+        __syncwarp();
+        if (EPI == kEpiAddNorm && lane < rows_here) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) { const float t = stg[lane * 33 + j]; ssq += t * t; }
+        }
+        __syncwarp();
+      }
+      // this warp is done reading the accumulator: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(b));
+      if (EPI == kEpiAddNorm && row < M) {
+        // the two warps of a quarter each saw half of the tile's columns: two partial sums per tile
+        a.f.ss_out[(long long)(tn * 2 + half) * a.f.ss_ld + row] = ssq;
       }
     }
+    if (!ok && lane == 0) *abort_flag = 1;
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(BN));
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols));
   }
   if (threadIdx.x == 0 && *abort_flag) atomicOr(status, kStInternal);
 }
 
 // ---------------------------------------------------------------------------------------------------
-// host side: tensor maps
+// host side
 // ---------------------------------------------------------------------------------------------------
-template <int EPI>
-void launch(const CUtensorMap* ta, const CUtensorMap* tb, const GemmArgs& a, cudaStream_t st) {
+int sm_count() {
+  static int n = [] {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+      v = 148;
+    return v;
+  }();
+  return n;
+}
+
+template <int BN, int EPI>
+void launch(const GemmArgs& a, cudaStream_t st) {
+  const CUtensorMap* ta = tma_map_bf16(a.A, a.M, a.K, a.lda, BM);
+  const CUtensorMap* tb = tma_map_bf16(a.W, a.N, a.K, a.ldw, BN);
+  if (!ta || !tb) {                            // cannot happen for shapes gemm_tc_supported accepted; report, do not guess
+    static const int flag = kStInternal;
+    cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st);
+    return;
+  }
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
     configured = true;
   }
-  dim3 grid(a.N / BN, (a.M + BM - 1) / BM);
-  gemm_tc_kernel<EPI><<<grid, kThreads, kSmemBytes, st>>>(*ta, *tb, a, a.status);
+  const long long tiles = (long long)((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
+  const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  gemm_tc_kernel<BN, EPI><<<grid, kThreads, Cfg<BN>::kSmemBytes, st>>>(*ta, *tb, a, a.status);
+}
+
+template <int BN>
+void launch_bn(const GemmArgs& a, cudaStream_t st) {
+  switch (a.epilogue) {
+    case kEpiStoreAct: launch<BN, kEpiStoreAct>(a, st); break;
+    case kEpiStoreF32: launch<BN, kEpiStoreF32>(a, st); break;
+    case kEpiAddF32: launch<BN, kEpiAddF32>(a, st); break;
+    case kEpiBiasTanhF32: launch<BN, kEpiBiasTanhF32>(a, st); break;
+    case kEpiSwiGLU: launch<BN, kEpiSwiGLU>(a, st); break;
+    case kEpiAddNorm: launch<BN, kEpiAddNorm>(a, st); break;
+    case kEpiRopeKV: launch<BN, kEpiRopeKV>(a, st); break;
+    default: break;
+  }
 }
 
 }  // namespace
 
+// Output-tile width.  Cost model: waves of tiles over the SMs times the time of one k-step of a tile, which is the
+// larger of the tensor-pipe time (2 BN clocks for four M128 N=BN K16 instructions) and the shared-memory feed time
+// ((16 KB + BN * 128 B) at 128 B per clock); a 128-wide tile sits exactly on that feed limit, hence its surcharge.
+int gemm_tc_tile_n(int M, int N) {
+  const long long tiles_m = (M + BM - 1) / BM;
+  static const int widths[4] = {256, 128, 64, 32}, step_cost[4] = {512, 288, 192, 160};
+  long long best = -1; int best_bn = 32;
+  for (int i = 0; i < 4; ++i) {
+    const int bn = widths[i];
+    if (bn > 32 && N < bn) continue;
+    const long long tiles = tiles_m * ((N + bn - 1) / bn);
+    const long long cost = ((tiles + sm_count() - 1) / sm_count()) * step_cost[i];
+    if (best < 0 || cost < best) { best = cost; best_bn = bn; }
+  }
+  return best_bn;
+}
+
+// Partial sums of squares a kEpiAddNorm launch writes per row (two per column tile).
+int gemm_tc_norm_parts(int M, int N) {
+  const int bn = gemm_tc_tile_n(M, N);
+  return 2 * ((N + bn - 1) / bn);
+}
+
 bool gemm_tc_supported(const GemmArgs& a) {
   if (!a.status || !tma_encode_fn()) return false;
-  if (a.K % BK || a.N % BN || a.M <= 0) return false;
+  if (a.K % BK || a.N % 32 || a.M <= 0) return false;
   if ((a.lda * 2) % 16 || (a.ldw * 2) % 16 || ((uintptr_t)a.A & 15) || ((uintptr_t)a.W & 15)) return false;
-  if (a.epilogue == kEpiStoreAct && (((uintptr_t)a.C & 3) || (a.ldc & 1))) return false;
-  if ((a.epilogue == kEpiStoreF32 || a.epilogue == kEpiAddF32) && (((uintptr_t)a.C & 15) || (a.ldc & 3))) return false;
-  return a.epilogue == kEpiStoreAct || a.epilogue == kEpiStoreF32 || a.epilogue == kEpiAddF32 ||
-         a.epilogue == kEpiBiasTanhF32;
+  return a.epilogue >= kEpiStoreAct && a.epilogue <= kEpiRopeKV;
 }
 
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
-  const CUtensorMap* ta = tma_map_bf16(a.A, a.M, a.K, a.lda, BM);
-  const CUtensorMap* tb = tma_map_bf16(a.W, a.N, a.K, a.ldw, BN);
-  if (!ta || !tb) { launch_gemm_simt(a, true, st); return; }
   LaunchScope ls(kcGemm, st);
-  switch (a.epilogue) {
-    case kEpiStoreAct: launch<kEpiStoreAct>(ta, tb, a, st); break;
-    case kEpiStoreF32: launch<kEpiStoreF32>(ta, tb, a, st); break;
-    case kEpiAddF32: launch<kEpiAddF32>(ta, tb, a, st); break;
-    case kEpiBiasTanhF32: launch<kEpiBiasTanhF32>(ta, tb, a, st); break;
-    default: break;
+  switch (gemm_tc_tile_n(a.M, a.N)) {
+    case 256: launch_bn<256>(a, st); break;
+    case 128: launch_bn<128>(a, st); break;
+    case 64: launch_bn<64>(a, st); break;
+    default: launch_bn<32>(a, st); break;
   }
 }
 
