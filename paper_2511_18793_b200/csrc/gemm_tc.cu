@@ -22,7 +22,7 @@ constexpr int BM = 128, BK = 64;
 constexpr int kTileBytesA = BM * BK * 2;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
-constexpr int kTransposeBytes = kEpiWarps * 32 * 33 * 4;   // per epilogue warp: a 32 x 32 fp32 block, rows padded to 33
+constexpr int kTransposeBytes = kEpiWarps * 32 * 32 * 4;   // per epilogue warp: a 32 x 32 fp32 block, chunks swizzled
 template <int BN> struct Cfg {
   static constexpr int kTileBytesB = BN * BK * 2;
   static constexpr int kStageBytes = kTileBytesA + kTileBytesB;
@@ -71,79 +71,130 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// The epilogue works in the "lane = column" domain: the 32 lanes of a warp hold 32 consecutive columns of one row, so
-// every global access is one contiguous segment per row.  It is split in two so that the loads of several rows are in
-// flight before the first dependent store:
-//   epi_prefetch  what the row needs from memory (old C for the accumulating epilogues, cos/sin for the rotary one);
-//   epi_apply     x = accumulator (already multiplied by the A operand's RMSNorm row scale where one applies), col =
-//                 this lane's per-column constant (norm gain / bias); returns what kEpiAddNorm sums squares of.
-struct EpiAux { float a, b; };
+// The epilogue works on 32 x 32 blocks of the accumulator.  tcgen05.ld hands a block out with lane = row; it is
+// transposed through shared memory (128-byte rows, 16-byte chunks XOR-swizzled by the row, so both sides are free of
+// bank conflicts) into "8 lanes per row, 4 consecutive columns per lane", in which every global access of a warp is
+// four contiguous row segments.  The work on a row is split in two so that the loads of several rows are in flight
+// before the first dependent store:
+//   epi_prefetch  what the lane needs from memory (old C for the accumulating epilogues, cos / sin for the rotary one);
+//   epi_apply     x = 4 accumulators (already multiplied by the A operand's RMSNorm row scale where one applies);
+//                 returns what kEpiAddNorm sums squares of.
+struct EpiAux { float4 a, b; };
+
+// What a lane needs to know about its 4 columns of the current 32-column group; computed once per group so that the
+// per-row code has no divisions left.  k = lane & 7 selects columns [4k, 4k + 4) of the group.
+struct ChunkCtx {
+  float4 col;        // norm gains (kEpiAddNorm) or biases (kEpiBiasTanhF32) of the lane's columns
+  int kind;          // kEpiRopeKV: 0 = q (rotate, to C), 1 = k (rotate, to the K cache), 2 = v (copy to the V cache)
+  int tab;           // kEpiRopeKV: first of the lane's 4 rotary-pair indices inside the head (cos / sin table column)
+  long long off;     // element offset of the lane's first output inside the row (C) or inside the token's cache entry
+};
+
+__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+}
 
 template <int EPI>
-__device__ __forceinline__ EpiAux epi_prefetch(const GemmArgs& g, int row, int n_chunk, int lane, int pos) {
-  EpiAux r{0.f, 0.f};
-  if (EPI == kEpiAddF32 || EPI == kEpiAddNorm) {
-    r.a = reinterpret_cast<const float*>(g.C)[(long long)row * g.ldc + n_chunk + lane];
-  } else if (EPI == kEpiRopeKV) {
+__device__ __forceinline__ ChunkCtx chunk_ctx(const GemmArgs& g, int n_chunk, int k) {
+  ChunkCtx cc{make_float4(0.f, 0.f, 0.f, 0.f), 0, 0, 0};
+  const int n = n_chunk + 4 * k;
+  if (EPI == kEpiAddNorm) {
+    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(reinterpret_cast<const __nv_bfloat16*>(g.f.gain) + n);
+    const float2 g0 = __bfloat1622float2(gp[0]), g1 = __bfloat1622float2(gp[1]);
+    cc.col = make_float4(g0.x, g0.y, g1.x, g1.y);
+  }
+  if (EPI == kEpiBiasTanhF32) cc.col = *reinterpret_cast<const float4*>(g.bias + n);
+  if (EPI == kEpiSwiGLU) cc.off = (n_chunk >> 1) + 4 * k;      // lanes k < 4: gate columns -> output features n_chunk / 2 + 4k ..
+  if (EPI == kEpiRopeKV) {
     const GemmFuse& f = g.f;
-    const int q_cols = f.Hq * f.hd;
-    if (n_chunk < q_cols + f.Hkv * f.hd) {
-      const int in_head = (n_chunk < q_cols ? n_chunk : n_chunk - q_cols) % f.hd;
-      const long long t = (long long)pos * (f.hd >> 1) + ((in_head >> 5) << 4) + (lane & 15);
-      r.a = f.cos_tab[t]; r.b = f.sin_tab[t];
+    const int q_cols = f.Hq * f.hd, k_cols = f.Hkv * f.hd, half = f.hd >> 1;
+    if (n_chunk < q_cols + k_cols) {
+      // columns e and 16 + e of the group hold the rotary pair (x_i, x_{i + hd/2}), i = 16 * (group inside the head) + e;
+      // lanes k < 4 hold e = 4k .. 4k + 3, lanes k + 4 their partners
+      const int nn = n_chunk < q_cols ? n_chunk : n_chunk - q_cols;
+      const int head = nn / f.hd, in_head = nn - head * f.hd;
+      cc.tab = ((in_head >> 5) << 4) + 4 * (k & 3);
+      const int d = k < 4 ? cc.tab : half + cc.tab;
+      cc.kind = n_chunk < q_cols ? 0 : 1;
+      cc.off = n_chunk < q_cols ? (long long)(n_chunk - in_head) + d : (long long)head * f.kv_head_stride + d;
+    } else {
+      const int nv = n - q_cols - k_cols;
+      const int head = nv / f.hd;
+      cc.kind = 2;
+      cc.off = (long long)head * f.kv_head_stride + (nv - head * f.hd);
+    }
+  }
+  return cc;
+}
+
+template <int EPI>
+__device__ __forceinline__ EpiAux epi_prefetch(const GemmArgs& g, const ChunkCtx& cc, int row, int n, int pos) {
+  EpiAux r;
+  r.a = r.b = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (EPI == kEpiAddF32 || EPI == kEpiAddNorm) {
+    r.a = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C) + (long long)row * g.ldc + n);
+  } else if (EPI == kEpiRopeKV) {
+    if (cc.kind < 2) {
+      const long long t = (long long)pos * (g.f.hd >> 1) + cc.tab;
+      r.a = *reinterpret_cast<const float4*>(g.f.cos_tab + t);
+      r.b = *reinterpret_cast<const float4*>(g.f.sin_tab + t);
     }
   }
   return r;
 }
 
+// `valid`: the row exists (shuffles are executed by every lane regardless).
 template <int EPI>
-__device__ __forceinline__ float epi_apply(const GemmArgs& g, int row, int n_chunk, int lane, float x, float col, EpiAux aux,
-                                          long long kv_dst) {
-  const int n = n_chunk + lane;
+__device__ __forceinline__ float4 epi_apply(const GemmArgs& g, const ChunkCtx& cc, bool valid, int row, int n, int k, float4 x,
+                                           const EpiAux& aux, long long kv_dst) {
   const long long o = (long long)row * g.ldc + n;
   if (EPI == kEpiStoreAct) {
-    reinterpret_cast<__nv_bfloat16*>(g.C)[o] = __float2bfloat16_rn(x);
+    if (valid) *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.C) + o) = pack_bf16x4(x.x, x.y, x.z, x.w);
   } else if (EPI == kEpiStoreF32) {
-    reinterpret_cast<float*>(g.C)[o] = x;
+    if (valid) *reinterpret_cast<float4*>(reinterpret_cast<float*>(g.C) + o) = x;
   } else if (EPI == kEpiAddF32) {
-    reinterpret_cast<float*>(g.C)[o] = aux.a + x;
+    if (valid)
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(g.C) + o) =
+          make_float4(aux.a.x + x.x, aux.a.y + x.y, aux.a.z + x.z, aux.a.w + x.w);
   } else if (EPI == kEpiBiasTanhF32) {
-    reinterpret_cast<float*>(g.C)[o] = tanhf(x + col);
+    if (valid)
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(g.C) + o) =
+          make_float4(tanhf(x.x + cc.col.x), tanhf(x.y + cc.col.y), tanhf(x.z + cc.col.z), tanhf(x.w + cc.col.w));
   } else if (EPI == kEpiSwiGLU) {
-    // lanes 0-15 hold gate columns, lanes 16-31 the matching up projections; output feature index n_chunk / 2 + lane
-    const float up = __shfl_down_sync(0xffffffffu, x, 16);
-    if (lane < 16)
-      reinterpret_cast<__nv_bfloat16*>(g.C)[(long long)row * g.ldc + (n_chunk >> 1) + lane] =
-          __float2bfloat16_rn(x / (1.f + __expf(-x)) * up);
+    // lanes k < 4 hold gate columns, lanes k + 4 the matching up projections
+    const float u0 = __shfl_xor_sync(0xffffffffu, x.x, 4), u1 = __shfl_xor_sync(0xffffffffu, x.y, 4);
+    const float u2 = __shfl_xor_sync(0xffffffffu, x.z, 4), u3 = __shfl_xor_sync(0xffffffffu, x.w, 4);
+    if (valid && k < 4)
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.C) + (long long)row * g.ldc + cc.off) =
+          pack_bf16x4(__fdividef(x.x, 1.f + __expf(-x.x)) * u0, __fdividef(x.y, 1.f + __expf(-x.y)) * u1,
+                      __fdividef(x.z, 1.f + __expf(-x.z)) * u2, __fdividef(x.w, 1.f + __expf(-x.w)) * u3);
   } else if (EPI == kEpiAddNorm) {
-    const float cn = aux.a + x;
-    reinterpret_cast<float*>(g.C)[o] = cn;
-    reinterpret_cast<__nv_bfloat16*>(g.f.xg)[(long long)row * g.N + n] = __float2bfloat16_rn(cn * col);
+    const float4 cn = make_float4(aux.a.x + x.x, aux.a.y + x.y, aux.a.z + x.z, aux.a.w + x.w);
+    if (valid) {
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(g.C) + o) = cn;
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.f.xg) + (long long)row * g.N + n) =
+          pack_bf16x4(cn.x * cc.col.x, cn.y * cc.col.y, cn.z * cc.col.z, cn.w * cc.col.w);
+    }
     return cn;
   } else if (EPI == kEpiRopeKV) {
-    const GemmFuse& f = g.f;
-    const int q_cols = f.Hq * f.hd, k_cols = f.Hkv * f.hd;
-    const int half = f.hd >> 1;
-    const float partner = __shfl_xor_sync(0xffffffffu, x, 16);
-    if (n_chunk < q_cols + k_cols) {
-      // lanes e and 16 + e hold the rotary pair (x_i, x_{i + hd/2}), i = 16 * group + e
-      const int in_head = (n_chunk < q_cols ? n_chunk : n_chunk - q_cols) % f.hd;
-      const int i = ((in_head >> 5) << 4) + (lane & 15);
-      const float y = lane < 16 ? x * aux.a - partner * aux.b : x * aux.a + partner * aux.b;
-      const int d = lane < 16 ? i : half + i;
-      if (n_chunk < q_cols) {
-        reinterpret_cast<__nv_bfloat16*>(g.C)[(long long)row * g.ldc + (n_chunk - in_head) + d] = __float2bfloat16_rn(y);
-      } else if (kv_dst >= 0) {
-        reinterpret_cast<__nv_bfloat16*>(f.k_cache)[kv_dst + (long long)((n_chunk - q_cols) / f.hd) * f.kv_head_stride + d] =
-            __float2bfloat16_rn(y);
-      }
-    } else if (kv_dst >= 0) {
-      const int nv = n - q_cols - k_cols;
-      reinterpret_cast<__nv_bfloat16*>(f.v_cache)[kv_dst + (long long)(nv / f.hd) * f.kv_head_stride + nv % f.hd] =
-          __float2bfloat16_rn(x);
+    const float p0 = __shfl_xor_sync(0xffffffffu, x.x, 4), p1 = __shfl_xor_sync(0xffffffffu, x.y, 4);
+    const float p2 = __shfl_xor_sync(0xffffffffu, x.z, 4), p3 = __shfl_xor_sync(0xffffffffu, x.w, 4);
+    float4 y = x;
+    if (cc.kind < 2) {
+      const float sg = k < 4 ? -1.f : 1.f;             // x_i' = x_i c - x_j s ;  x_j' = x_j c + x_i s
+      y = make_float4(x.x * aux.a.x + sg * p0 * aux.b.x, x.y * aux.a.y + sg * p1 * aux.b.y,
+                      x.z * aux.a.z + sg * p2 * aux.b.z, x.w * aux.a.w + sg * p3 * aux.b.w);
+    }
+    const uint2 packed = pack_bf16x4(y.x, y.y, y.z, y.w);
+    if (cc.kind == 0) {
+      if (valid) *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.C) + (long long)row * g.ldc + cc.off) = packed;
+    } else if (valid && kv_dst >= 0) {
+      __nv_bfloat16* cache = reinterpret_cast<__nv_bfloat16*>(cc.kind == 1 ? g.f.k_cache : g.f.v_cache);
+      *reinterpret_cast<uint2*>(cache + kv_dst + cc.off) = packed;
     }
   }
-  return 0.f;
+  return x;
 }
 
 template <int BN, int EPI>
@@ -237,7 +288,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
     // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;                      // TMEM lane quarter this warp may access
     const int half = (warp - 2) >> 2;            // which half of the tile's 32-column groups this warp takes
-    float* stg = reinterpret_cast<float*>(gen_base + STAGES * C::kStageBytes + 256) + (warp - 2) * (32 * 33);
+    float4* stg4 = reinterpret_cast<float4*>(gen_base + STAGES * C::kStageBytes + 256) + (warp - 2) * (32 * 8);
     int t_local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
@@ -264,37 +315,40 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
         if (n_chunk >= a.N) break;                               // ragged last tile (N is a multiple of 32)
         float v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * 32), v);
-        // transpose through shared memory: from lane = row (how TMEM hands the block out) to lane = column
+        // transpose through shared memory: from lane = row (how TMEM hands the block out) to 8 lanes per row
 #pragma unroll
-        for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j] * rs;
+        for (int j = 0; j < 8; ++j)
+          stg4[lane * 8 + (j ^ (lane & 7))] = make_float4(v[4 * j] * rs, v[4 * j + 1] * rs, v[4 * j + 2] * rs, v[4 * j + 3] * rs);
         __syncwarp();
-        float col = 0.f;
-        if (EPI == kEpiAddNorm) col = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.f.gain)[n_chunk + lane]);
-        if (EPI == kEpiBiasTanhF32) col = a.bias[n_chunk + lane];
-        for (int rr0 = 0; rr0 < rows_here; rr0 += 8) {
-          EpiAux aux[8];
+        const int k = lane & 7, rsub = lane >> 3;
+        const ChunkCtx cc = chunk_ctx<EPI>(a, n_chunk, k);
+        const int n = n_chunk + 4 * k;
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int rr = rr0 + u;
-            if (rr < rows_here) {
-              const int p_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, pos, rr) : 0;
-              aux[u] = epi_prefetch<EPI>(a, m0 + q * 32 + rr, n_chunk, lane, p_r);
-            }
+        for (int it0 = 0; it0 < 8; it0 += 4) {
+          if (it0 * 4 >= rows_here) break;                           // warp-uniform
+          EpiAux aux[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int r = (it0 + u) * 4 + rsub;
+            const int p_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, pos, r) : 0;
+            if (r < rows_here) aux[u] = epi_prefetch<EPI>(a, cc, m0 + q * 32 + r, n, p_r);
           }
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int rr = rr0 + u;
-            if (rr < rows_here) {
-              const long long kv_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, kvd, rr) : -1;
-              const float back = epi_apply<EPI>(a, m0 + q * 32 + rr, n_chunk, lane, stg[rr * 33 + lane], col, aux[u], kv_r);
-              if (EPI == kEpiAddNorm) stg[rr * 33 + lane] = back;
-            }
+          for (int u = 0; u < 4; ++u) {
+            const int r = (it0 + u) * 4 + rsub;
+            const long long kv_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, kvd, r) : -1;
+            const float4 x = stg4[r * 8 + (k ^ (r & 7))];
+            const float4 back = epi_apply<EPI>(a, cc, r < rows_here, m0 + q * 32 + r, n, k, x, aux[u], kv_r);
+            if (EPI == kEpiAddNorm) stg4[r * 8 + (k ^ (r & 7))] = back;
           }
         }
         __syncwarp();
         if (EPI == kEpiAddNorm && lane < rows_here) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) { const float t = stg[lane * 33 + j]; ssq += t * t; }
+          for (int j = 0; j < 8; ++j) {
+            const float4 t = stg4[lane * 8 + (j ^ (lane & 7))];
+            ssq += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+          }
         }
         __syncwarp();
       }
@@ -394,6 +448,8 @@ bool gemm_tc_supported(const GemmArgs& a) {
   if (!a.status || !tma_encode_fn()) return false;
   if (a.K % BK || a.N % 32 || a.M <= 0) return false;
   if ((a.lda * 2) % 16 || (a.ldw * 2) % 16 || ((uintptr_t)a.A & 15) || ((uintptr_t)a.W & 15)) return false;
+  if (((uintptr_t)a.C & 15) || (a.ldc & 3)) return false;          // the epilogue stores 8- and 16-byte vectors
+  if (a.epilogue == kEpiBiasTanhF32 && ((uintptr_t)a.bias & 15)) return false;
   return a.epilogue >= kEpiStoreAct && a.epilogue <= kEpiRopeKV;
 }
 
