@@ -25,6 +25,9 @@ sys.path.insert(0, ROOT)
 sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 METRIC, UNIT = "items_per_s_decoded", "items/s"
+# bumped whenever a kernel of the class changes in a way that can change its DRAM traffic: a traffic figure taken
+# from an older revision is reported as null
+KERNEL_REV = {"gemm": 3, "attention": 1}
 
 
 def load_peaks():
@@ -109,7 +112,11 @@ def oracle_sample(w, weights_np, catalog, hist, mode, budget_s=20.0, max_rows=No
 
 
 def algorithmic_work(w, stats_tokens_per_step, rounds):
-    """Algorithmic flops / bytes of one decode step, per kernel class (the per-unit figures are in the design doc)."""
+    """Algorithmic flops / bytes of one decode step, per kernel class.
+
+    GEMM: 2 flops per (token, weight) pair of every projection and of the LM head rows of levels 2..L.
+    Attention: the context K and V of every request once per (layer, pass) plus q and o of every token once
+    (bytes); 4 * head_dim flops per (token, query head, visible position)."""
     esz = 4 if w.dtype == "fp32" else 2
     d, hd, Hq, Hkv, F, nl = w.d_model, w.head_dim, w.n_q_heads, w.n_kv_heads, w.d_ffn, w.n_layers
     per_tok_params = nl * ((Hq + 2 * Hkv) * hd * d + d * Hq * hd + 3 * F * d)
@@ -302,6 +309,14 @@ def main():
         roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
     else:
         roof.update(bound="latency", note="dominant class is neither GEMM nor attention")
+    # DRAM traffic of the dominant kernel from the committed ncu capture of that kernel (bytes per launch, scaled by
+    # the units processed where the capture ran a smaller case); null when no capture matches the current kernel
+    tpath = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(tpath):
+        rec = json.load(open(tpath)).get(f"{dom}@{w.name}")
+        if rec and rec.get("kernel_rev") == KERNEL_REV.get(dom):
+            roof["traffic"] = rec["dram_bytes_per_launch"]
+            roof["traffic_note"] = rec.get("note")
     roof["classes"] = shares
     roof["attention_gbs"] = work["attention_bytes"] / (shares["attention"]["ms_per_step"] / 1e3) / 1e9 if "attention" in shares else None
     roof["gemm_tflops"] = work["gemm_flops"] / (shares["gemm"]["ms_per_step"] / 1e3) / 1e12 if "gemm" in shares else None

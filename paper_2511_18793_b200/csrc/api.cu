@@ -221,6 +221,7 @@ size_t carve(nezha_ctx* c) {
   e.tok_ext = cv.take<long long>((size_t)c->Mv_max * c->L);
   e.row_tok_count = cv.take<int>(c->Bmax); e.n_tokens = cv.take<int>(1);
   e.row_tok_start = cv.take<int>(c->Bmax); e.pf_row_start = cv.take<int>(c->Bmax); e.pf_row_count = cv.take<int>(c->Bmax);
+  e.req_info = cv.take<int4>(c->Bmax); e.pf_req_info = cv.take<int4>(c->Bmax);
   e.h_f32 = c->h_f32;
   return (cv.off + 255) & ~(size_t)255;
 }
@@ -272,6 +273,7 @@ void run_layers_fused(nezha_ctx* c, long long M, const int* M_dev, bool verify, 
     t.tok_row = e.tok_row; t.tok_ctx_len = e.tok_ctx_len; t.tok_ext = e.tok_ext; t.n_ext_max = verify ? c->L : 0;
     t.M = (int)M; t.M_dev = M_dev; t.Hq = c->Hq; t.Hkv = c->Hkv; t.hd = c->hd; t.scale = 1.f / sqrtf((float)c->hd);
     t.row_start = verify ? e.row_tok_start : e.pf_row_start; t.row_count = verify ? e.row_tok_count : e.pf_row_count;
+    t.req_info = verify ? e.req_info : e.pf_req_info;
     t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
     t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
     if (attention_tc_supported(t)) launch_attention_tc(t, c->st);
@@ -318,6 +320,7 @@ void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify, int n_
     t.tok_row = e.tok_row; t.tok_ctx_len = e.tok_ctx_len; t.tok_ext = e.tok_ext; t.n_ext_max = verify ? c->L : 0;
     t.M = (int)M; t.M_dev = M_dev; t.Hq = c->Hq; t.Hkv = c->Hkv; t.hd = c->hd; t.scale = 1.f / sqrtf((float)c->hd);
     t.row_start = verify ? e.row_tok_start : e.pf_row_start; t.row_count = verify ? e.row_tok_count : e.pf_row_count;
+    t.req_info = verify ? e.req_info : e.pf_req_info;
     t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
     t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
     if (c->bf16 && attention_tc_supported(t)) launch_attention_tc(t, c->st);

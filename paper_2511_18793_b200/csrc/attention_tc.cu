@@ -47,8 +47,80 @@ __device__ __forceinline__ uint32_t kv_addr(uint32_t tile, int pos, int chunk) {
   return tile + sub * (kPos * 128) + pos * 128 + ((c ^ (pos & 7)) << 4);
 }
 
+// The token's own extra KV rows (drafted codes of its tuple), straight from global memory, folded into the running
+// softmax state of the thread's two rows.  The loads of all (row, entry) pairs are issued together -- offsets, then
+// every K row, then every V row -- so the chain of dependent memory round trips is three long whatever the number
+// of entries.  E = compile-time bound of the entries per token (n_ext_max <= E).
+template <int HD, int E>
+__device__ __forceinline__ void fold_extra_rows(const AttnArgs& a, const int* tok, const int* head, const bool* live, int kvh,
+                                                int qc, float sc, float* m_run, float* l_run, float (*o)[4]) {
+  constexpr int NB = HD / 8;
+    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
+    const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
+    const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
+    long long off[2][E];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int e = 0; e < E; ++e)
+        off[i][e] = (live[i] && e < a.n_ext_max) ? a.tok_ext[(long long)tok[i] * a.n_ext_max + e] : -1;
+    // the 4 lanes of a quad own the same rows, so `off` is uniform inside the quad shuffles below
+    float sdot[2][E];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
+      __nv_bfloat162 qq[NB];
+#pragma unroll
+      for (int j = 0; j < NB; ++j) qq[j] = *reinterpret_cast<const __nv_bfloat162*>(qp + j * 8);
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        float sd = 0.f;
+        if (off[i][e] >= 0) {
+          const __nv_bfloat16* kp = ke + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
+#pragma unroll
+          for (int j = 0; j < NB; ++j) {
+            const __nv_bfloat162 kk = *reinterpret_cast<const __nv_bfloat162*>(kp + j * 8);
+            sd += __bfloat162float(qq[j].x) * __bfloat162float(kk.x) + __bfloat162float(qq[j].y) * __bfloat162float(kk.y);
+          }
+        }
+        sdot[i][e] = sd;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      float m_new = m_run[i];
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        float sd = sdot[i][e];
+        sd += __shfl_xor_sync(0xffffffffu, sd, 1);
+        sd += __shfl_xor_sync(0xffffffffu, sd, 2);
+        sdot[i][e] = off[i][e] >= 0 ? sd * sc : -INFINITY;
+        m_new = fmaxf(m_new, sdot[i][e]);
+      }
+      if (m_new == -INFINITY) continue;              // nothing visible at all (dead row)
+      const float c = (m_run[i] == -INFINITY) ? 0.f : exp2f(m_run[i] - m_new);
+      l_run[i] *= c;
+#pragma unroll
+      for (int j = 0; j < NB; ++j) { o[j][i * 2] *= c; o[j][i * 2 + 1] *= c; }
+      m_run[i] = m_new;
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        if (off[i][e] < 0) continue;
+        const float p = exp2f(sdot[i][e] - m_new);
+        l_run[i] += (qc == 0 ? p : 0.f);             // row sums are per-lane partials, reduced at the end
+        const __nv_bfloat16* vp = ve + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+          const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162*>(vp + j * 8);
+          o[j][i * 2] += p * __bfloat162float(vv.x);
+          o[j][i * 2 + 1] += p * __bfloat162float(vv.y);
+        }
+      }
+    }
+}
+
 template <int HD>
-__global__ void __launch_bounds__(kThreads) attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(kThreads, 3) attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                            const __grid_constant__ CUtensorMap tmV, AttnArgs a,
                                                            int* status) {
   constexpr int NH = HD / 64;                       // 64-column halves per tile
@@ -59,26 +131,38 @@ __global__ void __launch_bounds__(kThreads) attn_tc_kernel(const __grid_constant
 
   const int req_local = blockIdx.z, kvh = blockIdx.y, tile = blockIdx.x;
   const int G = a.Hq / a.Hkv;
-  const int n_tok = a.row_count[req_local];
+  const int4 info = a.req_info[req_local];          // {first token, token count, cache row, context length or -1}
+  const int tok0 = info.x, n_tok = info.y, request = info.z;
   const int R = n_tok * G;                          // query rows of this (request, kv head)
   const int r0 = tile * kRows;
   if (r0 >= R) return;
-  const int tok0 = a.row_start[req_local];
+  // context positions this tile needs: all of them, or (causal prefill) up to its last token's own position
+  const int max_ctx = info.w >= 0 ? info.w : min((r0 + kRows - 1) / G, n_tok - 1) + 1;
+  const int n_tiles = (max_ctx + kPos - 1) / kPos;
+  const int kv_row0 = (int)(((long long)request * a.Hkv + kvh) * (a.ctx_head_stride / HD));   // first cache row
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = base + kStages * kStageBytes;
-  __shared__ int s_max_ctx;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qr = lane >> 2, qc = lane & 3;          // fragment row (and +8) / column pair
 
-  if (threadIdx.x == 0) {
+  auto issue = [&](int t) {                          // thread 0 only
+    const int s = t % kStages;
+    const uint32_t bar = bar_base + 8u * s;
+    mbar_expect_tx(bar, kStageBytes);
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+      tma_load_2d(base + s * kStageBytes + h * (kPos * 128), &tmK, h * 64, kv_row0 + t * kPos, bar);
+      tma_load_2d(base + s * kStageBytes + kTileBytes + h * (kPos * 128), &tmV, h * 64, kv_row0 + t * kPos, bar);
+    }
+  };
+  if (threadIdx.x == 0) {                            // the first K/V tiles are on their way before anything else is read
     for (int s = 0; s < kStages; ++s) mbar_init(bar_base + 8u * s, 1);
     mbar_fence_init();
-    s_max_ctx = 0;
+    for (int t = 0; t < min(n_tiles, kStages); ++t) issue(t);
   }
-  __syncthreads();
 
   // the two rows this thread owns
   int row[2], tok[2], head[2], ctx[2];
@@ -90,9 +174,8 @@ __global__ void __launch_bounds__(kThreads) attn_tc_kernel(const __grid_constant
     const int rr = live[i] ? row[i] : r0;           // dead rows shadow the tile's first row (never stored)
     tok[i] = tok0 + rr / G;
     head[i] = kvh * G + rr % G;
-    ctx[i] = live[i] ? a.tok_ctx_len[tok[i]] : 0;
+    ctx[i] = !live[i] ? 0 : (info.w >= 0 ? info.w : rr / G + 1);
   }
-  atomicMax(&s_max_ctx, max(ctx[0], ctx[1]));
 
   // Q fragments (A operand): a0 = (qr, k0..1), a1 = (qr+8, k0..1), a2 = (qr, k8..9), a3 = (qr+8, k8..9)
   uint32_t qf[KS][4];
@@ -108,24 +191,7 @@ __global__ void __launch_bounds__(kThreads) attn_tc_kernel(const __grid_constant
       }
     }
   }
-  __syncthreads();
-  const int max_ctx = s_max_ctx;
-  const int n_tiles = (max_ctx + kPos - 1) / kPos;
-  const int request = a.tok_row[tok0];
-  const int kv_row0 = (int)(((long long)request * a.Hkv + kvh) * (a.ctx_head_stride / HD));   // first cache row
-
-  auto issue = [&](int t) {                          // thread 0 only
-    const int s = t % kStages;
-    const uint32_t bar = bar_base + 8u * s;
-    mbar_expect_tx(bar, kStageBytes);
-#pragma unroll
-    for (int h = 0; h < NH; ++h) {
-      tma_load_2d(base + s * kStageBytes + h * (kPos * 128), &tmK, h * 64, kv_row0 + t * kPos, bar);
-      tma_load_2d(base + s * kStageBytes + kTileBytes + h * (kPos * 128), &tmV, h * 64, kv_row0 + t * kPos, bar);
-    }
-  };
-  if (threadIdx.x == 0)
-    for (int t = 0; t < min(n_tiles, kStages); ++t) issue(t);
+  __syncthreads();                                   // barrier initialisation visible to every waiter
 
   float o[NB][4];
 #pragma unroll
@@ -222,46 +288,9 @@ __global__ void __launch_bounds__(kThreads) attn_tc_kernel(const __grid_constant
     return;
   }
 
-  // ---- the token's own extra KV rows (drafted codes of its tuple), straight from global memory
-  if (a.n_ext_max > 0) {
-    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
-    const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
-    const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
-      for (int e = 0; e < a.n_ext_max; ++e) {
-        const long long off = live[i] ? a.tok_ext[(long long)tok[i] * a.n_ext_max + e] : -1;
-        // the 4 lanes of a quad own the same rows, so `off` is uniform inside the quad shuffles below
-        const long long eo = off + (long long)kvh * a.ext_head_stride + qc * 2;
-        float sdot = 0.f;
-        if (off >= 0) {
-#pragma unroll
-          for (int j = 0; j < NB; ++j) {
-            const __nv_bfloat162 qq = *reinterpret_cast<const __nv_bfloat162*>(qp + j * 8);
-            const __nv_bfloat162 kk = *reinterpret_cast<const __nv_bfloat162*>(ke + eo + j * 8);
-            sdot += __bfloat162float(qq.x) * __bfloat162float(kk.x) + __bfloat162float(qq.y) * __bfloat162float(kk.y);
-          }
-        }
-        sdot += __shfl_xor_sync(0xffffffffu, sdot, 1);
-        sdot += __shfl_xor_sync(0xffffffffu, sdot, 2);
-        if (off >= 0) {
-          const float sv = sdot * sc;
-          const float m_new = fmaxf(m_run[i], sv);
-          const float c = (m_run[i] == -INFINITY) ? 0.f : exp2f(m_run[i] - m_new);
-          const float p = exp2f(sv - m_new);
-          l_run[i] = l_run[i] * c + (qc == 0 ? p : 0.f);   // row sums are per-lane partials, reduced at the end
-          m_run[i] = m_new;
-#pragma unroll
-          for (int j = 0; j < NB; ++j) {
-            const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162*>(ve + eo + j * 8);
-            o[j][i * 2] = o[j][i * 2] * c + p * __bfloat162float(vv.x);
-            o[j][i * 2 + 1] = o[j][i * 2 + 1] * c + p * __bfloat162float(vv.y);
-          }
-        }
-      }
-    }
-  }
+  // ---- the token's own extra KV rows (drafted codes of its tuple)
+  if (a.n_ext_max > 4) fold_extra_rows<HD, kMaxLevels>(a, tok, head, live, kvh, qc, sc, m_run, l_run, o);
+  else if (a.n_ext_max > 0) fold_extra_rows<HD, 4>(a, tok, head, live, kvh, qc, sc, m_run, l_run, o);
 
   // ---- normalise and store
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out);
@@ -295,7 +324,7 @@ void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cud
 }  // namespace
 
 bool attention_tc_supported(const AttnArgs& a) {
-  if (!a.status || !a.row_start || !a.row_count || a.n_rows <= 0 || a.max_tokens_per_row <= 0) return false;
+  if (!a.status || !a.req_info || a.n_rows <= 0 || a.max_tokens_per_row <= 0) return false;
   if (a.hd != 64 && a.hd != 128) return false;
   if (!tma_encode_fn()) return false;
   if (a.ctx_head_stride % a.hd || a.ctx_row_stride != a.ctx_head_stride * a.Hkv) return false;

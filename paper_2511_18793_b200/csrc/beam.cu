@@ -332,7 +332,7 @@ __global__ void nodes_count_kernel(EngineState e, int batch) {
   if (threadIdx.x == 0) n_alive = 0;
   __syncthreads();
   if (m >= L) {
-    if (threadIdx.x == 0) { e.row_tok_count[b] = 0; e.row_cur[b] = -1; }
+    if (threadIdx.x == 0) { e.row_tok_count[b] = 0; e.row_cur[b] = -1; e.req_info[b] = make_int4(0, 0, b, 0); }
     for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) e.d_alive[b * e.Kmax + k] = 0;
     return;
   }
@@ -369,6 +369,7 @@ __global__ void nodes_fill_kernel(EngineState e, int batch) {
     for (int i = 0; i < b; ++i) off += e.row_tok_count[i];
     s_off = off;
     e.row_tok_start[b] = off;
+    if (e.row_tok_count[b] > 0) e.req_info[b] = make_int4(off, e.row_tok_count[b], b, e.row_P[b]);
     if (b == batch - 1) *e.n_tokens = off + e.row_tok_count[b];
     int c = 0;
     for (int k = 0; k < Kmax; ++k) { s_alive_rank[k] = c; c += e.d_alive[b * Kmax + k]; }
@@ -434,7 +435,10 @@ __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams
   const long long slab_elems = (long long)Kmax * e.Hkv * e.hd;
   const long long row_elems = (long long)(L - 1) * slab_elems;
   if (b == 0 && threadIdx.x == 0) *e.n_tokens = batch * per_row;
-  if (threadIdx.x == 0) { e.row_tok_start[b] = b * per_row; e.row_tok_count[b] = per_row; }
+  if (threadIdx.x == 0) {
+    e.row_tok_start[b] = b * per_row; e.row_tok_count[b] = per_row;
+    e.req_info[b] = make_int4(b * per_row, per_row, b, P);
+  }
   for (int i = threadIdx.x; i < L * Kmax; i += blockDim.x) e.node_index[(long long)b * L * Kmax + i] = -1;
   __syncthreads();
   for (int idx = threadIdx.x; idx < per_row; idx += blockDim.x) {
@@ -691,7 +695,10 @@ __global__ void prefill_tokens_kernel(EngineState e, const int* hist, const int*
   }
   e.tok_id[idx] = tok; e.tok_pos[idx] = p; e.tok_row[idx] = b; e.tok_ctx_len[idx] = p + 1;
   e.tok_kv_dst[idx] = ((long long)b * e.Hkv * S_cap + p) * e.hd;
-  if (p == 0) { e.row_P[b] = P; e.pf_row_start[lb] = lb * S_call; e.pf_row_count[lb] = S_call; }
+  if (p == 0) {
+    e.row_P[b] = P; e.pf_row_start[lb] = lb * S_call; e.pf_row_count[lb] = S_call;
+    e.pf_req_info[lb] = make_int4(lb * S_call, S_call, b, -1);
+  }
   if (p >= P - 1 && p <= P - 1 + L) h_rows[lb * (L + 1) + (p - (P - 1))] = (int)idx;
 }
 

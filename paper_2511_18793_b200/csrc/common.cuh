@@ -188,6 +188,8 @@ struct AttnArgs {
   float scale;
   // grouping of the token list by request (tokens of a request are contiguous), for the tensor-core kernel
   const int* row_start; const int* row_count;   // [n_rows] first token / token count of each request in this pass
+  const int4* req_info;                         // [n_rows] {first token, token count, cache row, context length visible to
+                                                //  every token of the request, or -1: token j of the request sees j + 1}
   int n_rows, max_tokens_per_row;
   long long ctx_rows_total;                     // requests * kv heads * positions of the layer's context cache
   int* status;

@@ -37,6 +37,8 @@ struct EngineState {
   int* row_tok_count;   // [Bmax]
   int* row_tok_start;   // [Bmax] first token of the request in the list
   int* pf_row_start; int* pf_row_count;   // [Bmax] the same for a prefill chunk (indexed by row within the chunk)
+  int4* req_info; int4* pf_req_info;      // [Bmax] {first token, token count, cache row, context length or -1 = causal}:
+                                          //        all the attention kernel needs to know about a request, in one load
   int* n_tokens;        // [1]
   int* counters;        // [8]: 0 unfinished rows, 1 primary tokens (round), 2 accepted levels (round), 3 drafted (round)
 
