@@ -197,6 +197,9 @@ def main():
     catalog = synth.make_catalog(w)
     hist = synth.make_histories(w, catalog)
     cat_dev = torch.from_numpy(catalog).to(dev)
+    # a stream of its own (not the legacy default stream), so that the library may capture its rounds into CUDA graphs;
+    # made current, so that the flushes, copies and timing events below are ordered on it too
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
     eng = binding.Engine(binding.make_config(w), weights, cat_dev, w.load_factor, stream=torch.cuda.current_stream())
     n_unique = eng.build_hashset()
     assert n_unique == w.n_items

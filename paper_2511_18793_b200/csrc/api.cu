@@ -2,8 +2,11 @@
 // No model arithmetic happens on the host; it only orders kernel launches.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
+#include <array>
+#include <map>
 #include <string>
 #include <vector>
 
@@ -22,6 +25,9 @@ void launch_prefill_tokens(const EngineState& e, const int* hist, const int* n_h
                            int S_call, int S_cap, int* h_rows, cudaStream_t st);
 unsigned long long profile_total_launches();
 void profile_enable(bool on);
+bool profile_is_on();
+void profile_counts(long long* out);
+void profile_add(const long long* delta);
 void profile_read(nezha_profile* out);
 bool gemm_tc_supported(const GemmArgs& a);
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
@@ -74,6 +80,10 @@ struct nezha_ctx {
   int* h_rows; unsigned long long* n_unique_dev;
   EngineState es;
   int* host_counters;       // pinned
+  // CUDA graphs of the decode segments (one per round), keyed by everything that shapes the launch sequence
+  struct Segment { int seen; cudaGraphExec_t exec; long long launches[kcCount]; };
+  std::map<std::array<uintptr_t, 16>, Segment> segments;
+  bool use_graphs;
   int state;                // 0 created, 1 hash set built, 2 prefilled
   int batch;                // prefilled batch
   std::string err;
@@ -412,6 +422,40 @@ nezha_status pending_device_error(nezha_ctx* c) {
   return NEZHA_OK;
 }
 
+// Runs one segment of a decode call (the part before the rounds, or one round).  The launch sequence of a segment
+// is fixed by its key, so after one eager run it is captured into a CUDA graph and replayed from then on: one
+// launch per round instead of dozens, and no launch gaps between its kernels.  Eager when the stream cannot be
+// captured, while per-launch event timing is on, or if capture fails.
+template <typename F>
+nezha_status run_segment(nezha_ctx* c, const std::array<uintptr_t, 16>& key, F&& body) {
+  if (!c->use_graphs || profile_is_on()) { body(); return NEZHA_OK; }
+  nezha_ctx::Segment& sg = c->segments[key];
+  if (sg.exec) {
+    NZ_CUDA(c, cudaGraphLaunch(sg.exec, c->st));
+    profile_add(sg.launches);
+    return NEZHA_OK;
+  }
+  if (sg.seen++ == 0 || sg.seen > 3) { body(); return NEZHA_OK; }    // first run eager (one-time set-up calls); give up after failures
+  long long before[kcCount], after[kcCount];
+  profile_counts(before);
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); body(); return NEZHA_OK; }
+  body();
+  const cudaError_t e = cudaStreamEndCapture(c->st, &graph);
+  profile_counts(after);
+  if (e != cudaSuccess || !graph || cudaGraphInstantiate(&sg.exec, graph, 0) != cudaSuccess) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    sg.exec = nullptr;
+    body();                                       // nothing ran during the failed capture
+    return NEZHA_OK;
+  }
+  cudaGraphDestroy(graph);
+  for (int i = 0; i < kcCount; ++i) sg.launches[i] = after[i] - before[i];
+  NZ_CUDA(c, cudaGraphLaunch(sg.exec, c->st));   // the capture itself executed nothing
+  return NEZHA_OK;
+}
+
 nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* drafts, const int* n_draft,
                          int* out_codes, float* out_scores, int* out_count, nezha_decode_stats* stats,
                          const nezha_trace* trace) {
@@ -425,29 +469,33 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
   if (trace) tr = *trace;
   nezha_decode_stats sd{};
   const int R = L - 1;
-  if (tr.drafts) launch_fill_i32(tr.drafts, (long long)R * batch * K * L, -1, c->st);
-  if (tr.n_draft) launch_fill_i32(tr.n_draft, (long long)R * batch, -1, c->st);
-  if (tr.accepted_len) launch_fill_i32(tr.accepted_len, (long long)R * batch * K, -1, c->st);
-  if (tr.level_reached) launch_fill_i32(tr.level_reached, (long long)R * batch, -1, c->st);
-  launch_fill_i32(out_codes, (long long)batch * K * L, -1, c->st);
-  launch_fill_f32(out_scores, (long long)batch * K, -INFINITY, c->st);
-  launch_fill_i32(out_count, batch, 0, c->st);
-  launch_init_decode(e, batch, c->st);
-
-  if (mode == NEZHA_MODE_DRAFT) {
-    draft_phase(c, batch, K, true, 1, true);
-    const size_t lv = (size_t)L * c->Bmax * c->Kmax;
-    launch_write_out(e.dw_codes + lv * L, e.dw_score + lv, e.dw_count + (size_t)L * c->Bmax, c->Kmax, L, batch, K,
-                     out_codes, out_scores, out_count, c->st);
-    nezha_status ps = pending_device_error(c);
-    if (stats) *stats = sd;
-    return ps;
-  }
-
-  // B_1 from the prefill hidden state h_0 (Algorithm 1's LM head, top-K and pruning at l = 1)
-  gemm(c, c->h_act, (long long)(L + 1) * c->d, c->lm_head, c->d, c->logits0, c->cfg.T[0], batch, nullptr, c->cfg.T[0], c->d,
-       kEpiStoreF32);
-  {
+  auto key_of = [&](int segment) {
+    std::array<uintptr_t, 16> k{};
+    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)mode;
+    k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
+    k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
+    k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams; k[14] = (uintptr_t)tr.beam_scores;
+    return k;
+  };
+  nezha_status rs = run_segment(c, key_of(0), [&] {
+    if (tr.drafts) launch_fill_i32(tr.drafts, (long long)R * batch * K * L, -1, c->st);
+    if (tr.n_draft) launch_fill_i32(tr.n_draft, (long long)R * batch, -1, c->st);
+    if (tr.accepted_len) launch_fill_i32(tr.accepted_len, (long long)R * batch * K, -1, c->st);
+    if (tr.level_reached) launch_fill_i32(tr.level_reached, (long long)R * batch, -1, c->st);
+    launch_fill_i32(out_codes, (long long)batch * K * L, -1, c->st);
+    launch_fill_f32(out_scores, (long long)batch * K, -INFINITY, c->st);
+    launch_fill_i32(out_count, batch, 0, c->st);
+    launch_init_decode(e, batch, c->st);
+    if (mode == NEZHA_MODE_DRAFT) {
+      draft_phase(c, batch, K, true, 1, true);
+      const size_t lv = (size_t)L * c->Bmax * c->Kmax;
+      launch_write_out(e.dw_codes + lv * L, e.dw_score + lv, e.dw_count + (size_t)L * c->Bmax, c->Kmax, L, batch, K,
+                       out_codes, out_scores, out_count, c->st);
+      return;
+    }
+    // B_1 from the prefill hidden state h_0 (Algorithm 1's LM head, top-K and pruning at l = 1)
+    gemm(c, c->h_act, (long long)(L + 1) * c->d, c->lm_head, c->d, c->logits0, c->cfg.T[0], batch, nullptr, c->cfg.T[0], c->d,
+         kEpiStoreF32);
     SelectArgs s = select_base(c, batch, K);
     const size_t lv_out = (size_t)1 * c->Bmax * c->Kmax;
     s.logits = c->logits0; s.row_stride = c->cfg.T[0]; s.col_off = 0; s.src_row = nullptr; s.src_mul = 1;
@@ -459,30 +507,40 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     // settle level 1 (for L == 1 this also writes the result)
     launch_fill_i32(e.row_cur, batch, 0, c->st);
     launch_advance(e, batch, 0, K, out_codes, out_scores, out_count, c->st);
+  });
+  if (rs != NEZHA_OK) return rs;
+  if (mode == NEZHA_MODE_DRAFT) {
+    nezha_status ps = pending_device_error(c);
+    if (stats) *stats = sd;
+    return ps;
   }
   for (int round = 1; round <= R; ++round) {
-    NZ_CUDA(c, cudaMemsetAsync(e.counters, 0, 8 * sizeof(int), c->st));
-    if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
-    else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
-    else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, true);
-    launch_build_nodes(e, batch, c->st);
-    verify_pass(c, (long long)batch * K * (L - round), batch, K * (L - round));
-    for (int n = round; n < L; ++n) {
-      SelectArgs s = select_base(c, batch, K);
-      const size_t lv_in = (size_t)n * c->Bmax * c->Kmax, lv_out = (size_t)(n + 1) * c->Bmax * c->Kmax;
-      s.logits = c->logits_v; s.row_stride = c->Nv; s.col_off = e.li.off[n] - e.li.off[1];
-      s.src_row = e.tb_src + lv_in; s.src_mul = 0;
-      s.in_codes = e.tb_codes + lv_in * L; s.in_score = e.tb_score + lv_in; s.in_count = e.tb_count + (size_t)n * c->Bmax;
-      s.n = n; s.T = c->cfg.T[n]; s.per_beam = s.T; s.filter = (n + 1 == L) ? 1 : 0;
-      s.gate = e.row_cur; s.gate_mode = 1; s.gate_value = n;
-      s.out_codes = e.tb_codes + lv_out * L; s.out_score = e.tb_score + lv_out; s.out_parent = e.tb_parent + lv_out;
-      s.out_count = e.tb_count + (size_t)(n + 1) * c->Bmax;
-      launch_select(s, c->st);
-      launch_advance(e, batch, n, K, out_codes, out_scores, out_count, c->st);
-    }
-    launch_round_end(e, batch, K, round, tr, c->st);
-    NZ_CUDA(c, cudaMemcpyAsync(c->host_counters, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    rs = run_segment(c, key_of(round), [&] {
+      cudaMemsetAsync(e.counters, 0, 8 * sizeof(int), c->st);
+      if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
+      else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
+      else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, true);
+      launch_build_nodes(e, batch, c->st);
+      verify_pass(c, (long long)batch * K * (L - round), batch, K * (L - round));
+      for (int n = round; n < L; ++n) {
+        SelectArgs s = select_base(c, batch, K);
+        const size_t lv_in = (size_t)n * c->Bmax * c->Kmax, lv_out = (size_t)(n + 1) * c->Bmax * c->Kmax;
+        s.logits = c->logits_v; s.row_stride = c->Nv; s.col_off = e.li.off[n] - e.li.off[1];
+        s.src_row = e.tb_src + lv_in; s.src_mul = 0;
+        s.in_codes = e.tb_codes + lv_in * L; s.in_score = e.tb_score + lv_in; s.in_count = e.tb_count + (size_t)n * c->Bmax;
+        s.n = n; s.T = c->cfg.T[n]; s.per_beam = s.T; s.filter = (n + 1 == L) ? 1 : 0;
+        s.gate = e.row_cur; s.gate_mode = 1; s.gate_value = n;
+        s.out_codes = e.tb_codes + lv_out * L; s.out_score = e.tb_score + lv_out; s.out_parent = e.tb_parent + lv_out;
+        s.out_count = e.tb_count + (size_t)(n + 1) * c->Bmax;
+        launch_select(s, c->st);
+        launch_advance(e, batch, n, K, out_codes, out_scores, out_count, c->st);
+      }
+      launch_round_end(e, batch, K, round, tr, c->st);
+      cudaMemcpyAsync(c->host_counters, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st);
+    });
+    if (rs != NEZHA_OK) return rs;
     NZ_CUDA(c, cudaStreamSynchronize(c->st));
+    NZ_CUDA(c, cudaGetLastError());
     sd.rounds = round;
     sd.primary_tokens += c->host_counters[1];
     sd.accepted_levels += c->host_counters[2];
@@ -521,6 +579,8 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   nezha_ctx* c = new nezha_ctx();
   c->cfg = *cfg; c->n_items = n_items; c->load_factor = load_factor; c->catalog = catalog_codes;
   c->st = (cudaStream_t)cuda_stream; c->arena = nullptr; c->state = 0; c->batch = 0;
+  // the legacy default stream cannot be captured; NEZHA_NO_GRAPHS=1 keeps every launch eager
+  c->use_graphs = cuda_stream != nullptr && !getenv("NEZHA_NO_GRAPHS");
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;
@@ -831,6 +891,8 @@ const char* nezha_last_error(const nezha_ctx* c) { return c ? c->err.c_str() : "
 
 void nezha_destroy(nezha_ctx* c) {
   if (!c) return;
+  for (auto& kv : c->segments)
+    if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
   if (c->host_counters) cudaFreeHost(c->host_counters);
   delete c;
 }

@@ -66,13 +66,25 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
     const unsigned long long mult_n = a.li.mult[a.n];
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
-      const int t = lane + 32 * j;
-      if (t < a.T) {
+      if (lane + 32 * j < a.T) {
         key[j] -= lse;                                   // log-probability
-        if (all_codes) {
-          key[j] += base;                                // rank by cumulative log-probability
-          if (a.filter && !hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n)) key[j] = -INFINITY;
+        if (all_codes) key[j] += base;                   // rank by cumulative log-probability
+      }
+    }
+    if (all_codes && a.filter) {                         // Eq. 5 on every extension of the beam, 8 probes in flight
+      constexpr int PB = VPL < 8 ? VPL : 8;
+#pragma unroll
+      for (int j0 = 0; j0 < VPL; j0 += PB) {
+        unsigned long long pk[PB]; bool want_probe[PB], ok[PB];
+#pragma unroll
+        for (int j = 0; j < PB; ++j) {
+          want_probe[j] = lane + 32 * (j0 + j) < a.T;
+          pk[j] = prefix_key + (unsigned long long)(lane + 32 * (j0 + j)) * mult_n;
         }
+        hs_contains_many<PB>(a.hs, pk, want_probe, ok);
+#pragma unroll
+        for (int j = 0; j < PB; ++j)
+          if (want_probe[j] && !ok[j]) key[j0 + j] = -INFINITY;
       }
     }
     // ordered extraction

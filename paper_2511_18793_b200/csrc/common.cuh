@@ -83,6 +83,30 @@ __device__ __forceinline__ bool hs_contains_thread(const HashSetView& hs, unsign
   return false;
 }
 
+// Membership of N keys per thread with the memory round trips overlapped: the home buckets of all keys are loaded
+// first (independent loads), and only a key whose home bucket is full without holding it walks on alone.
+template <int N>
+__device__ __forceinline__ void hs_contains_many(const HashSetView& hs, const unsigned long long* keys, const bool* want,
+                                                 bool* found) {
+  ulonglong2 lo[N], hi[N];
+#pragma unroll
+  for (int j = 0; j < N; ++j) {
+    if (want[j]) {
+      const ulonglong2* p = reinterpret_cast<const ulonglong2*>(hs.slots + hs_bucket(keys[j], hs.n_buckets) * kBucketSlots);
+      lo[j] = __ldg(p); hi[j] = __ldg(p + 1);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < N; ++j) {
+    found[j] = false;
+    if (!want[j]) continue;
+    const unsigned long long k = keys[j];
+    if (lo[j].x == k || lo[j].y == k || hi[j].x == k || hi[j].y == k) found[j] = true;
+    else if (lo[j].x == kEmptyKey || lo[j].y == kEmptyKey || hi[j].x == kEmptyKey || hi[j].y == kEmptyKey) found[j] = false;
+    else found[j] = hs_contains_thread(hs, k);        // home bucket full: rare at the load factors in use
+  }
+}
+
 // --------------------------------------------------------------------------------------------------
 // model / engine description shared by the host code and the kernels
 // --------------------------------------------------------------------------------------------------

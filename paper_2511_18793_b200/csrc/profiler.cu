@@ -35,6 +35,17 @@ LaunchScope::~LaunchScope() {
 
 unsigned long long profile_total_launches() { return g_total; }
 
+bool profile_is_on() { return g_on; }
+
+// Launch counts per class so far (for code that replays a captured CUDA graph: it snapshots before and after the
+// capture and adds the difference on every replay).
+void profile_counts(long long* out) {
+  for (int i = 0; i < kcCount; ++i) out[i] = g_launches[i];
+}
+void profile_add(const long long* delta) {
+  for (int i = 0; i < kcCount; ++i) { g_launches[i] += delta[i]; g_total += (unsigned long long)delta[i]; }
+}
+
 void profile_enable(bool on) {
   g_on = on;
   g_used = 0;

@@ -49,7 +49,8 @@ def e2e_tolerance(w, std=0.02):
 class Case:
     """Engine + oracle on one workload.  Weights are drawn once and handed to both sides as the same bytes."""
 
-    def __init__(self, w, device="cuda", max_beam=None, catalog=None, hist=None, weights=None, oracle_dtype=np.float64):
+    def __init__(self, w, device="cuda", max_beam=None, catalog=None, hist=None, weights=None, oracle_dtype=np.float64,
+                 stream=None):
         from paper_2511_18793_b200 import binding
         self.binding = binding
         self.w = w
@@ -60,7 +61,7 @@ class Case:
         self.cat_dev = torch.from_numpy(self.catalog).to(device)
         cfg = binding.make_config(w, max_batch=self.hist.shape[0], max_beam=max_beam or w.beam,
                                   max_hist_items=self.hist.shape[1])
-        self.eng = binding.Engine(cfg, self.weights, self.cat_dev, load_factor=w.load_factor)
+        self.eng = binding.Engine(cfg, self.weights, self.cat_dev, load_factor=w.load_factor, stream=stream)
         self.n_unique = self.eng.build_hashset()
         self.hist_dev = torch.from_numpy(self.hist).to(device)
         self.n_hist = torch.full((self.hist.shape[0],), self.hist.shape[1], dtype=torch.int32, device=device)

@@ -127,3 +127,39 @@ def test_bf16_shapes_ragged_histories(shape):
     scores = out["trace"]["beam_scores"].cpu().numpy()
     for b in range(w.batch):
         check_levels(case, b, beams[:, b], scores[:, b], w.beam)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_graph_replay_equals_eager_launches(name):
+    """On a stream of its own the library captures every round of a decode call into a CUDA graph after one eager
+    run and replays it afterwards.  Eager, capturing and replaying calls must give the same bits as an engine on the
+    default stream (which never captures), in every mode, with and without trace outputs and with injected drafts."""
+    w = synth.WORKLOADS[name]
+    ref = Case(w).prefill()
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(st):
+        cap = Case(w, weights=ref.weights, catalog=ref.catalog, hist=ref.hist, stream=st).prefill()
+        for mode in (1, 0, 2):
+            want = ref.eng.decode(w.beam, mode=mode, trace=(mode == 1))
+            out = cap.eng.alloc_outputs(w.batch, w.beam, trace=(mode == 1))
+            for call in range(4):                                   # eager, capture, replay, replay
+                got = cap.eng.decode(w.beam, mode=mode, out=out)
+                st.synchronize()
+                for k in ("codes", "scores", "count"):
+                    assert torch.equal(got[k], want[k]), (mode, call, k)
+                assert got["stats"].rounds == want["stats"].rounds
+                assert got["stats"].primary_tokens == want["stats"].primary_tokens
+                if mode == 1:
+                    for k, v in want["trace"].items():
+                        assert torch.equal(got["trace"][k], v), (call, k)
+        drafts = want["codes"].clone().clamp_(min=0)
+        nd = want["count"].clone()
+        w1 = ref.eng.decode_with_drafts(w.beam, drafts, nd)
+        out = cap.eng.alloc_outputs(w.batch, w.beam)
+        for call in range(3):
+            g1 = cap.eng.decode_with_drafts(w.beam, drafts, nd, out=out)
+            st.synchronize()
+            assert torch.equal(g1["codes"], w1["codes"]) and torch.equal(g1["scores"], w1["scores"])
+            assert g1["stats"].rounds == w1["stats"].rounds
+    torch.cuda.synchronize()
