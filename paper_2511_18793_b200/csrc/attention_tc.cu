@@ -1,12 +1,17 @@
 // Tensor-core KV-cache attention (bf16) with TMA-staged K/V tiles.
 //
-// One CTA = (request, KV head, tile of 64 query rows).  The query rows of a (request, KV head) pair are all of the
-// request's tokens in this pass times the G query heads of the group, so the request's context K/V is streamed
-// from HBM once per (request, KV head, layer) and shared by every beam, draft level and grouped head -- not
-// re-read per token.  K/V tiles of 64 positions are brought into shared memory by TMA (128-byte swizzle, a
-// 3-deep ring), S = Q K^T and O += P V run on mma.sync m16n8k16 with fp32 accumulation and an online softmax in
-// registers.  The per-token extra KV rows (the token's own tuple's drafted codes, at most L-1 of them) are
-// folded in afterwards straight from global memory.  The full-barrier wait is bounded (error flag + return).
+// One CTA = (request, KV head, tile of 16 * RW query rows).  The query rows of a (request, KV head) pair are all of the
+// request's tokens in this pass times the G query heads of the group, so the request's context K/V is streamed once
+// per (request, KV head, layer) and shared by every beam, draft level and grouped head -- not re-read per token.
+// A producer warp brings K/V tiles of 64 positions into a shared-memory ring with TMA (128-byte swizzle); RW x KW
+// consumer warps run S = Q K^T and O += P V on mma.sync m16n8k16 (fp32 accumulation) with an online softmax in
+// registers.  Two shapes of the same kernel:
+//   RW = 4, KW = 1   64 rows per CTA, every warp walks all tiles                       (many query rows per request)
+//   RW = 1, KW = 4   16 rows per CTA, the four warps take every fourth tile and their   (few rows: one beam set of a
+//                    softmax states are merged through shared memory at the end          small model, plain decode)
+// Ring slots are handed back to the producer with per-slot "empty" mbarriers, so warps never wait for each other.
+// The per-token extra KV rows (the token's own tuple's drafted codes, at most L-1 of them) are folded in afterwards
+// straight from global memory.  Every barrier wait is bounded (abort flag + error status + return).
 #include <math.h>
 
 #include "tma.cuh"
@@ -15,10 +20,7 @@ namespace nz {
 
 namespace {
 
-constexpr int kRows = 64;        // query rows per CTA (4 warps x 16)
 constexpr int kPos = 64;         // KV positions per tile
-constexpr int kStages = 3;
-constexpr int kThreads = 128;
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -38,6 +40,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ float ex2(float x) {      // 2^x, flushing; ex2(-inf) = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // Address of the 16-byte chunk `chunk` (dims chunk*8 .. +7) of position `pos` inside a K or V stage buffer made of
 // HD/64 sub-tiles of [64 positions x 128 bytes], each written by TMA with the 128-byte swizzle.
@@ -48,86 +55,99 @@ __device__ __forceinline__ uint32_t kv_addr(uint32_t tile, int pos, int chunk) {
 }
 
 // The token's own extra KV rows (drafted codes of its tuple), straight from global memory, folded into the running
-// softmax state of the thread's two rows.  The loads of all (row, entry) pairs are issued together -- offsets, then
-// every K row, then every V row -- so the chain of dependent memory round trips is three long whatever the number
-// of entries.  E = compile-time bound of the entries per token (n_ext_max <= E).
+// softmax state of the thread's two rows (m in the scaled log2 domain).  The loads of all (row, entry) pairs are
+// issued together -- offsets, then every K row, then every V row -- so the chain of dependent memory round trips is
+// three long whatever the number of entries.  E = compile-time bound of the entries per token (n_ext_max <= E).
 template <int HD, int E>
 __device__ __forceinline__ void fold_extra_rows(const AttnArgs& a, const int* tok, const int* head, const bool* live, int kvh,
                                                 int qc, float sc, float* m_run, float* l_run, float (*o)[4]) {
   constexpr int NB = HD / 8;
-    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
-    const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
-    const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
-    long long off[2][E];
+  const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
+  const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
+  const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
+  long long off[2][E];
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
+  for (int i = 0; i < 2; ++i)
 #pragma unroll
-      for (int e = 0; e < E; ++e)
-        off[i][e] = (live[i] && e < a.n_ext_max) ? a.tok_ext[(long long)tok[i] * a.n_ext_max + e] : -1;
-    // the 4 lanes of a quad own the same rows, so `off` is uniform inside the quad shuffles below
-    float sdot[2][E];
+    for (int e = 0; e < E; ++e)
+      off[i][e] = (live[i] && e < a.n_ext_max) ? a.tok_ext[(long long)tok[i] * a.n_ext_max + e] : -1;
+  // the 4 lanes of a quad own the same rows, so `off` is uniform inside the quad shuffles below
+  float sdot[2][E];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
-      __nv_bfloat162 qq[NB];
+  for (int i = 0; i < 2; ++i) {
+    const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
+    __nv_bfloat162 qq[NB];
 #pragma unroll
-      for (int j = 0; j < NB; ++j) qq[j] = *reinterpret_cast<const __nv_bfloat162*>(qp + j * 8);
+    for (int j = 0; j < NB; ++j) qq[j] = *reinterpret_cast<const __nv_bfloat162*>(qp + j * 8);
 #pragma unroll
-      for (int e = 0; e < E; ++e) {
-        float sd = 0.f;
-        if (off[i][e] >= 0) {
-          const __nv_bfloat16* kp = ke + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
-#pragma unroll
-          for (int j = 0; j < NB; ++j) {
-            const __nv_bfloat162 kk = *reinterpret_cast<const __nv_bfloat162*>(kp + j * 8);
-            sd += __bfloat162float(qq[j].x) * __bfloat162float(kk.x) + __bfloat162float(qq[j].y) * __bfloat162float(kk.y);
-          }
-        }
-        sdot[i][e] = sd;
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      float m_new = m_run[i];
-#pragma unroll
-      for (int e = 0; e < E; ++e) {
-        float sd = sdot[i][e];
-        sd += __shfl_xor_sync(0xffffffffu, sd, 1);
-        sd += __shfl_xor_sync(0xffffffffu, sd, 2);
-        sdot[i][e] = off[i][e] >= 0 ? sd * sc : -INFINITY;
-        m_new = fmaxf(m_new, sdot[i][e]);
-      }
-      if (m_new == -INFINITY) continue;              // nothing visible at all (dead row)
-      const float c = (m_run[i] == -INFINITY) ? 0.f : exp2f(m_run[i] - m_new);
-      l_run[i] *= c;
-#pragma unroll
-      for (int j = 0; j < NB; ++j) { o[j][i * 2] *= c; o[j][i * 2 + 1] *= c; }
-      m_run[i] = m_new;
-#pragma unroll
-      for (int e = 0; e < E; ++e) {
-        if (off[i][e] < 0) continue;
-        const float p = exp2f(sdot[i][e] - m_new);
-        l_run[i] += (qc == 0 ? p : 0.f);             // row sums are per-lane partials, reduced at the end
-        const __nv_bfloat16* vp = ve + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
+    for (int e = 0; e < E; ++e) {
+      float sd = 0.f;
+      if (off[i][e] >= 0) {
+        const __nv_bfloat16* kp = ke + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
 #pragma unroll
         for (int j = 0; j < NB; ++j) {
-          const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162*>(vp + j * 8);
-          o[j][i * 2] += p * __bfloat162float(vv.x);
-          o[j][i * 2 + 1] += p * __bfloat162float(vv.y);
+          const __nv_bfloat162 kk = *reinterpret_cast<const __nv_bfloat162*>(kp + j * 8);
+          sd += __bfloat162float(qq[j].x) * __bfloat162float(kk.x) + __bfloat162float(qq[j].y) * __bfloat162float(kk.y);
         }
       }
+      sdot[i][e] = sd;
     }
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    float m_new = m_run[i];
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      float sd = sdot[i][e];
+      sd += __shfl_xor_sync(0xffffffffu, sd, 1);
+      sd += __shfl_xor_sync(0xffffffffu, sd, 2);
+      sdot[i][e] = off[i][e] >= 0 ? sd * sc : -INFINITY;
+      m_new = fmaxf(m_new, sdot[i][e]);
+    }
+    if (m_new == -INFINITY) continue;              // nothing visible at all (dead row)
+    const float c = ex2(m_run[i] - m_new);
+    l_run[i] *= c;
+#pragma unroll
+    for (int j = 0; j < NB; ++j) { o[j][i * 2] *= c; o[j][i * 2 + 1] *= c; }
+    m_run[i] = m_new;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      if (off[i][e] < 0) continue;
+      const float p = ex2(sdot[i][e] - m_new);
+      l_run[i] += (qc == 0 ? p : 0.f);             // row sums are per-lane partials, reduced at the end
+      const __nv_bfloat16* vp = ve + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
+#pragma unroll
+      for (int j = 0; j < NB; ++j) {
+        const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162*>(vp + j * 8);
+        o[j][i * 2] += p * __bfloat162float(vv.x);
+        o[j][i * 2 + 1] += p * __bfloat162float(vv.y);
+      }
+    }
+  }
 }
 
-template <int HD>
-__global__ void __launch_bounds__(kThreads, 3) attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                           const __grid_constant__ CUtensorMap tmV, AttnArgs a,
-                                                           int* status) {
+template <int HD, int RW, int KW>
+struct AttnCfg {
+  static constexpr int kStages = KW == 1 ? 3 : 4;                 // a multiple of KW: slot s always serves warp group s % KW
+  static constexpr int kConsumers = RW * KW;
+  static constexpr int kThreads = (kConsumers + 1) * 32;          // + the producer warp
+  static constexpr int kTileBytes = kPos * HD * 2;                // one K (or V) tile
+  static constexpr int kStageBytes = 2 * kTileBytes;
+  static constexpr int kMergeFloats = (HD / 8) * 4 + 4;           // o fragments + (m, l) of two rows, per thread
+  static constexpr int kMergeBytes = (KW - 1) * RW * kMergeFloats * 32 * 4;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 128 + kMergeBytes;
+};
+
+template <int HD, int RW, int KW>
+__global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                                               const __grid_constant__ CUtensorMap tmV,
+                                                                               AttnArgs a, int* status) {
+  using C = AttnCfg<HD, RW, KW>;
+  constexpr int S = C::kStages;
   constexpr int NH = HD / 64;                       // 64-column halves per tile
-  constexpr int kTileBytes = kPos * HD * 2;         // one K (or V) tile
-  constexpr int kStageBytes = 2 * kTileBytes;
   constexpr int KS = HD / 16;                       // k-steps of Q K^T
   constexpr int NB = HD / 8;                        // n-blocks of the output
+  constexpr int kRows = 16 * RW;
 
   const int req_local = blockIdx.z, kvh = blockIdx.y, tile = blockIdx.x;
   const int G = a.Hq / a.Hkv;
@@ -143,149 +163,198 @@ __global__ void __launch_bounds__(kThreads, 3) attn_tc_kernel(const __grid_const
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = base + kStages * kStageBytes;
+  uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bar_base = base + S * C::kStageBytes;            // full[S], empty[S], then the abort flag
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(gen_base + S * C::kStageBytes + 8 * 2 * S);
+  float* merge = reinterpret_cast<float*>(gen_base + S * C::kStageBytes + 128);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qr = lane >> 2, qc = lane & 3;          // fragment row (and +8) / column pair
-
-  auto issue = [&](int t) {                          // thread 0 only
-    const int s = t % kStages;
-    const uint32_t bar = bar_base + 8u * s;
-    mbar_expect_tx(bar, kStageBytes);
-#pragma unroll
-    for (int h = 0; h < NH; ++h) {
-      tma_load_2d(base + s * kStageBytes + h * (kPos * 128), &tmK, h * 64, kv_row0 + t * kPos, bar);
-      tma_load_2d(base + s * kStageBytes + kTileBytes + h * (kPos * 128), &tmV, h * 64, kv_row0 + t * kPos, bar);
-    }
-  };
-  if (threadIdx.x == 0) {                            // the first K/V tiles are on their way before anything else is read
-    for (int s = 0; s < kStages; ++s) mbar_init(bar_base + 8u * s, 1);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), RW); }
+    *abort_flag = 0;
     mbar_fence_init();
-    for (int t = 0; t < min(n_tiles, kStages); ++t) issue(t);
   }
-
-  // the two rows this thread owns
-  int row[2], tok[2], head[2], ctx[2];
-  bool live[2];
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    row[i] = r0 + warp * 16 + qr + i * 8;
-    live[i] = row[i] < R;
-    const int rr = live[i] ? row[i] : r0;           // dead rows shadow the tile's first row (never stored)
-    tok[i] = tok0 + rr / G;
-    head[i] = kvh * G + rr % G;
-    ctx[i] = !live[i] ? 0 : (info.w >= 0 ? info.w : rr / G + 1);
-  }
-
-  // Q fragments (A operand): a0 = (qr, k0..1), a1 = (qr+8, k0..1), a2 = (qr, k8..9), a3 = (qr+8, k8..9)
-  uint32_t qf[KS][4];
-  {
-    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        qf[ks][i] = *reinterpret_cast<const uint32_t*>(qp + ks * 16);
-        qf[ks][i + 2] = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8);
-      }
-    }
-  }
-  __syncthreads();                                   // barrier initialisation visible to every waiter
+  __syncthreads();
 
   float o[NB][4];
-#pragma unroll
-  for (int j = 0; j < NB; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
-  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-  const float sc = a.scale * 1.4426950408889634f;   // work in base 2
-  bool aborted = false;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // m in the scaled log2 domain
+  int tok[2] = {0, 0}, head[2] = {0, 0};
+  bool live[2] = {false, false};
+  const int qr = lane >> 2, qc = lane & 3;          // fragment row (and +8) / column pair
+  const float sc = a.scale * 1.4426950408889634f;   // scores are kept in base 2
+  const int rw = warp % RW, g = warp / RW;          // consumer coordinates (the last warp is the producer)
 
-  for (int t = 0; t < n_tiles; ++t) {
-    const int s = t % kStages;
-    const int gave_up = mbar_wait(bar_base + 8u * s, (t / kStages) & 1) ? 0 : 1;
-    if (__syncthreads_or(gave_up)) { aborted = true; break; }   // uniform exit for the whole CTA
-    const uint32_t kt = base + s * kStageBytes, vt = kt + kTileBytes;
-
-    // ---- S = Q K^T (16 rows x 64 positions per warp)
-    float sacc[8][4];
+  if (warp == C::kConsumers) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int t = 0;
+      bool ok = true;
+      for (; t < n_tiles; ++t) {
+        const int s = t % S;
+        if (t >= S && !mbar_wait_or_abort(empty_bar(s), ((t / S) - 1) & 1, abort_flag)) { ok = false; break; }
+        mbar_expect_tx(full_bar(s), C::kStageBytes);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-#pragma unroll
-      for (int jp = 0; jp < 4; ++jp) {               // pairs of n-blocks (16 positions)
-        const int m = lane >> 3;                     // which 8x8 matrix this lane addresses
-        const int pos = jp * 16 + (m >> 1) * 8 + (lane & 7);
-        const int chunk = ks * 2 + (m & 1);
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(kv_addr<HD>(kt, pos, chunk), b0, b1, b2, b3);
-        mma_bf16(sacc[jp * 2], qf[ks], b0, b1);
-        mma_bf16(sacc[jp * 2 + 1], qf[ks], b2, b3);
+        for (int h = 0; h < NH; ++h) {
+          tma_load_2d(base + s * C::kStageBytes + h * (kPos * 128), &tmK, h * 64, kv_row0 + t * kPos, full_bar(s));
+          tma_load_2d(base + s * C::kStageBytes + C::kTileBytes + h * (kPos * 128), &tmV, h * 64, kv_row0 + t * kPos, full_bar(s));
+        }
+      }
+      if (!ok) {                                     // drain the copies still in flight before the CTA's smem goes away
+        *abort_flag = 1;
+        for (int j = max(0, t - S); j < t; ++j) mbar_wait(full_bar(j % S), (j / S) & 1);
       }
     }
-    // ---- scale, mask, online softmax (rows qr and qr+8; columns j*8 + qc*2 + {0,1})
-    const int p_base = t * kPos + qc * 2;
-    float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int i = e >> 1;
-        const int p = p_base + j * 8 + (e & 1);
-        const float v = (p < ctx[i]) ? sacc[j][e] * sc : -INFINITY;
-        sacc[j][e] = v;
-        mx[i] = fmaxf(mx[i], v);
-      }
-    }
-    float corr[2];
+  } else {
+    // ------------------------------------------------------------------ consumers
+    int ctx[2];
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
-      mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
-      mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
-      const float m_new = fmaxf(m_run[i], mx[i]);
-      corr[i] = (m_run[i] == -INFINITY) ? 0.f : exp2f(m_run[i] - m_new);
-      m_run[i] = m_new;
+      const int row = r0 + rw * 16 + qr + i * 8;
+      live[i] = row < R;
+      const int rr = live[i] ? row : r0;            // dead rows shadow the tile's first row (never stored)
+      tok[i] = tok0 + rr / G;
+      head[i] = kvh * G + rr % G;
+      ctx[i] = !live[i] ? 0 : (info.w >= 0 ? info.w : rr / G + 1);
     }
-    float rs[2] = {0.f, 0.f};
-    uint32_t pf[4][4];                               // P as A fragments for the 4 k-steps of P V
+    // Q fragments (A operand): a0 = (qr, k0..1), a1 = (qr+8, k0..1), a2 = (qr, k8..9), a3 = (qr+8, k8..9)
+    uint32_t qf[KS][4];
+    {
+      const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      float p0 = (m_run[0] == -INFINITY) ? 0.f : exp2f(sacc[j][0] - m_run[0]);
-      float p1 = (m_run[0] == -INFINITY) ? 0.f : exp2f(sacc[j][1] - m_run[0]);
-      float p2 = (m_run[1] == -INFINITY) ? 0.f : exp2f(sacc[j][2] - m_run[1]);
-      float p3 = (m_run[1] == -INFINITY) ? 0.f : exp2f(sacc[j][3] - m_run[1]);
-      rs[0] += p0 + p1; rs[1] += p2 + p3;
-      pf[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
-      pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
-    }
+      for (int i = 0; i < 2; ++i) {
+        const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
 #pragma unroll
-    for (int i = 0; i < 2; ++i) l_run[i] = l_run[i] * corr[i] + rs[i];
-#pragma unroll
-    for (int j = 0; j < NB; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[0]; o[j][2] *= corr[1]; o[j][3] *= corr[1]; }
-    // ---- O += P V
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks) {
-#pragma unroll
-      for (int np = 0; np < NB / 2; ++np) {          // pairs of n-blocks (16 dims)
-        const int m = lane >> 3;
-        const int pos = ks * 16 + (m & 1) * 8 + (lane & 7);
-        const int chunk = np * 2 + (m >> 1);
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(kv_addr<HD>(vt, pos, chunk), b0, b1, b2, b3);
-        mma_bf16(o[np * 2], pf[ks], b0, b1);
-        mma_bf16(o[np * 2 + 1], pf[ks], b2, b3);
+        for (int ks = 0; ks < KS; ++ks) {
+          qf[ks][i] = *reinterpret_cast<const uint32_t*>(qp + ks * 16);
+          qf[ks][i + 2] = *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8);
+        }
       }
     }
-    __syncthreads();                                 // everyone is done with stage s
-    if (threadIdx.x == 0 && t + kStages < n_tiles) issue(t + kStages);
-  }
-  if (aborted) {
-    if (threadIdx.x == 0) {
-      atomicOr(status, kStInternal);
-      // drain copies that may still be in flight (bounded) before the CTA's shared memory goes away
-      for (int s = 0; s < kStages; ++s) mbar_wait(bar_base + 8u * s, 0);
+#pragma unroll
+    for (int j = 0; j < NB; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+    const int ctx_min = __reduce_min_sync(0xffffffffu, min(ctx[0], ctx[1]));   // tiles below it need no masking
+
+    for (int t = g; t < n_tiles; t += KW) {
+      const int s = t % S;
+      const bool got = mbar_wait_or_abort(full_bar(s), (t / S) & 1, abort_flag);
+      if (!__all_sync(0xffffffffu, got)) { if (lane == 0) *abort_flag = 1; break; }
+      const uint32_t kt = base + s * C::kStageBytes, vt = kt + C::kTileBytes;
+
+      // ---- S = Q K^T (16 rows x 64 positions per warp)
+      float sacc[8][4];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f; }
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+        for (int jp = 0; jp < 4; ++jp) {             // pairs of n-blocks (16 positions)
+          const int m = lane >> 3;                   // which 8x8 matrix this lane addresses
+          const int pos = jp * 16 + (m >> 1) * 8 + (lane & 7);
+          const int chunk = ks * 2 + (m & 1);
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(kv_addr<HD>(kt, pos, chunk), b0, b1, b2, b3);
+          mma_bf16(sacc[jp * 2], qf[ks], b0, b1);
+          mma_bf16(sacc[jp * 2 + 1], qf[ks], b2, b3);
+        }
+      }
+      // ---- mask (only tiles that reach past some row's context), online softmax in base 2
+      // rows qr and qr+8; columns j*8 + qc*2 + {0,1}
+      if ((t + 1) * kPos > ctx_min) {
+        const int p_base = t * kPos + qc * 2;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (p_base + j * 8 + (e & 1) >= ctx[e >> 1]) sacc[j][e] = -INFINITY;
+        }
+      }
+      float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        mx[0] = fmaxf(mx[0], fmaxf(sacc[j][0], sacc[j][1]));
+        mx[1] = fmaxf(mx[1], fmaxf(sacc[j][2], sacc[j][3]));
+      }
+      float corr[2], neg_m[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
+        mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
+        const float m_new = fmaxf(m_run[i], mx[i] * sc);
+        const float m_safe = m_new == -INFINITY ? 0.f : m_new;     // a row that has seen nothing yet
+        corr[i] = ex2(m_run[i] - m_safe);
+        m_run[i] = m_new;
+        neg_m[i] = -m_safe;
+      }
+      float rs[2] = {0.f, 0.f};
+      uint32_t pf[4][4];                             // P as A fragments for the 4 k-steps of P V
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float p0 = ex2(fmaf(sacc[j][0], sc, neg_m[0])), p1 = ex2(fmaf(sacc[j][1], sc, neg_m[0]));
+        const float p2 = ex2(fmaf(sacc[j][2], sc, neg_m[1])), p3 = ex2(fmaf(sacc[j][3], sc, neg_m[1]));
+        rs[0] += p0 + p1; rs[1] += p2 + p3;
+        pf[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
+        pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+      }
+#pragma unroll
+      for (int i = 0; i < 2; ++i) l_run[i] = l_run[i] * corr[i] + rs[i];
+#pragma unroll
+      for (int j = 0; j < NB; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[0]; o[j][2] *= corr[1]; o[j][3] *= corr[1]; }
+      // ---- O += P V
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+        for (int np = 0; np < NB / 2; ++np) {        // pairs of n-blocks (16 dims)
+          const int m = lane >> 3;
+          const int pos = ks * 16 + (m & 1) * 8 + (lane & 7);
+          const int chunk = np * 2 + (m >> 1);
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(kv_addr<HD>(vt, pos, chunk), b0, b1, b2, b3);
+          mma_bf16(o[np * 2], pf[ks], b0, b1);
+          mma_bf16(o[np * 2 + 1], pf[ks], b2, b3);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar(s));      // this warp is done with slot s
     }
+    if (KW > 1 && g > 0) {                           // hand the partial softmax state to warp group 0
+      float* dst = merge + ((size_t)((g - 1) * RW + rw) * C::kMergeFloats) * 32 + lane;
+#pragma unroll
+      for (int j = 0; j < NB; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dst[(j * 4 + e) * 32] = o[j][e];
+      dst[(NB * 4 + 0) * 32] = m_run[0]; dst[(NB * 4 + 1) * 32] = m_run[1];
+      dst[(NB * 4 + 2) * 32] = l_run[0]; dst[(NB * 4 + 3) * 32] = l_run[1];
+    }
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(status, kStInternal);
     return;
+  }
+  if (warp >= RW) return;                            // the rest is warp group 0's
+
+  if (KW > 1) {
+#pragma unroll 1
+    for (int og = 1; og < KW; ++og) {
+      const float* src = merge + ((size_t)((og - 1) * RW + rw) * C::kMergeFloats) * 32 + lane;
+      const float m_o[2] = {src[(NB * 4 + 0) * 32], src[(NB * 4 + 1) * 32]};
+      const float l_o[2] = {src[(NB * 4 + 2) * 32], src[(NB * 4 + 3) * 32]};
+      float c_s[2], c_o[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const float m_new = fmaxf(m_run[i], m_o[i]);
+        const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+        c_s[i] = ex2(m_run[i] - m_safe); c_o[i] = ex2(m_o[i] - m_safe);
+        l_run[i] = l_run[i] * c_s[i] + l_o[i] * c_o[i];
+        m_run[i] = m_new;
+      }
+#pragma unroll
+      for (int j = 0; j < NB; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[j][e] = o[j][e] * c_s[e >> 1] + src[(j * 4 + e) * 32] * c_o[e >> 1];
+    }
   }
 
   // ---- the token's own extra KV rows (drafted codes of its tuple)
@@ -308,17 +377,17 @@ __global__ void __launch_bounds__(kThreads, 3) attn_tc_kernel(const __grid_const
   }
 }
 
-template <int HD>
+template <int HD, int RW, int KW>
 void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cudaStream_t st) {
-  constexpr int smem = kStages * 2 * kPos * HD * 2 + 1024 + 64;
+  using C = AttnCfg<HD, RW, KW>;
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(attn_tc_kernel<HD, RW, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     configured = true;
   }
   const int G = a.Hq / a.Hkv;
-  dim3 grid((a.max_tokens_per_row * G + kRows - 1) / kRows, a.Hkv, a.n_rows);
-  attn_tc_kernel<HD><<<grid, kThreads, smem, st>>>(*tk, *tv, a, a.status);
+  dim3 grid((a.max_tokens_per_row * G + 16 * RW - 1) / (16 * RW), a.Hkv, a.n_rows);
+  attn_tc_kernel<HD, RW, KW><<<grid, C::kThreads, C::kSmemBytes, st>>>(*tk, *tv, a, a.status);
 }
 
 }  // namespace
@@ -338,8 +407,10 @@ void launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   const CUtensorMap* tv = tma_map_bf16(a.v_ctx, rows, a.hd, a.hd, kPos);
   if (!tk || !tv) { launch_attention_simt(a, true, st); return; }
   LaunchScope ls(kcAttention, st);
-  if (a.hd == 64) launch<64>(tk, tv, a, st);
-  else launch<128>(tk, tv, a, st);
+  // few query rows per (request, KV head): 16-row CTAs whose warps split the KV tiles; else 64-row CTAs
+  const bool few = (long long)a.max_tokens_per_row * (a.Hq / a.Hkv) <= 32;
+  if (a.hd == 64) { if (few) launch<64, 1, 4>(tk, tv, a, st); else launch<64, 4, 1>(tk, tv, a, st); }
+  else { if (few) launch<128, 1, 4>(tk, tv, a, st); else launch<128, 4, 1>(tk, tv, a, st); }
 }
 
 }  // namespace nz
