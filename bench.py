@@ -137,6 +137,9 @@ def main():
     ap.add_argument("--workload", default="small")
     ap.add_argument("--mode", type=int, default=1, help="0 draft-only, 1 verified (default), 2 plain autoregressive")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--drafts", default="natural", choices=["natural", "perfect"],
+                    help="mode 1 only: 'natural' = the (random-init) draft head's own drafts; 'perfect' = the true top-k "
+                         "tuples injected as round-1 drafts (best case: one round, everything accepted)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
     args = ap.parse_args()
@@ -155,7 +158,8 @@ def main():
                           f"batch {w.batch} x beam {w.beam}, seed {w.seed}",
               "mode": {0: "draft-only (Algorithm 3)", 1: "verified (Algorithm 2)", 2: "autoregressive (Algorithm 1)"}[args.mode],
               "batch": w.batch, "beam": w.beam, "l2": "flushed between steps (256 MB write, outside the timed events)",
-              "drafts": "natural (random-init draft head)"}
+              "drafts": "natural (random-init draft head)" if args.drafts == "natural" or args.mode != 1 else
+                        "perfect (the true top-k tuples injected as round-1 drafts)"}
 
     # ------------------------------------------------------------------ reference arm: the oracle on host cores
     if args.impl == "reference":
@@ -218,7 +222,14 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    inject = None
+    if args.drafts == "perfect" and args.mode == 1:
+        ar = eng.decode(w.beam, mode=2)
+        inject = (ar["codes"].clone().clamp_(min=0), ar["count"].clone())
+
     def step():
+        if inject is not None:
+            return eng.decode_with_drafts(w.beam, inject[0], inject[1], out=out)
         return eng.decode(w.beam, mode=args.mode, out=out)
 
     for _ in range(max(args.warmup, 3)):

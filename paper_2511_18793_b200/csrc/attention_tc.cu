@@ -128,7 +128,7 @@ __device__ __forceinline__ void fold_extra_rows(const AttnArgs& a, const int* to
 
 template <int HD, int RW, int KW>
 struct AttnCfg {
-  static constexpr int kStages = KW == 1 ? 3 : 4;                 // a multiple of KW: slot s always serves warp group s % KW
+  static constexpr int kStages = KW == 1 ? 3 : KW;                // a multiple of KW: slot s always serves warp group s % KW
   static constexpr int kConsumers = RW * KW;
   static constexpr int kThreads = (kConsumers + 1) * 32;          // + the producer warp
   static constexpr int kTileBytes = kPos * HD * 2;                // one K (or V) tile
@@ -409,8 +409,8 @@ void launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   LaunchScope ls(kcAttention, st);
   // few query rows per (request, KV head): 16-row CTAs whose warps split the KV tiles; else 64-row CTAs
   const bool few = (long long)a.max_tokens_per_row * (a.Hq / a.Hkv) <= 32;
-  if (a.hd == 64) { if (few) launch<64, 1, 4>(tk, tv, a, st); else launch<64, 4, 1>(tk, tv, a, st); }
-  else { if (few) launch<128, 1, 4>(tk, tv, a, st); else launch<128, 4, 1>(tk, tv, a, st); }
+  if (a.hd == 64) { if (few) launch<64, 1, 2>(tk, tv, a, st); else launch<64, 4, 1>(tk, tv, a, st); }
+  else { if (few) launch<128, 1, 2>(tk, tv, a, st); else launch<128, 4, 1>(tk, tv, a, st); }
 }
 
 }  // namespace nz
