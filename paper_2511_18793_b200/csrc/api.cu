@@ -31,7 +31,6 @@ void profile_add(const long long* delta);
 void profile_read(nezha_profile* out);
 bool gemm_tc_supported(const GemmArgs& a);
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
-int gemm_tc_norm_parts(int M, int N);
 bool attention_tc_supported(const AttnArgs& a);
 void launch_attention_tc(const AttnArgs& a, cudaStream_t st);
 }  // namespace nz
@@ -84,6 +83,8 @@ struct nezha_ctx {
   struct Segment { int seen; cudaGraphExec_t exec; long long launches[kcCount]; };
   std::map<std::array<uintptr_t, 16>, Segment> segments;
   bool use_graphs;
+  int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
+  int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
   int state;                // 0 created, 1 hash set built, 2 prefilled
   int batch;                // prefilled batch
   std::string err;
@@ -210,8 +211,8 @@ size_t carve(nezha_ctx* c) {
   c->fused = c->bf16 && (c->hd == 64 || c->hd == 128) && c->d % 64 == 0 && c->F % 64 == 0;
   c->ss_a = c->ss_b = c->ss_e = nullptr;
   if (c->fused) {
-    c->ss_a = cv.take<float>((size_t)(c->d / 16) * c->Ms);      // up to two partial sums per 32-column tile
-    c->ss_b = cv.take<float>((size_t)(c->d / 16) * c->Ms);
+    c->ss_a = cv.take<float>((size_t)(c->d / 32) * c->Ms);      // one partial sum per 32 columns
+    c->ss_b = cv.take<float>((size_t)(c->d / 32) * c->Ms);
     c->ss_e = cv.take<float>((size_t)c->Ms);
   }
   // engine state
@@ -244,15 +245,16 @@ void gemm(nezha_ctx* c, const void* A, long long lda, const void* W, long long l
 }
 
 // A projection of the fused tensor-core path.  ss_in / parts: partial sums of squares of the A operand's rows (its
-// RMSNorm scale is applied in the epilogue), or null.  Returns the number of column tiles (= partial sums written
-// by a kEpiAddNorm epilogue) of such a launch.
+// RMSNorm scale is applied in the epilogue), or null.  Returns the number of partial sums per row a kEpiAddNorm
+// epilogue of this launch writes (one per 32 columns).
 int gemm_fused(nezha_ctx* c, const void* A, long long lda, const void* W, void* C, long long ldc, long long M,
                const int* M_dev, int N, int K, int epi, const float* ss_in, int ss_parts, const GemmFuse* extra) {
   GemmArgs a{A, lda, W, (long long)K, C, ldc, (int)M, M_dev, N, K, epi, nullptr, c->es.status};
   if (extra) a.f = *extra;
   a.f.ss_in = ss_in; a.f.ss_in_parts = ss_parts; a.f.ss_ld = c->Ms; a.f.inv_dim = 1.f / (float)c->d; a.f.eps = c->cfg.rms_eps;
+  a.M_expected = c->m_expected;
   launch_gemm_tc(a, c->st);
-  return gemm_tc_norm_parts((int)M, N);
+  return N / 32;
 }
 
 // The layers of the primary model on the fused path.  On entry resid holds the embeddings, xn = embedding * gain of
@@ -475,6 +477,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
     k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
     k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams; k[14] = (uintptr_t)tr.beam_scores;
+    k[15] = (uintptr_t)c->m_seen[segment];           // the expected token count shapes the tiling of the round's GEMMs
     return k;
   };
   nezha_status rs = run_segment(c, key_of(0), [&] {
@@ -515,6 +518,8 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     return ps;
   }
   for (int round = 1; round <= R; ++round) {
+    // drafts are mostly rejected or mostly accepted in a steady workload, so the round's token count repeats: tile for it
+    c->m_expected = c->m_seen[round];
     rs = run_segment(c, key_of(round), [&] {
       cudaMemsetAsync(e.counters, 0, 8 * sizeof(int), c->st);
       if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
@@ -538,9 +543,11 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
       launch_round_end(e, batch, K, round, tr, c->st);
       cudaMemcpyAsync(c->host_counters, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st);
     });
-    if (rs != NEZHA_OK) return rs;
+    if (rs != NEZHA_OK) { c->m_expected = 0; return rs; }
     NZ_CUDA(c, cudaStreamSynchronize(c->st));
     NZ_CUDA(c, cudaGetLastError());
+    c->m_expected = 0;
+    c->m_seen[round] = (c->host_counters[1] + 127) / 128 * 128;
     sd.rounds = round;
     sd.primary_tokens += c->host_counters[1];
     sd.accepted_levels += c->host_counters[2];
@@ -581,6 +588,8 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   c->st = (cudaStream_t)cuda_stream; c->arena = nullptr; c->state = 0; c->batch = 0;
   // the legacy default stream cannot be captured; NEZHA_NO_GRAPHS=1 keeps every launch eager
   c->use_graphs = cuda_stream != nullptr && !getenv("NEZHA_NO_GRAPHS");
+  c->m_expected = 0;
+  for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;

@@ -135,16 +135,16 @@ enum GemmEpilogue : int {
   kEpiBiasTanhF32 = 3,  // C (float) = tanh(acc + bias[n])     (Eq. 3)
   // ---- fused epilogues of the tensor-core kernel only -------------------------------------------------------
   kEpiSwiGLU = 4,       // weight rows interleaved [16 gate, 16 up]: C (act)[m, n/2 ..] = silu(gate) * up
-  kEpiAddNorm = 5,      // C (float) += acc; xg (act)[m, n] = C * gain[n]; ss_out[tile_n][m] = sum_n C^2 (this tile)
+  kEpiAddNorm = 5,      // C (float) += acc; xg (act)[m, n] = C * gain[n]; ss_out[n / 32][m] = sum of C^2 over the 32 columns
   kEpiRopeKV = 6        // fused QKV projection: rotary embedding on q and k, q to C, k and v to the KV cache
 };
 
 // Extras of the fused epilogues.  RMSNorm is split around the GEMMs: the producer of the residual stream
-// (kEpiAddNorm) leaves x * gain as the next GEMM's A operand and per-tile partial sums of x^2; the consumer GEMM
+// (kEpiAddNorm) leaves x * gain as the next GEMM's A operand and partial sums of x^2 per 32 columns; the consumer GEMM
 // multiplies its accumulator rows by rsqrt(mean(x^2) + eps), summing the partials in a fixed order.
 struct GemmFuse {
   const float* ss_in; int ss_in_parts; long long ss_ld; float inv_dim, eps;   // row scale of the A operand (or null)
-  float* ss_out;                     // [N / tile_n][ss_ld]
+  float* ss_out;                     // [N / 32][ss_ld]
   void* xg; const void* gain;        // kEpiAddNorm: next A operand [M, N] (activation type) and its norm gain [N]
   // kEpiRopeKV: weight rows of every q / k head permuted so that each 32-column group holds 16 rotary pairs
   const int* tok_pos; const long long* kv_dst; long long kv_head_stride;
@@ -163,6 +163,7 @@ struct GemmArgs {
   const float* bias;
   int* status;           // device status word (bounded waits report here)
   GemmFuse f;            // zero-initialised unless a fused epilogue is asked for
+  int M_expected;        // 0, or the row count the caller expects on the device (<= M): only shapes the tiling
 };
 
 void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);

@@ -26,7 +26,8 @@ constexpr int kTransposeBytes = kEpiWarps * 32 * 32 * 4;   // per epilogue warp:
 template <int BN> struct Cfg {
   static constexpr int kTileBytesB = BN * BK * 2;
   static constexpr int kStageBytes = kTileBytesA + kTileBytesB;
-  static constexpr int kStages = BN >= 128 ? 4 : 6;
+  // as many stages as fit beside the transpose tiles: short-M launches are bound by bytes in flight per CTA
+  static constexpr int kStages = BN == 256 ? 4 : BN == 128 ? 6 : BN == 64 ? 8 : 9;
   static constexpr int kSmemBytes =
       kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTransposeBytes;
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;       // two accumulators; a power of two >= 32
@@ -308,7 +309,6 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
       if (!ok) break;
       tc_fence_after();
       const int rows_here = min(32, M - (m0 + q * 32));          // rows of this quarter that exist (may be <= 0)
-      float ssq = 0.f;
 #pragma unroll 1
       for (int c = half; c < BN / 32; c += 2) {
         const int n_chunk = n0 + c * 32;
@@ -344,11 +344,14 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
         }
         __syncwarp();
         if (EPI == kEpiAddNorm && lane < rows_here) {
+          // one partial sum of squares per 32-column group, added up in column order: the same bits whatever the tile width
+          float ssq = 0.f;
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float4 t = stg4[lane * 8 + (j ^ (lane & 7))];
-            ssq += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+            ssq += t.x * t.x; ssq += t.y * t.y; ssq += t.z * t.z; ssq += t.w * t.w;
           }
+          a.f.ss_out[(long long)(n_chunk >> 5) * a.f.ss_ld + row] = ssq;
         }
         __syncwarp();
       }
@@ -356,10 +359,6 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty(b));
-      if (EPI == kEpiAddNorm && row < M) {
-        // the two warps of a quarter each saw half of the tile's columns: two partial sums per tile
-        a.f.ss_out[(long long)(tn * 2 + half) * a.f.ss_ld + row] = ssq;
-      }
     }
     if (!ok && lane == 0) *abort_flag = 1;
   }
@@ -438,12 +437,6 @@ int gemm_tc_tile_n(int M, int N) {
   return best_bn;
 }
 
-// Partial sums of squares a kEpiAddNorm launch writes per row (two per column tile).
-int gemm_tc_norm_parts(int M, int N) {
-  const int bn = gemm_tc_tile_n(M, N);
-  return 2 * ((N + bn - 1) / bn);
-}
-
 bool gemm_tc_supported(const GemmArgs& a) {
   if (!a.status || !tma_encode_fn()) return false;
   if (a.K % BK || a.N % 32 || a.M <= 0) return false;
@@ -455,7 +448,7 @@ bool gemm_tc_supported(const GemmArgs& a) {
 
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
   LaunchScope ls(kcGemm, st);
-  switch (gemm_tc_tile_n(a.M, a.N)) {
+  switch (gemm_tc_tile_n(a.M_expected > 0 && a.M_expected < a.M ? a.M_expected : a.M, a.N)) {
     case 256: launch_bn<256>(a, st); break;
     case 128: launch_bn<128>(a, st); break;
     case 64: launch_bn<64>(a, st); break;
