@@ -521,7 +521,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     // drafts are mostly rejected or mostly accepted in a steady workload, so the round's token count repeats: tile for it
     c->m_expected = c->m_seen[round];
     rs = run_segment(c, key_of(round), [&] {
-      cudaMemsetAsync(e.counters, 0, 8 * sizeof(int), c->st);
+      launch_fill_i32(e.counters, 8, 0, c->st);
       if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
       else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
       else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, true);

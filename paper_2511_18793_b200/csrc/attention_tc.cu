@@ -149,6 +149,8 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
   constexpr int NB = HD / 8;                        // n-blocks of the output
   constexpr int kRows = 16 * RW;
 
+  pdl_wait();                                       // before the first global read and before any exit
+  pdl_launch();
   const int req_local = blockIdx.z, kvh = blockIdx.y, tile = blockIdx.x;
   const int G = a.Hq / a.Hkv;
   const int4 info = a.req_info[req_local];          // {first token, token count, cache row, context length or -1}
@@ -387,7 +389,7 @@ void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cud
   }
   const int G = a.Hq / a.Hkv;
   dim3 grid((a.max_tokens_per_row * G + 16 * RW - 1) / (16 * RW), a.Hkv, a.n_rows);
-  attn_tc_kernel<HD, RW, KW><<<grid, C::kThreads, C::kSmemBytes, st>>>(*tk, *tv, a, a.status);
+  launch_pdl(attn_tc_kernel<HD, RW, KW>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *tk, *tv, a, a.status);
 }
 
 }  // namespace

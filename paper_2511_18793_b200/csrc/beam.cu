@@ -29,6 +29,8 @@ __device__ __forceinline__ bool cand_better(float s, int r, int t, float s2, int
 
 template <int VPL>
 __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   if (a.gate_mode == 1 && a.gate[b] != a.gate_value) return;
   if (a.gate_mode == 2 && !(a.gate[b] < a.gate_value)) return;
@@ -212,10 +214,10 @@ void launch_select(const SelectArgs& a, cudaStream_t st) {
   if (a.batch <= 0) return;
   const size_t smem = select_smem_bytes(a.in_stride, a.K);
   LaunchScope ls(kcSelect, st);
-  if (a.T <= 32) select_kernel<1><<<a.batch, 256, smem, st>>>(a);
-  else if (a.T <= 256) select_kernel<8><<<a.batch, 256, smem, st>>>(a);
-  else if (a.T <= 512) select_kernel<16><<<a.batch, 256, smem, st>>>(a);
-  else select_kernel<32><<<a.batch, 256, smem, st>>>(a);
+  if (a.T <= 32) launch_pdl(select_kernel<1>, dim3(a.batch), dim3(256), smem, st, a);
+  else if (a.T <= 256) launch_pdl(select_kernel<8>, dim3(a.batch), dim3(256), smem, st, a);
+  else if (a.T <= 512) launch_pdl(select_kernel<16>, dim3(a.batch), dim3(256), smem, st, a);
+  else launch_pdl(select_kernel<32>, dim3(a.batch), dim3(256), smem, st, a);
 }
 
 // ====================================================================================================
@@ -224,16 +226,22 @@ void launch_select(const SelectArgs& a, cudaStream_t st) {
 namespace {
 
 __global__ void fill_i32_kernel(int* p, long long n, int v) {
+  pdl_wait();
+  pdl_launch();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
     p[i] = v;
 }
 __global__ void fill_f32_kernel(float* p, long long n, float v) {
+  pdl_wait();
+  pdl_launch();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
     p[i] = v;
 }
 
 // B_0 = { empty beam, score 0 } for every request; nothing settled.
 __global__ void init_decode_kernel(EngineState e, int batch) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b == 0)
     for (int i = 0; i < 8; ++i) e.counters[i] = 0;
@@ -251,6 +259,8 @@ __global__ void init_decode_kernel(EngineState e, int batch) {
 // Start of a round's drafting (Algorithm 2's drafting step): the draft head continues from the true beams B_m, or from
 // the empty beam in the first round (Algorithm 3's initialisation).
 __global__ void draft_init_kernel(EngineState e, int batch, int from_scratch) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   if (b >= batch) return;
   const int m = e.row_m[b];
@@ -269,6 +279,8 @@ __global__ void draft_init_kernel(EngineState e, int batch, int from_scratch) {
 
 // Caller-supplied drafts for the round (or none: n_draft == nullptr and drafts == nullptr -> zero drafts).
 __global__ void draft_set_kernel(EngineState e, int batch, int K, const int* drafts, const int* n_draft) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   if (b >= batch) return;
   const int cnt = (drafts && e.row_m[b] < e.L) ? max(0, min(n_draft[b], K)) : 0;
@@ -289,6 +301,8 @@ __global__ void draft_set_kernel(EngineState e, int batch, int K, const int* dra
 // Eq. 2 input: x = h_l + s_l for every (request, beam); s_1 = h_0 (Eq. 1).
 template <typename T>
 __global__ void draft_x_kernel(EngineState e, int batch, int l, T* x) {
+  pdl_wait();
+  pdl_launch();
   const int bk = blockIdx.x;                       // b * Kmax + k
   const int b = bk / e.Kmax;
   if (b >= batch) return;
@@ -303,6 +317,8 @@ __global__ void draft_x_kernel(EngineState e, int batch, int l, T* x) {
 //   requests drafting (d_m < l): survivor k of level l, its parent's state, the code just chosen.
 template <typename T>
 __global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* embed, T* A) {
+  pdl_wait();
+  pdl_launch();
   const int bk = blockIdx.x;
   const int b = bk / e.Kmax, k = bk - b * e.Kmax;
   if (b >= batch) return;
@@ -337,6 +353,8 @@ __global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* em
 // of levels m+1..L-1 of every alive draft (slot = draft index).  Tokens of a request are contiguous; requests
 // are laid out in order (each block sums the counts of the requests before it).
 __global__ void nodes_count_kernel(EngineState e, int batch) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   const int m = e.row_m[b];
   const int L = e.L;
@@ -373,6 +391,8 @@ __global__ void nodes_count_kernel(EngineState e, int batch) {
 }
 
 __global__ void nodes_fill_kernel(EngineState e, int batch) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   const int L = e.L, Kmax = e.Kmax;
   __shared__ int s_off, s_alive_rank[128], s_n_alive;
@@ -440,6 +460,8 @@ __global__ void nodes_fill_kernel(EngineState e, int batch) {
 
 // Teacher-forced nodes: beams given by the caller, every beam processes all of its `level` codes.
 __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams, int level, const int* prefixes) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   const int L = e.L, Kmax = e.Kmax;
   const int per_row = n_beams * level;
@@ -479,6 +501,8 @@ __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams
 //                the (n+1)-prefix of a draft, its hidden state is already in the pass and selection goes on;
 //                else level n+1 is the rejection level and the request waits for the next round.
 __global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   if (e.row_cur[b] != n) return;
   const int L = e.L, Kmax = e.Kmax;
@@ -535,6 +559,8 @@ __global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_
 // End of a round: accepted length of every draft = the largest i <= (level reached) with D[k][0..i) in B_i;
 // trace outputs; counters for the host (unfinished requests, primary tokens, accepted levels).
 __global__ void round_end_kernel(EngineState e, int batch, int K, int round, nezha_trace tr, int m_before_unused) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   const int L = e.L, Kmax = e.Kmax;
   const int took_part = e.row_tok_count[b] > 0;
@@ -580,6 +606,8 @@ __global__ void round_end_kernel(EngineState e, int batch, int K, int round, nez
 
 __global__ void write_out_kernel(const int* codes, const float* score, const int* count, int stride, int L, int K,
                                  int* out_codes, float* out_score, int* out_count) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   const int cnt = min(count[b], K);
   for (int k = threadIdx.x; k < K; k += blockDim.x) {
@@ -594,6 +622,8 @@ __global__ void write_out_kernel(const int* codes, const float* score, const int
 // row = row_index ? row_index[b*idx_stride + r] : b*row_mul + r*beam_mul
 __global__ void copy_logits_kernel(const float* src, long long row_stride, int col_off, const int* row_index, int row_mul,
                                    int beam_mul, int n_beams, int idx_stride, int T, float* dst) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x / n_beams, r = blockIdx.x % n_beams;
   const long long row = row_index ? row_index[(long long)b * idx_stride + r] : (long long)b * row_mul + (long long)r * beam_mul;
   if (row < 0) return;
@@ -602,6 +632,8 @@ __global__ void copy_logits_kernel(const float* src, long long row_stride, int c
 }
 
 __global__ void trace_beams_kernel(EngineState e, int batch, int K, nezha_trace tr) {
+  pdl_wait();
+  pdl_launch();
   const int b = blockIdx.x;
   const int L = e.L;
   for (int n = 1; n <= L; ++n) {
@@ -621,66 +653,66 @@ __global__ void trace_beams_kernel(EngineState e, int batch, int K, nezha_trace 
 void launch_fill_i32(int* p, long long n, int v, cudaStream_t st) {
   if (n <= 0) return;
   LaunchScope ls(kcMisc, st);
-  fill_i32_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, st>>>(p, n, v);
+  launch_pdl(fill_i32_kernel, dim3((unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184)), dim3(256), 0, st, p, n, v);
 }
 void launch_fill_f32(float* p, long long n, float v, cudaStream_t st) {
   if (n <= 0) return;
   LaunchScope ls(kcMisc, st);
-  fill_f32_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, st>>>(p, n, v);
+  launch_pdl(fill_f32_kernel, dim3((unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184)), dim3(256), 0, st, p, n, v);
 }
 void launch_init_decode(const EngineState& e, int batch, cudaStream_t st) {
   LaunchScope ls(kcMisc, st);
-  init_decode_kernel<<<(batch + 127) / 128, 128, 0, st>>>(e, batch);
+  launch_pdl(init_decode_kernel, dim3((batch + 127) / 128), dim3(128), 0, st, e, batch);
 }
 void launch_draft_init(const EngineState& e, int batch, int from_scratch, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
-  draft_init_kernel<<<batch, 64, 0, st>>>(e, batch, from_scratch);
+  launch_pdl(draft_init_kernel, dim3(batch), dim3(64), 0, st, e, batch, from_scratch);
 }
 void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
-  draft_set_kernel<<<batch, 64, 0, st>>>(e, batch, K, drafts, n_draft);
+  launch_pdl(draft_set_kernel, dim3(batch), dim3(64), 0, st, e, batch, K, drafts, n_draft);
 }
 void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
-  if (bf16) draft_x_kernel<__nv_bfloat16><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (__nv_bfloat16*)x);
-  else draft_x_kernel<float><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (float*)x);
+  if (bf16) launch_pdl(draft_x_kernel<__nv_bfloat16>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (__nv_bfloat16*)x);
+  else launch_pdl(draft_x_kernel<float>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (float*)x);
 }
 void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
                          cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
   if (bf16)
-    trans_gather_kernel<__nv_bfloat16><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (const __nv_bfloat16*)embed,
+    launch_pdl(trans_gather_kernel<__nv_bfloat16>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const __nv_bfloat16*)embed,
                                                                       (__nv_bfloat16*)A);
-  else trans_gather_kernel<float><<<batch * e.Kmax, 128, 0, st>>>(e, batch, l, (const float*)embed, (float*)A);
+  else launch_pdl(trans_gather_kernel<float>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const float*)embed, (float*)A);
 }
 void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st) {
   LaunchScope ls(kcNodes, st, 2);
-  nodes_count_kernel<<<batch, 64, 0, st>>>(e, batch);
-  nodes_fill_kernel<<<batch, 128, 0, st>>>(e, batch);
+  launch_pdl(nodes_count_kernel, dim3(batch), dim3(64), 0, st, e, batch);
+  launch_pdl(nodes_fill_kernel, dim3(batch), dim3(128), 0, st, e, batch);
 }
 void launch_nodes_from_prefixes(const EngineState& e, int batch, int n_beams, int level, const int* prefixes,
                                 cudaStream_t st) {
   LaunchScope ls(kcNodes, st);
-  nodes_from_prefixes_kernel<<<batch, 128, 0, st>>>(e, batch, n_beams, level, prefixes);
+  launch_pdl(nodes_from_prefixes_kernel, dim3(batch), dim3(128), 0, st, e, batch, n_beams, level, prefixes);
 }
 void launch_advance(const EngineState& e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count,
                     cudaStream_t st) {
   LaunchScope ls(kcAccept, st);
-  advance_kernel<<<batch, 64, 0, st>>>(e, batch, n, K, out_codes, out_score, out_count);
+  launch_pdl(advance_kernel, dim3(batch), dim3(64), 0, st, e, batch, n, K, out_codes, out_score, out_count);
 }
 void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, cudaStream_t st) {
   LaunchScope ls(kcAccept, st);
-  round_end_kernel<<<batch, 64, 0, st>>>(e, batch, K, round, tr, 0);
+  launch_pdl(round_end_kernel, dim3(batch), dim3(64), 0, st, e, batch, K, round, tr, 0);
 }
 void launch_write_out(const int* codes, const float* score, const int* count, int stride, int L, int batch, int K,
                       int* out_codes, float* out_score, int* out_count, cudaStream_t st) {
   LaunchScope ls(kcMisc, st);
-  write_out_kernel<<<batch, 64, 0, st>>>(codes, score, count, stride, L, K, out_codes, out_score, out_count);
+  launch_pdl(write_out_kernel, dim3(batch), dim3(64), 0, st, codes, score, count, stride, L, K, out_codes, out_score, out_count);
 }
 void launch_copy_logits(const float* src, long long row_stride, int col_off, const int* row_index, int row_mul,
                         int beam_mul, int batch, int n_beams, int idx_stride, int T, float* dst, cudaStream_t st) {
   LaunchScope ls(kcMisc, st);
-  copy_logits_kernel<<<batch * n_beams, 128, 0, st>>>(src, row_stride, col_off, row_index, row_mul, beam_mul, n_beams,
+  launch_pdl(copy_logits_kernel, dim3(batch * n_beams), dim3(128), 0, st, src, row_stride, col_off, row_index, row_mul, beam_mul, n_beams,
                                                       idx_stride, T, dst);
 }
 
@@ -688,6 +720,8 @@ void launch_copy_logits(const float* src, long long row_stride, int col_off, con
 // S_call positions (padding sits after the real tokens, so causal attention never shows it to them).
 __global__ void prefill_tokens_kernel(EngineState e, const int* hist, const int* n_hist, int b0, int rows, int max_n,
                                       int S_call, int S_cap, int* h_rows) {
+  pdl_wait();
+  pdl_launch();
   const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (idx >= (long long)rows * S_call) return;
   const int lb = (int)(idx / S_call), p = (int)(idx % S_call), b = b0 + lb;
@@ -718,11 +752,11 @@ void launch_prefill_tokens(const EngineState& e, const int* hist, const int* n_h
                            int S_call, int S_cap, int* h_rows, cudaStream_t st) {
   const long long n = (long long)rows * S_call;
   LaunchScope ls(kcNodes, st);
-  prefill_tokens_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(e, hist, n_hist, b0, rows, max_n, S_call, S_cap, h_rows);
+  launch_pdl(prefill_tokens_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, e, hist, n_hist, b0, rows, max_n, S_call, S_cap, h_rows);
 }
 void launch_trace_beams(const EngineState& e, int batch, int K, const nezha_trace& tr, cudaStream_t st) {
   LaunchScope ls(kcMisc, st);
-  trace_beams_kernel<<<batch, 64, 0, st>>>(e, batch, K, tr);
+  launch_pdl(trace_beams_kernel, dim3(batch), dim3(64), 0, st, e, batch, K, tr);
 }
 
 }  // namespace nz

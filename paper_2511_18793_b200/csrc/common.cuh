@@ -32,6 +32,30 @@ struct LaunchScope {
 };
 
 // --------------------------------------------------------------------------------------------------
+// programmatic dependent launch: the kernels of the decode path are launched so that a kernel may be scheduled, and
+// run the part of its prologue that touches no global memory, while its predecessor in the stream is still finishing
+// --------------------------------------------------------------------------------------------------
+// EVERY thread block of a kernel launched with launch_pdl must execute pdl_wait() before its first global memory
+// access and before it exits (a block that exits without waiting lets the grid "complete" while its predecessor is
+// still running, and the grid after it would then start too early).  pdl_wait() returns once the preceding grid has
+// completed and its writes are visible; pdl_launch() lets the following grid start being scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+bool pdl_enabled();     // false when NEZHA_NO_PDL is set: plain stream-ordered launches
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// --------------------------------------------------------------------------------------------------
 // small device helpers
 // --------------------------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -96,6 +96,8 @@ __global__ void embed_norm_kernel(const __nv_bfloat16* __restrict__ table, const
                                   const int* M_dev, int d, float* __restrict__ resid,
                                   const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xg,
                                   float* __restrict__ ss) {
+  pdl_wait();
+  pdl_launch();
   const int m = M_dev ? min(M, *M_dev) : M;
   const int i = blockIdx.x;
   if (i >= m) return;
@@ -137,7 +139,7 @@ void launch_embed_norm(const void* table, const int* tokens, int M, const int* M
                        const void* gain, void* xg, float* ss, cudaStream_t st) {
   if (M <= 0) return;
   LaunchScope ls(kcEmbed, st);
-  embed_norm_kernel<<<M, 128, 0, st>>>((const __nv_bfloat16*)table, tokens, M, M_dev, d, resid,
+  launch_pdl(embed_norm_kernel, dim3(M), dim3(128), 0, st, (const __nv_bfloat16*)table, tokens, M, M_dev, d, resid,
                                        (const __nv_bfloat16*)gain, (__nv_bfloat16*)xg, ss);
 }
 void launch_permute_rotary_rows(const void* src, void* dst, int rows, int hd, int cols, cudaStream_t st) {

@@ -204,11 +204,6 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
                                                            int* status) {
   using C = Cfg<BN>;
   constexpr int STAGES = C::kStages;
-  const int M = a.M_dev ? min(a.M, *a.M_dev) : a.M;
-  const int tiles_m = (M + BM - 1) / BM, tiles_n = (a.N + BN - 1) / BN;
-  const int n_tiles = tiles_m * tiles_n;
-  if ((int)blockIdx.x >= n_tiles) return;
-
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = base + STAGES * C::kStageBytes;
@@ -240,6 +235,12 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched no global memory; from here on the preceding kernel's results are needed
+  pdl_wait();
+  pdl_launch();
+  const int M = a.M_dev ? min(a.M, *a.M_dev) : a.M;
+  const int tiles_m = (M + BM - 1) / BM, tiles_n = (a.N + BN - 1) / BN;
+  const int n_tiles = tiles_m * tiles_n;     // a CTA without a tile falls through every role loop
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -401,7 +402,7 @@ void launch(const GemmArgs& a, cudaStream_t st) {
   }
   const long long tiles = (long long)((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  gemm_tc_kernel<BN, EPI><<<grid, kThreads, Cfg<BN>::kSmemBytes, st>>>(*ta, *tb, a, a.status);
+  launch_pdl(gemm_tc_kernel<BN, EPI>, dim3(grid), dim3(kThreads), Cfg<BN>::kSmemBytes, st, *ta, *tb, a, a.status);
 }
 
 template <int BN>

@@ -1,5 +1,7 @@
 // Launch counting and optional per-kernel-class CUDA-event timing.  Process-wide, not thread-safe: meant for
 // one benchmarking thread.
+#include <stdlib.h>
+
 #include <vector>
 
 #include "common.cuh"
@@ -31,6 +33,11 @@ LaunchScope::LaunchScope(int cls_, cudaStream_t st_, int n_launches) : cls(cls_)
 
 LaunchScope::~LaunchScope() {
   if (slot >= 0) cudaEventRecord(g_pairs[slot].b, st);
+}
+
+bool pdl_enabled() {
+  static const bool on = getenv("NEZHA_NO_PDL") == nullptr;
+  return on;
 }
 
 unsigned long long profile_total_launches() { return g_total; }
