@@ -28,6 +28,12 @@ METRIC, UNIT = "items_per_s_decoded", "items/s"
 # bumped whenever a kernel of the class changes in a way that can change its DRAM traffic: a traffic figure taken
 # from an older revision is reported as null
 KERNEL_REV = {"gemm": 3, "attention": 1}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the launches of the class in one decode step
+# (ncu, eager launches, L2 flushed before the step)
+NCU_TRAFFIC = {
+    "gemm@small": {"kernel_rev": 3, "dram_bytes_per_launch": 3.34e6, "source": "profiles/gemm_tc_kernel_ncu.md, section A"},
+    "attention@small": {"kernel_rev": 1, "dram_bytes_per_launch": 29.6e6, "source": "profiles/attn_tc_kernel_ncu.md"},
+}
 
 
 def load_peaks():
@@ -323,14 +329,12 @@ def main():
         roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
     else:
         roof.update(bound="latency", note="dominant class is neither GEMM nor attention")
-    # DRAM traffic of the dominant kernel from the committed ncu capture of that kernel (bytes per launch, scaled by
-    # the units processed where the capture ran a smaller case); null when no capture matches the current kernel
-    tpath = os.path.join(ROOT, "profiles", "ncu_traffic.json")
-    if os.path.exists(tpath):
-        rec = json.load(open(tpath)).get(f"{dom}@{w.name}")
-        if rec and rec.get("kernel_rev") == KERNEL_REV.get(dom):
-            roof["traffic"] = rec["dram_bytes_per_launch"]
-            roof["traffic_note"] = rec.get("note")
+    # DRAM traffic of the dominant kernel from the ncu capture of that kernel in this workload (bytes per launch);
+    # null when no capture matches the current kernel revision
+    rec = NCU_TRAFFIC.get(f"{dom}@{w.name}")
+    if rec and rec["kernel_rev"] == KERNEL_REV.get(dom):
+        roof["traffic"] = rec["dram_bytes_per_launch"]
+        roof["traffic_source"] = rec["source"]
     roof["classes"] = shares
     roof["attention_gbs"] = work["attention_bytes"] / (shares["attention"]["ms_per_step"] / 1e3) / 1e9 if "attention" in shares else None
     roof["gemm_tflops"] = work["gemm_flops"] / (shares["gemm"]["ms_per_step"] / 1e3) / 1e12 if "gemm" in shares else None
