@@ -158,7 +158,7 @@ enum GemmEpilogue : int {
   kEpiAddF32 = 2,       // C (float) += acc                    (residual stream)
   kEpiBiasTanhF32 = 3,  // C (float) = tanh(acc + bias[n])     (Eq. 3)
   // ---- fused epilogues of the tensor-core kernel only -------------------------------------------------------
-  kEpiSwiGLU = 4,       // weight rows interleaved [16 gate, 16 up]: C (act)[m, n/2 ..] = silu(gate) * up
+  kEpiSwiGLU = 4,       // weight rows interleaved (gate, gate, up, up per 4 columns): C (act)[m, n/2] = silu(gate) * up
   kEpiAddNorm = 5,      // C (float) += acc; xg (act)[m, n] = C * gain[n]; ss_out[n / 32][m] = sum of C^2 over the 32 columns
   kEpiRopeKV = 6        // fused QKV projection: rotary embedding on q and k, q to C, k and v to the KV cache
 };
@@ -170,7 +170,7 @@ struct GemmFuse {
   const float* ss_in; int ss_in_parts; long long ss_ld; float inv_dim, eps;   // row scale of the A operand (or null)
   float* ss_out;                     // [N / 32][ss_ld]
   void* xg; const void* gain;        // kEpiAddNorm: next A operand [M, N] (activation type) and its norm gain [N]
-  // kEpiRopeKV: weight rows of every q / k head permuted so that each 32-column group holds 16 rotary pairs
+  // kEpiRopeKV: weight rows of every q / k head permuted so that every 4 consecutive columns hold two rotary pairs
   const int* tok_pos; const long long* kv_dst; long long kv_head_stride;
   void* k_cache; void* v_cache; const float* cos_tab; const float* sin_tab;
   int Hq, Hkv, hd;

@@ -116,23 +116,25 @@ __global__ void embed_norm_kernel(const __nv_bfloat16* __restrict__ table, const
   if (threadIdx.x == 0) ss[i] = red[0] + red[1] + red[2] + red[3];
 }
 
-// Weight re-layouts of the fused tensor-core path (run once, at context creation).
-//   rotary: inside every head of hd rows, output rows [32 g, 32 g + 16) are input rows [16 g, 16 g + 16) and output
-//           rows [32 g + 16, 32 g + 32) are input rows [hd/2 + 16 g, ...): every 32-row group holds 16 rotary pairs.
-//   gate/up: output rows [32 t, 32 t + 16) are gate rows [16 t, ...), rows [32 t + 16, 32 t + 32) the matching up rows.
+// Weight re-layouts of the fused tensor-core path (run once, at context creation).  The GEMM epilogue hands every
+// lane 4 consecutive output columns; the rows are ordered so that those 4 columns are everything the lane needs:
+//   rotary:  inside every head of hd rows, the 4 rows 32 g + 4 k .. + 3 are input rows i, i + 1, i + hd/2, i + 1 + hd/2
+//            with i = 16 g + 2 k  (two rotary pairs);
+//   gate/up: rows 32 t + 4 k .. + 3 are gate rows f, f + 1 and up rows f, f + 1 with f = 16 t + 2 k.
 __global__ void permute_rotary_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
                                            int hd, int cols) {
   const int r = blockIdx.x;
-  const int h = r / hd, w = r % hd, g = w >> 5, j = w & 31;
-  const int sr = h * hd + (j < 16 ? 16 * g + j : (hd >> 1) + 16 * g + (j - 16));
-  for (int c = threadIdx.x; c < cols; c += blockDim.x) dst[(long long)r * cols + c] = src[(long long)sr * cols + c];
+  const int h = r / hd, w = r % hd, g = w >> 5, j = w & 31, k = j >> 2, c = j & 3;
+  const int sr = h * hd + 16 * g + 2 * k + (c & 1) + (c >= 2 ? (hd >> 1) : 0);
+  for (int t = threadIdx.x; t < cols; t += blockDim.x) dst[(long long)r * cols + t] = src[(long long)sr * cols + t];
 }
 __global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ gate, const __nv_bfloat16* __restrict__ up,
                                           __nv_bfloat16* __restrict__ dst, int cols) {
   const int r = blockIdx.x;
-  const int t = r >> 5, j = r & 31;
-  const __nv_bfloat16* src = (j < 16 ? gate + (long long)(16 * t + j) * cols : up + (long long)(16 * t + j - 16) * cols);
-  for (int c = threadIdx.x; c < cols; c += blockDim.x) dst[(long long)r * cols + c] = src[c];
+  const int t = r >> 5, j = r & 31, k = j >> 2, c = j & 3;
+  const long long f = 16 * t + 2 * k + (c & 1);
+  const __nv_bfloat16* src = (c < 2 ? gate : up) + f * cols;
+  for (int i = threadIdx.x; i < cols; i += blockDim.x) dst[(long long)r * cols + i] = src[i];
 }
 
 void launch_embed_norm(const void* table, const int* tokens, int M, const int* M_dev, int d, float* resid,

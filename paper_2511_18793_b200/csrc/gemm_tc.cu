@@ -106,19 +106,17 @@ __device__ __forceinline__ ChunkCtx chunk_ctx(const GemmArgs& g, int n_chunk, in
     cc.col = make_float4(g0.x, g0.y, g1.x, g1.y);
   }
   if (EPI == kEpiBiasTanhF32) cc.col = *reinterpret_cast<const float4*>(g.bias + n);
-  if (EPI == kEpiSwiGLU) cc.off = (n_chunk >> 1) + 4 * k;      // lanes k < 4: gate columns -> output features n_chunk / 2 + 4k ..
+  if (EPI == kEpiSwiGLU) cc.off = (n_chunk >> 1) + 2 * k;      // the lane's columns are (gate, gate, up, up) of 2 features
   if (EPI == kEpiRopeKV) {
     const GemmFuse& f = g.f;
-    const int q_cols = f.Hq * f.hd, k_cols = f.Hkv * f.hd, half = f.hd >> 1;
+    const int q_cols = f.Hq * f.hd, k_cols = f.Hkv * f.hd;
     if (n_chunk < q_cols + k_cols) {
-      // columns e and 16 + e of the group hold the rotary pair (x_i, x_{i + hd/2}), i = 16 * (group inside the head) + e;
-      // lanes k < 4 hold e = 4k .. 4k + 3, lanes k + 4 their partners
+      // the lane's columns are (x_i, x_{i+1}, x_{i+hd/2}, x_{i+1+hd/2}), i = 16 * (32-column group inside the head) + 2k
       const int nn = n_chunk < q_cols ? n_chunk : n_chunk - q_cols;
       const int head = nn / f.hd, in_head = nn - head * f.hd;
-      cc.tab = ((in_head >> 5) << 4) + 4 * (k & 3);
-      const int d = k < 4 ? cc.tab : half + cc.tab;
+      cc.tab = ((in_head >> 5) << 4) + 2 * k;
       cc.kind = n_chunk < q_cols ? 0 : 1;
-      cc.off = n_chunk < q_cols ? (long long)(n_chunk - in_head) + d : (long long)head * f.kv_head_stride + d;
+      cc.off = n_chunk < q_cols ? (long long)(n_chunk - in_head) + cc.tab : (long long)head * f.kv_head_stride + cc.tab;
     } else {
       const int nv = n - q_cols - k_cols;
       const int head = nv / f.hd;
@@ -138,14 +136,14 @@ __device__ __forceinline__ EpiAux epi_prefetch(const GemmArgs& g, const ChunkCtx
   } else if (EPI == kEpiRopeKV) {
     if (cc.kind < 2) {
       const long long t = (long long)pos * (g.f.hd >> 1) + cc.tab;
-      r.a = *reinterpret_cast<const float4*>(g.f.cos_tab + t);
-      r.b = *reinterpret_cast<const float4*>(g.f.sin_tab + t);
+      const float2 cs = *reinterpret_cast<const float2*>(g.f.cos_tab + t), sn = *reinterpret_cast<const float2*>(g.f.sin_tab + t);
+      r.a = make_float4(cs.x, cs.y, sn.x, sn.y);
     }
   }
   return r;
 }
 
-// `valid`: the row exists (shuffles are executed by every lane regardless).
+// `valid`: the row exists.
 template <int EPI>
 __device__ __forceinline__ float4 epi_apply(const GemmArgs& g, const ChunkCtx& cc, bool valid, int row, int n, int k, float4 x,
                                            const EpiAux& aux, long long kv_dst) {
@@ -163,13 +161,11 @@ __device__ __forceinline__ float4 epi_apply(const GemmArgs& g, const ChunkCtx& c
       *reinterpret_cast<float4*>(reinterpret_cast<float*>(g.C) + o) =
           make_float4(tanhf(x.x + cc.col.x), tanhf(x.y + cc.col.y), tanhf(x.z + cc.col.z), tanhf(x.w + cc.col.w));
   } else if (EPI == kEpiSwiGLU) {
-    // lanes k < 4 hold gate columns, lanes k + 4 the matching up projections
-    const float u0 = __shfl_xor_sync(0xffffffffu, x.x, 4), u1 = __shfl_xor_sync(0xffffffffu, x.y, 4);
-    const float u2 = __shfl_xor_sync(0xffffffffu, x.z, 4), u3 = __shfl_xor_sync(0xffffffffu, x.w, 4);
-    if (valid && k < 4)
-      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.C) + (long long)row * g.ldc + cc.off) =
-          pack_bf16x4(__fdividef(x.x, 1.f + __expf(-x.x)) * u0, __fdividef(x.y, 1.f + __expf(-x.y)) * u1,
-                      __fdividef(x.z, 1.f + __expf(-x.z)) * u2, __fdividef(x.w, 1.f + __expf(-x.w)) * u3);
+    if (valid) {
+      const __nv_bfloat162 y = __floats2bfloat162_rn(__fdividef(x.x, 1.f + __expf(-x.x)) * x.z,
+                                                     __fdividef(x.y, 1.f + __expf(-x.y)) * x.w);
+      *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(g.C) + (long long)row * g.ldc + cc.off) = y;
+    }
   } else if (EPI == kEpiAddNorm) {
     const float4 cn = make_float4(aux.a.x + x.x, aux.a.y + x.y, aux.a.z + x.z, aux.a.w + x.w);
     if (valid) {
@@ -179,20 +175,17 @@ __device__ __forceinline__ float4 epi_apply(const GemmArgs& g, const ChunkCtx& c
     }
     return cn;
   } else if (EPI == kEpiRopeKV) {
-    const float p0 = __shfl_xor_sync(0xffffffffu, x.x, 4), p1 = __shfl_xor_sync(0xffffffffu, x.y, 4);
-    const float p2 = __shfl_xor_sync(0xffffffffu, x.z, 4), p3 = __shfl_xor_sync(0xffffffffu, x.w, 4);
-    float4 y = x;
-    if (cc.kind < 2) {
-      const float sg = k < 4 ? -1.f : 1.f;             // x_i' = x_i c - x_j s ;  x_j' = x_j c + x_i s
-      y = make_float4(x.x * aux.a.x + sg * p0 * aux.b.x, x.y * aux.a.y + sg * p1 * aux.b.y,
-                      x.z * aux.a.z + sg * p2 * aux.b.z, x.w * aux.a.w + sg * p3 * aux.b.w);
-    }
-    const uint2 packed = pack_bf16x4(y.x, y.y, y.z, y.w);
-    if (cc.kind == 0) {
-      if (valid) *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.C) + (long long)row * g.ldc + cc.off) = packed;
-    } else if (valid && kv_dst >= 0) {
-      __nv_bfloat16* cache = reinterpret_cast<__nv_bfloat16*>(cc.kind == 1 ? g.f.k_cache : g.f.v_cache);
-      *reinterpret_cast<uint2*>(cache + kv_dst + cc.off) = packed;
+    if (cc.kind == 2) {
+      if (valid && kv_dst >= 0)
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(g.f.v_cache) + kv_dst + cc.off) = pack_bf16x4(x.x, x.y, x.z, x.w);
+    } else if (valid && (cc.kind == 0 || kv_dst >= 0)) {
+      // x_i' = x_i c - x_j s ;  x_j' = x_j c + x_i s   (j = i + hd/2; aux.a = cos_i, cos_{i+1}, sin_i, sin_{i+1})
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(x.x * aux.a.x - x.z * aux.a.z, x.y * aux.a.y - x.w * aux.a.w);
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(x.z * aux.a.x + x.x * aux.a.z, x.w * aux.a.y + x.y * aux.a.w);
+      __nv_bfloat16* dst = cc.kind == 0 ? reinterpret_cast<__nv_bfloat16*>(g.C) + (long long)row * g.ldc + cc.off
+                                        : reinterpret_cast<__nv_bfloat16*>(g.f.k_cache) + kv_dst + cc.off;
+      *reinterpret_cast<__nv_bfloat162*>(dst) = lo;
+      *reinterpret_cast<__nv_bfloat162*>(dst + (g.f.hd >> 1)) = hi;
     }
   }
   return x;
