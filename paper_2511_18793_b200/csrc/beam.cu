@@ -27,8 +27,18 @@ __device__ __forceinline__ bool cand_better(float s, int r, int t, float s2, int
   return t < t2;
 }
 
+// Monotone map float -> unsigned (larger float, larger integer), so that a warp maximum is one redux instruction.
+__device__ __forceinline__ unsigned ordered_bits(float f) {
+  const unsigned u = __float_as_uint(f + 0.f);           // + 0: minus zero and plus zero rank alike
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(unsigned o) {
+  return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
+}
+constexpr unsigned kOrderedNegInf = 0x007fffffu;          // ordered_bits(-inf)
+
 template <int VPL>
-__global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
+__global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x;
@@ -89,20 +99,19 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
           if (want_probe[j] && !ok[j]) key[j0 + j] = -INFINITY;
       }
     }
-    // ordered extraction
+    // ordered extraction: one warp arg-max per survivor (two redux instructions; ties go to the smaller code)
     int cnt = 0;
     for (int it = 0; it < want; ++it) {
-      float bv = -INFINITY; int bt = 0x7fffffff;
+      unsigned bo = 0u; int bt = 0x7fffffff;
 #pragma unroll
-      for (int j = 0; j < VPL; ++j)
-        if (key[j] > bv) { bv = key[j]; bt = lane + 32 * j; }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
-        if (ov > bv || (ov == bv && ot < bt)) { bv = ov; bt = ot; }
+      for (int j = 0; j < VPL; ++j) {
+        const unsigned o = ordered_bits(key[j]);
+        if (o > bo) { bo = o; bt = lane + 32 * j; }
       }
-      if (bv == -INFINITY) break;
+      const unsigned mo = __reduce_max_sync(0xffffffffu, bo);
+      if (mo <= kOrderedNegInf) break;
+      bt = __reduce_min_sync(0xffffffffu, bo == mo ? bt : 0x7fffffff);
+      const float bv = from_ordered_bits(mo);
       if ((bt & 31) == lane) {
 #pragma unroll
         for (int j = 0; j < VPL; ++j)
@@ -157,14 +166,12 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
         if (br == 0x7fffffff || cand_better(s, r, t, bs, br, bt)) { bs = s; br = r; bt = t; }
       }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float os = __shfl_xor_sync(0xffffffffu, bs, o);
-      const int orr = __shfl_xor_sync(0xffffffffu, br, o);
-      const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
-      if (orr != 0x7fffffff && (br == 0x7fffffff || cand_better(os, orr, ot, bs, br, bt))) { bs = os; br = orr; bt = ot; }
-    }
-    if (br == 0x7fffffff) break;
+    // warp arg-best: maximum score, then the smallest (parent rank, code) among the lanes that hold it
+    const unsigned bo = br == 0x7fffffff ? 0u : ordered_bits(bs);
+    const unsigned mo = __reduce_max_sync(0xffffffffu, bo);
+    if (mo == 0u) break;                                   // every list is exhausted
+    const unsigned pick = __reduce_min_sync(0xffffffffu, bo == mo ? ((unsigned)br << 16 | (unsigned)bt) : 0xffffffffu);
+    bs = from_ordered_bits(mo); br = (int)(pick >> 16); bt = (int)(pick & 0xffffu);
 #pragma unroll
     for (int q = 0; q < RPL; ++q)
       if (lane + 32 * q == br) ++ptr[q];
@@ -214,10 +221,12 @@ void launch_select(const SelectArgs& a, cudaStream_t st) {
   if (a.batch <= 0) return;
   const size_t smem = select_smem_bytes(a.in_stride, a.K);
   LaunchScope ls(kcSelect, st);
-  if (a.T <= 32) launch_pdl(select_kernel<1>, dim3(a.batch), dim3(256), smem, st, a);
-  else if (a.T <= 256) launch_pdl(select_kernel<8>, dim3(a.batch), dim3(256), smem, st, a);
-  else if (a.T <= 512) launch_pdl(select_kernel<16>, dim3(a.batch), dim3(256), smem, st, a);
-  else launch_pdl(select_kernel<32>, dim3(a.batch), dim3(256), smem, st, a);
+  const int warps = a.in_stride < 8 ? 8 : a.in_stride > 16 ? 16 : a.in_stride;   // a warp per beam where that fits
+  const dim3 block(32 * warps);
+  if (a.T <= 32) launch_pdl(select_kernel<1>, dim3(a.batch), block, smem, st, a);
+  else if (a.T <= 256) launch_pdl(select_kernel<8>, dim3(a.batch), block, smem, st, a);
+  else if (a.T <= 512) launch_pdl(select_kernel<16>, dim3(a.batch), block, smem, st, a);
+  else launch_pdl(select_kernel<32>, dim3(a.batch), block, smem, st, a);
 }
 
 // ====================================================================================================
