@@ -146,6 +146,7 @@ def main():
     ap.add_argument("--drafts", default="natural", choices=["natural", "perfect"],
                     help="mode 1 only: 'natural' = the (random-init) draft head's own drafts; 'perfect' = the true top-k "
                          "tuples injected as round-1 drafts (best case: one round, everything accepted)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (requests per decode call)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
     args = ap.parse_args()
@@ -159,6 +160,8 @@ def main():
     from paper_2511_18793_b200 import synth
 
     w = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = synth.scaled(w, batch=args.batch)
     config = {"workload": f"{w.name}: {w.n_layers}L d{w.d_model} {w.n_q_heads}q/{w.n_kv_heads}kv ffn{w.d_ffn}, "
                           f"L={w.L} T={w.T[0]}, catalogue {w.n_items} ({w.catalog}), history {w.n_hist} items, "
                           f"batch {w.batch} x beam {w.beam}, seed {w.seed}",
@@ -346,7 +349,8 @@ def main():
             "clocks": clocks, "gpu_launches": int(launches),
             "rounds_per_step": rounds / args.steps, "primary_tokens_per_step": tokens / args.steps,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "includes": "H2D histories + prefill + decode + D2H results", "steps": e2e_steps},
+                    "includes": "H2D histories + prefill + decode + D2H results", "steps": e2e_steps,
+                    "ms_per_step": float(te.item()) / e2e_steps},
             "roofline": roof}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

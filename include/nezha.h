@@ -162,6 +162,19 @@ nezha_status nezha_decode_with_drafts(nezha_ctx* ctx, int32_t batch, int32_t bea
                                       int32_t* out_codes, float* out_scores, int32_t* out_count,
                                       nezha_decode_stats* stats, const nezha_trace* trace);
 
+/* Variants of the draft head: the ablations of Section 4.3 ("Ablation Study").  Defaults give Eq. 1-3 and Eq. 5 as
+ * printed.  Takes effect from the next nezha_decode / nezha_draft_logits call; never touches the primary model, so
+ * modes 1 and 2 still return Algorithm 1's result.
+ *   NEZHA_OPT_DRAFT_TRANSITION  0: s_{l+1} = tanh(W_s s_l + W_e e_l + b) (Eq. 3)    1: s_{l+1} = s_l + e_l   (NEZHA-3)
+ *   NEZHA_OPT_DRAFT_INPUTS      0: logits from h_l + s_l (Eq. 2)   1: from h_l alone, no context state (NEZHA-1)
+ *                               2: from s_l alone (NEZHA-2)
+ *   NEZHA_OPT_DRAFT_FILTER      1: hash-set filter at the last level (Eq. 5)        0: no filter              (NEZHA-4)
+ * Errors: NEZHA_ERR_ARG (unknown option or value). */
+#define NEZHA_OPT_DRAFT_TRANSITION 0
+#define NEZHA_OPT_DRAFT_INPUTS 1
+#define NEZHA_OPT_DRAFT_FILTER 2
+nezha_status nezha_set_option(nezha_ctx* ctx, int32_t option, int32_t value);
+
 /* ---- stage-wise entry points (the same kernels as nezha_decode, one step at a time) ------------------- */
 
 /* h_0..h_L of the prefilled rows as fp32: device float [batch, L+1, d].  Asynchronous. */

@@ -280,7 +280,10 @@ class Request:
 # ----------------------------------------------------------------------------------------------------
 
 class DraftHead:
-    def __init__(self, shape: ModelShape, weights: Dict[str, object], additive_transition: bool = False):
+    def __init__(self, shape: ModelShape, weights: Dict[str, object], additive_transition: bool = False,
+                 use_hidden: bool = True, use_state: bool = True):
+        """The switches are the ablation variants of Section 4.3: additive_transition = NEZHA-3 (Transition replaced by
+        addition), use_state=False = NEZHA-1 (no context state, hence no transition), use_hidden=False = NEZHA-2."""
         self.s = shape
         self.w_logit = [np.asarray(a, dtype=np.float64) for a in weights["draft_logit"]]
         self.ws = np.asarray(weights["draft_ws"], dtype=np.float64)
@@ -288,10 +291,12 @@ class DraftHead:
         self.b = np.asarray(weights["draft_b"], dtype=np.float64)
         self.embed = weights["embed"]
         self.additive = additive_transition
+        self.use_hidden, self.use_state = use_hidden, use_state
 
     def logits(self, level: int, h_l: np.ndarray, s_l: np.ndarray) -> np.ndarray:
         """Eq. 2 (level is 0-based: level 0 predicts the first code from h_1 and s_1)."""
-        return self.w_logit[level] @ (h_l + s_l)
+        x = (h_l if self.use_hidden else 0.0) + (s_l if self.use_state else 0.0)
+        return self.w_logit[level] @ (x + np.zeros_like(h_l))
 
     def transition(self, level: int, s_l: np.ndarray, code: int) -> np.ndarray:
         """Eq. 3 with e_l = embedding of the chosen level-`level` code."""

@@ -20,6 +20,7 @@ lib = C.CDLL(LIB_PATH)
 
 MAX_LEVELS = 8
 MODE_DRAFT, MODE_VERIFIED, MODE_AR = 0, 1, 2
+OPT_DRAFT_TRANSITION, OPT_DRAFT_INPUTS, OPT_DRAFT_FILTER = 0, 1, 2
 STATUS_NAMES = ["OK", "ERR_ARG", "ERR_STATE", "ERR_ARENA_TOO_SMALL", "ERR_CUDA", "ERR_HASH_FULL", "ERR_CATALOG",
                 "ERR_UNSUPPORTED"]
 
@@ -72,6 +73,8 @@ lib.nezha_decode.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, C.POINTER(Nez
 lib.nezha_decode_with_drafts.restype = C.c_int
 lib.nezha_decode_with_drafts.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, C.POINTER(NezhaDecodeStats),
                                          C.POINTER(NezhaTrace)]
+lib.nezha_set_option.restype = C.c_int
+lib.nezha_set_option.argtypes = [_vp, _i32, _i32]
 lib.nezha_get_hidden.restype = C.c_int
 lib.nezha_get_hidden.argtypes = [_vp, _vp]
 lib.nezha_primary_logits.restype = C.c_int
@@ -104,7 +107,7 @@ lib.nezha_destroy.argtypes = [_vp]
 NOALLOC_MAX_TUPLES = 1 << 20
 EXPORTS = ["nezha_arena_bytes", "nezha_create", "nezha_build_hashset", "nezha_pack", "nezha_probe",
            "nezha_contains_noalloc", "nezha_prefill",
-           "nezha_decode", "nezha_decode_with_drafts", "nezha_get_hidden", "nezha_primary_logits",
+           "nezha_decode", "nezha_decode_with_drafts", "nezha_set_option", "nezha_get_hidden", "nezha_primary_logits",
            "nezha_draft_logits", "nezha_select", "nezha_gemm", "nezha_launch_count", "nezha_profile_enable",
            "nezha_profile_read", "nezha_sync", "nezha_last_error", "nezha_destroy"]
 
@@ -270,6 +273,9 @@ class Engine:
                                                  C.byref(stats), C.byref(tr) if tr is not None else None))
         out["stats"] = stats
         return out
+
+    def set_option(self, option: int, value: int):
+        self._check(lib.nezha_set_option(self._h, option, value))
 
     def get_hidden(self) -> torch.Tensor:
         h = torch.empty(self.batch, self.L + 1, self.cfg.d_model, dtype=torch.float32, device=self.arena.device)

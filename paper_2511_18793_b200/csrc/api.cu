@@ -83,6 +83,7 @@ struct nezha_ctx {
   struct Segment { int seen; cudaGraphExec_t exec; long long launches[kcCount]; };
   std::map<std::array<uintptr_t, 16>, Segment> segments;
   bool use_graphs;
+  int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
   int state;                // 0 created, 1 hash set built, 2 prefilled
@@ -161,6 +162,7 @@ size_t carve(nezha_ctx* c) {
   Carver cv{c->arena, 0};
   EngineState& e = c->es;
   e.Bmax = c->Bmax; e.Kmax = c->Kmax; e.L = c->L; e.d = c->d; e.Hkv = c->Hkv; e.hd = c->hd;
+  e.draft_use_h = 1; e.draft_use_s = 1; e.draft_additive = 0;
   e.status = cv.take<int>(8);
   e.counters = cv.take<int>(8);
   c->n_unique_dev = cv.take<unsigned long long>(1);
@@ -375,8 +377,11 @@ void draft_logits_level(nezha_ctx* c, int batch, int l) {
        kEpiStoreF32);
 }
 
-// Eq. 3 for every (request, beam slot): s_{l+1} = tanh(W_s s_l + W_e e_l + b).
+// Eq. 3 for every (request, beam slot): s_{l+1} = tanh(W_s s_l + W_e e_l + b); s_l + e_l in the additive ablation;
+// nothing at all when the head does not use the context state.
 void draft_transition_level(nezha_ctx* c, int batch, int l) {
+  if (!c->es.draft_use_s) return;
+  if (c->es.draft_additive) { launch_trans_add(c->es, batch, l, c->embed, c->bf16, c->st); return; }
   launch_trans_gather(c->es, batch, l, c->embed, c->a_se, c->bf16, c->st);
   float* out = c->es.state_lv + (size_t)(l + 1) * c->Bmax * c->Kmax * c->d;
   gemm(c, c->a_se, 2 * c->d, c->draft_wse, 2 * c->d, out, c->d, (long long)batch * c->Kmax, nullptr, c->d, 2 * c->d,
@@ -473,7 +478,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
   const int R = L - 1;
   auto key_of = [&](int segment) {
     std::array<uintptr_t, 16> k{};
-    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)mode;
+    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16);
     k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
     k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
     k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams; k[14] = (uintptr_t)tr.beam_scores;
@@ -490,7 +495,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     launch_fill_i32(out_count, batch, 0, c->st);
     launch_init_decode(e, batch, c->st);
     if (mode == NEZHA_MODE_DRAFT) {
-      draft_phase(c, batch, K, true, 1, true);
+      draft_phase(c, batch, K, true, 1, c->opt_filter != 0);
       const size_t lv = (size_t)L * c->Bmax * c->Kmax;
       launch_write_out(e.dw_codes + lv * L, e.dw_score + lv, e.dw_count + (size_t)L * c->Bmax, c->Kmax, L, batch, K,
                        out_codes, out_scores, out_count, c->st);
@@ -524,7 +529,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
       launch_fill_i32(e.counters, 8, 0, c->st);
       if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
       else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
-      else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, true);
+      else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, c->opt_filter != 0);
       launch_build_nodes(e, batch, c->st);
       verify_pass(c, (long long)batch * K * (L - round), batch, K * (L - round));
       for (int n = round; n < L; ++n) {
@@ -590,6 +595,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   c->use_graphs = cuda_stream != nullptr && !getenv("NEZHA_NO_GRAPHS");
   c->m_expected = 0;
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
+  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;
@@ -734,6 +740,23 @@ nezha_status nezha_decode_with_drafts(nezha_ctx* c, int32_t batch, int32_t beam_
   if (!drafts || !n_draft) return fail(c, NEZHA_ERR_ARG, "nezha_decode_with_drafts: null drafts");
   return decode_impl(c, batch, beam_width, NEZHA_MODE_VERIFIED, drafts, n_draft, out_codes, out_scores, out_count, stats,
                      trace);
+}
+
+nezha_status nezha_set_option(nezha_ctx* c, int32_t option, int32_t value) {
+  if (!c) return NEZHA_ERR_ARG;
+  switch (option) {
+    case NEZHA_OPT_DRAFT_TRANSITION:
+      if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: transition must be 0 or 1");
+      c->opt_transition = value; c->es.draft_additive = value; break;
+    case NEZHA_OPT_DRAFT_INPUTS:
+      if (value < 0 || value > 2) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: inputs must be 0, 1 or 2");
+      c->opt_inputs = value; c->es.draft_use_h = value != 2; c->es.draft_use_s = value != 1; break;
+    case NEZHA_OPT_DRAFT_FILTER:
+      if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: filter must be 0 or 1");
+      c->opt_filter = value; break;
+    default: return fail(c, NEZHA_ERR_ARG, "nezha_set_option: unknown option");
+  }
+  return NEZHA_OK;
 }
 
 nezha_status nezha_get_hidden(nezha_ctx* c, float* out) {

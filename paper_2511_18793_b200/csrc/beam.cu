@@ -318,13 +318,15 @@ __global__ void draft_x_kernel(EngineState e, int batch, int l, T* x) {
   const float* h = e.h_f32 + ((long long)b * (e.L + 1) + l) * e.d;
   const float* s = (l == 1) ? e.h_f32 + (long long)b * (e.L + 1) * e.d
                             : e.state_lv + ((long long)l * e.Bmax * e.Kmax + bk) * e.d;
-  for (int c = threadIdx.x; c < e.d; c += blockDim.x) x[(long long)bk * e.d + c] = from_f32<T>(h[c] + s[c]);
+  const float uh = e.draft_use_h ? 1.f : 0.f, us = e.draft_use_s ? 1.f : 0.f;     // ablations: drop h_l or s_l
+  for (int c = threadIdx.x; c < e.d; c += blockDim.x) x[(long long)bk * e.d + c] = from_f32<T>(uh * h[c] + us * s[c]);
 }
 
 // Eq. 3 input rows [s_l ; e_l] for the step s_l -> s_{l+1}.
 //   requests still teacher-forcing (d_m >= l): beam k of the start set, its own state, its l-th code;
 //   requests drafting (d_m < l): survivor k of level l, its parent's state, the code just chosen.
-template <typename T>
+//   ADD = true (ablation: Transition replaced by addition): writes s_{l+1} = s_l + e_l (fp32) itself, no GEMM follows.
+template <typename T, bool ADD>
 __global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* embed, T* A) {
   pdl_wait();
   pdl_launch();
@@ -332,6 +334,7 @@ __global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* em
   const int b = bk / e.Kmax, k = bk - b * e.Kmax;
   if (b >= batch) return;
   T* dst = A + (long long)bk * 2 * e.d;
+  float* nxt = e.state_lv + ((long long)(l + 1) * e.Bmax * e.Kmax + bk) * e.d;
   const int dm = e.d_m[b];
   int src_level, parent;
   bool live = dm < e.L || e.row_m[b] < e.L;
@@ -343,15 +346,16 @@ __global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* em
   const int code = live ? e.dw_codes[s_idx * e.L + (l - 1)] : -1;
   live = live && code >= 0 && parent >= 0;
   if (!live) {
-    for (int c = threadIdx.x; c < 2 * e.d; c += blockDim.x) dst[c] = from_f32<T>(0.f);
+    if (ADD) { for (int c = threadIdx.x; c < e.d; c += blockDim.x) nxt[c] = 0.f; }
+    else { for (int c = threadIdx.x; c < 2 * e.d; c += blockDim.x) dst[c] = from_f32<T>(0.f); }
     return;
   }
   const float* s = (l == 1) ? e.h_f32 + (long long)b * (e.L + 1) * e.d
                             : e.state_lv + ((long long)l * e.Bmax * e.Kmax + (long long)b * e.Kmax + parent) * e.d;
   const T* emb = embed + (long long)(e.li.off[l - 1] + code) * e.d;
   for (int c = threadIdx.x; c < e.d; c += blockDim.x) {
-    dst[c] = from_f32<T>(s[c]);
-    dst[e.d + c] = emb[c];
+    if (ADD) { nxt[c] = s[c] + to_f32(emb[c]); }
+    else { dst[c] = from_f32<T>(s[c]); dst[e.d + c] = emb[c]; }
   }
 }
 
@@ -690,9 +694,18 @@ void launch_trans_gather(const EngineState& e, int batch, int l, const void* emb
                          cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
   if (bf16)
-    launch_pdl(trans_gather_kernel<__nv_bfloat16>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const __nv_bfloat16*)embed,
+    launch_pdl(trans_gather_kernel<__nv_bfloat16, false>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const __nv_bfloat16*)embed,
                                                                       (__nv_bfloat16*)A);
-  else launch_pdl(trans_gather_kernel<float>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const float*)embed, (float*)A);
+  else launch_pdl(trans_gather_kernel<float, false>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const float*)embed, (float*)A);
+}
+void launch_trans_add(const EngineState& e, int batch, int l, const void* embed, bool bf16, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
+  if (bf16)
+    launch_pdl(trans_gather_kernel<__nv_bfloat16, true>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l,
+               (const __nv_bfloat16*)embed, (__nv_bfloat16*)nullptr);
+  else
+    launch_pdl(trans_gather_kernel<float, true>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const float*)embed,
+               (float*)nullptr);
 }
 void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st) {
   LaunchScope ls(kcNodes, st, 2);

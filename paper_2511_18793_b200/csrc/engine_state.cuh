@@ -13,6 +13,8 @@ struct EngineState {
   LevelInfo li;
   HashSetView hs;
   int* status;
+  // draft-head variants (the ablations of Section 4.3); defaults 1, 1, 0 = Eq. 2 and Eq. 3 as printed
+  int draft_use_h, draft_use_s, draft_additive;
 
   // true beams, [L+1][Bmax][Kmax]([L])
   int* tb_codes; float* tb_score; int* tb_parent; int* tb_count;   // tb_count: [L+1][Bmax]
@@ -71,6 +73,7 @@ void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts,
 void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st);
 void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
                          cudaStream_t st);
+void launch_trans_add(const EngineState& e, int batch, int l, const void* embed, bool bf16, cudaStream_t st);
 void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st);
 void launch_nodes_from_prefixes(const EngineState& e, int batch, int n_beams, int level, const int* prefixes,
                                 cudaStream_t st);

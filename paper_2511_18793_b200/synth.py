@@ -62,6 +62,10 @@ WORKLOADS: Dict[str, Workload] = {
     "1.5b": Workload("1.5b", "bf16", 28, 1536, 12, 2, 8960, 4, (256,) * 4, 100_000_000, "zipf", 200, 128, 50, 3),
     "7b": Workload("7b", "bf16", 32, 4096, 32, 8, 11008, 4, (256,) * 4, 100_000_000, "zipf", 500, 32, 20, 4,
                    draft_noise=0.05),
+    # The setting of the paper's own public-data experiments (Section 4.1, Tables 2 and 3): semantic IDs of L = 3 codes
+    # over codebooks of 512, beam 10, histories of about a dozen items, tens of thousands of items, a backbone of the
+    # size of the 1B-parameter model it names (16 layers, d = 2048, 32 query / 8 KV heads, FFN 8192).
+    "paper": Workload("paper", "bf16", 16, 2048, 32, 8, 8192, 3, (512,) * 3, 57_000, "zipf", 12, 64, 10, 5),
 }
 
 

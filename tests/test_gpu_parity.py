@@ -257,3 +257,52 @@ def test_ragged_histories_and_small_beams():
         for b, n in enumerate([w.n_hist, 7, 0]):
             ref = O.ar_beam_search(model, case.req(b, n), K, V)[-1]
             assert assert_topk_matches(codes[b], scores[b], count[b], ref, K, tolerance(w))
+
+
+# ---------------------------------------------------------------------------------------- ablation variants (Section 4.3)
+VARIANTS = {                       # name -> (options to set, oracle head arguments, hash filter on)
+    "nezha1_no_state": ({1: 1}, dict(use_state=False), True),
+    "nezha2_no_hidden": ({1: 2}, dict(use_hidden=False), True),
+    "nezha3_additive": ({0: 1}, dict(additive_transition=True), True),
+    "nezha4_no_filter": ({2: 0}, dict(), False),
+}
+
+
+@pytest.mark.parametrize("variant", sorted(VARIANTS))
+@pytest.mark.parametrize("name", ["tiny", "small_cut"])
+def test_draft_head_variants(name, variant):
+    """nezha_set_option against the oracle's draft head with the same switch: teacher-forced logits, mode 0 output, and
+    mode 1 still equal to mode 2 (the variants never touch the primary model)."""
+    w = synth.WORKLOADS["tiny"] if name == "tiny" else \
+        synth.scaled(synth.WORKLOADS["small"], n_layers=2, n_items=100_000, batch=4, n_hist=20)
+    case = Case(w).prefill()
+    opts, head_kw, filt = VARIANTS[variant]
+    for k, v in opts.items():
+        case.eng.set_option(k, v)
+    model, _, V = case.oracle
+    from helpers import oracle_shape
+    head = O.DraftHead(oracle_shape(w), synth.weights_to_numpy(case.weights), **head_kw)
+    rng = np.random.default_rng(3)
+    tol = tolerance(w)
+    for level in range(w.L):
+        pre = np.stack([rng.integers(0, w.T[l], size=(w.batch, w.beam)) for l in range(level)], axis=2).astype(np.int32) \
+            if level else None
+        got = case.eng.draft_logits(w.beam, level, None if pre is None else torch.from_numpy(pre).cuda()).cpu().numpy()
+        for b in range(w.batch):
+            for r in range(w.beam):
+                st = O.teacher_forced_state(head, case.req(b), tuple(pre[b, r]) if level else ())
+                assert np.abs(got[b, r] - head.logits(level, case.req(b).h[level + 1], st)).max() < tol
+    out = case.eng.decode(w.beam, mode=0)
+    codes, scores, count = (out[k].cpu().numpy() for k in ("codes", "scores", "count"))
+    for b in range(w.batch):
+        ref = O.nezha_draft(head, case.req(b), w.beam, V if filt else None)[-1]
+        assert_topk_matches(codes[b], scores[b], count[b], ref, w.beam, tol)
+    if not filt:
+        live = np.arange(w.beam)[None, :] < count[:, None]
+        assert not V.contains(codes[live]).all() or w.name == "tiny"     # without Eq. 5 hallucinated tuples get through
+    m1, m2 = case.eng.decode(w.beam, mode=1), case.eng.decode(w.beam, mode=2)
+    assert torch.equal(m1["codes"], m2["codes"]) and torch.equal(m1["count"], m2["count"])
+    with pytest.raises(case.binding.NezhaError):
+        case.eng.set_option(7, 0)
+    with pytest.raises(case.binding.NezhaError):
+        case.eng.set_option(1, 3)

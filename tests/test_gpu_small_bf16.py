@@ -129,6 +129,28 @@ def test_bf16_shapes_ragged_histories(shape):
         check_levels(case, b, beams[:, b], scores[:, b], w.beam)
 
 
+def test_paper_setting_three_levels_of_512_codes():
+    """L = 3 levels over codebooks of 512 (the paper's own setting), beam 10, short histories: every mode, all requests,
+    on a two-layer cut of the 1B-sized backbone."""
+    w = synth.scaled(synth.WORKLOADS["paper"], n_layers=2, batch=6)
+    case = Case(w).prefill()
+    model, head, V = case.oracle
+    assert case.n_unique == w.n_items
+    out = case.eng.decode(w.beam, mode=1, trace=True)
+    ar = case.eng.decode(w.beam, mode=2)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
+    beams, scores = out["trace"]["beams"].cpu().numpy(), out["trace"]["beam_scores"].cpu().numpy()
+    dr = case.eng.decode(w.beam, mode=0)
+    dcodes, dscores, dcount = (dr[k].cpu().numpy() for k in ("codes", "scores", "count"))
+    for b in range(w.batch):
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam)
+        ref = O.nezha_draft(head, case.req(b), w.beam, V)[-1]
+        assert_topk_matches(dcodes[b], dscores[b], dcount[b], ref, w.beam, tolerance(w))
+    codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
+    live = np.arange(w.beam)[None, :] < count[:, None]
+    assert V.contains(codes[live]).all()
+
+
 @pytest.mark.parametrize("name", ["tiny", "small"])
 def test_graph_replay_equals_eager_launches(name):
     """On a stream of its own the library captures every round of a decode call into a CUDA graph after one eager

@@ -381,3 +381,41 @@ def test_speculative_round_two_drafts_extend_true_beams():
         st = O.teacher_forced_state(head, req, bm.codes[:2])
         lp = float(O.log_softmax(head.logits(2, req.h[3], st))[bm.codes[2]])
         assert abs(float(bm.score) - (float(parent.score) + lp)) < 1e-5
+
+
+# ---------------------------------------------------------------------------------------- ablation variants (Section 4.3)
+def test_ablation_variants_of_the_draft_head():
+    """NEZHA-1 (no context state): every level's distribution ignores the prefix, so the joint log-probability is a sum
+    of per-level terms and the beam search equals the brute-force top-K of that sum over the valid tuples.
+    NEZHA-2 (no hidden state): the logits are W s_l, i.e. the default head's on a request whose h_1..h_L are zero.
+    NEZHA-3 (additive transition): s_{l+1} = s_l + e_l, written out here from the weights."""
+    w, W, cat, model, head, V, hist = _micro()
+    shape = oracle_shape(w)
+    req = model.prefill(hist[1])
+    f = lambda n: np.asarray(W[n], dtype=np.float64)
+    # NEZHA-1
+    h1 = O.DraftHead(shape, W, use_state=False)
+    per_level = [torch.log_softmax(torch.from_numpy(np.asarray(W["draft_logit"][l], dtype=np.float64) @ req.h[l + 1]), -1).numpy()
+                 for l in range(w.L)]
+    brute = sorted(((sum(per_level[l][t[l]] for l in range(w.L)), t) for t in _all_tuples(w.T) if V.contains(np.asarray([t]))[0]),
+                   key=lambda x: (-x[0], x[1]))
+    got = O.nezha_draft(h1, req, w.beam, V)[-1]
+    assert codes_of(got) == [t for _, t in brute[: len(got)]] and len(got) == min(w.beam, len(brute))
+    assert np.allclose(scores_of(got), [s for s, _ in brute[: len(got)]], atol=1e-5)
+    # NEZHA-2
+    h2 = O.DraftHead(shape, W, use_hidden=False)
+    req0 = O.Request(P=req.P, h=np.concatenate([req.h[:1], np.zeros_like(req.h[1:])]), ctx_kv=req.ctx_kv)
+    assert codes_of(O.nezha_draft(h2, req, w.beam, V)[-1]) == codes_of(O.nezha_draft(head, req0, w.beam, V)[-1])
+    assert np.array_equal(h2.logits(1, req.h[2], req.h[0]), np.asarray(W["draft_logit"][1], dtype=np.float64) @ req.h[0])
+    assert codes_of(O.nezha_draft(h2, req, w.beam, V)[-1]) != codes_of(O.nezha_draft(head, req, w.beam, V)[-1])
+    # NEZHA-3
+    h3 = O.DraftHead(shape, W, additive_transition=True)
+    s2 = h3.transition(0, req.h[0], 3)
+    assert np.array_equal(s2, req.h[0] + f("embed")[3])
+    assert np.array_equal(h3.transition(1, s2, 1), req.h[0] + f("embed")[3] + f("embed")[w.T[0] + 1])
+    lp = O.joint_logprob_draft(h3, req, (3, 1, 2))
+    zs = [np.asarray(W["draft_logit"][0], dtype=np.float64) @ (req.h[1] + req.h[0]),
+          np.asarray(W["draft_logit"][1], dtype=np.float64) @ (req.h[2] + s2),
+          np.asarray(W["draft_logit"][2], dtype=np.float64) @ (req.h[3] + s2 + f("embed")[w.T[0] + 1])]
+    want = sum(float(torch.log_softmax(torch.from_numpy(z), -1)[c]) for z, c in zip(zs, (3, 1, 2)))
+    assert abs(lp - want) < 1e-12
