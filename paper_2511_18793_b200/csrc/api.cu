@@ -289,6 +289,7 @@ void run_layers_fused(nezha_ctx* c, long long M, const int* M_dev, bool verify, 
     t.row_start = verify ? e.row_tok_start : e.pf_row_start; t.row_count = verify ? e.row_tok_count : e.pf_row_count;
     t.req_info = verify ? e.req_info : e.pf_req_info;
     t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
+    t.rows_expected = (c->m_expected > 0 && n_rows > 0) ? (c->m_expected + n_rows - 1) / n_rows * (c->Hq / c->Hkv) : 0;
     t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
     if (attention_tc_supported(t)) launch_attention_tc(t, c->st);
     else launch_attention_simt(t, true, c->st);

@@ -409,10 +409,25 @@ void launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   const CUtensorMap* tv = tma_map_bf16(a.v_ctx, rows, a.hd, a.hd, kPos);
   if (!tk || !tv) { launch_attention_simt(a, true, st); return; }
   LaunchScope ls(kcAttention, st);
-  // few query rows per (request, KV head): 16-row CTAs whose warps split the KV tiles; else 64-row CTAs
-  const bool few = (long long)a.max_tokens_per_row * (a.Hq / a.Hkv) <= 32;
-  if (a.hd == 64) { if (few) launch<64, 1, 2>(tk, tv, a, st); else launch<64, 4, 1>(tk, tv, a, st); }
-  else { if (few) launch<128, 1, 2>(tk, tv, a, st); else launch<128, 4, 1>(tk, tv, a, st); }
+  // Query rows per (request, KV head): the bound the grid must cover, and what the caller expects (shapes the tile only).
+  const int G = a.Hq / a.Hkv;
+  const long long r_bound = (long long)a.max_tokens_per_row * G;
+  const long long r = a.rows_expected > 0 && a.rows_expected < r_bound ? a.rows_expected : r_bound;
+  if (r <= 32) {                                     // 16-row CTAs whose two consumer warps split the KV tiles
+    if (a.hd == 64) launch<64, 1, 2>(tk, tv, a, st); else launch<128, 1, 2>(tk, tv, a, st);
+    return;
+  }
+  // otherwise the fewest CTAs of at most 128 rows, each as short as covers the rows: little padding, K/V streamed
+  // as few times as possible
+  const int groups = (int)((r + 15) / 16), n_ctas = (groups + 7) / 8;
+  const int rw = (groups + n_ctas - 1) / n_ctas;     // 3 .. 8 warps of 16 rows
+#define NZ_ATTN_CASE(RW_) \
+  case RW_: if (a.hd == 64) launch<64, RW_, 1>(tk, tv, a, st); else launch<128, RW_, 1>(tk, tv, a, st); break;
+  switch (rw) {
+    NZ_ATTN_CASE(3) NZ_ATTN_CASE(4) NZ_ATTN_CASE(5) NZ_ATTN_CASE(6) NZ_ATTN_CASE(7)
+    default: if (a.hd == 64) launch<64, 8, 1>(tk, tv, a, st); else launch<128, 8, 1>(tk, tv, a, st); break;
+  }
+#undef NZ_ATTN_CASE
 }
 
 }  // namespace nz

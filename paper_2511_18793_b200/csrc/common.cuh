@@ -240,6 +240,7 @@ struct AttnArgs {
   const int4* req_info;                         // [n_rows] {first token, token count, cache row, context length visible to
                                                 //  every token of the request, or -1: token j of the request sees j + 1}
   int n_rows, max_tokens_per_row;
+  int rows_expected;                            // 0, or the query rows per (request, kv head) the caller expects: tiling only
   long long ctx_rows_total;                     // requests * kv heads * positions of the layer's context cache
   int* status;
 };
