@@ -20,7 +20,9 @@ def _ref(A, W):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 512), (1920, 1536, 512), (77, 768, 2048), (640, 512, 1024),
-                                    (1, 128, 64), (129, 128, 4864)])
+                                    (1, 128, 64), (129, 128, 4864),
+                                    # large enough for the CTA-pair kernel (256 x 256 tiles), ragged in M and in N
+                                    (5000, 2304, 896), (18000, 1152, 512), (4100, 512, 2048)])
 @pytest.mark.parametrize("path", [1, 2])
 def test_gemm_epilogues(ctx, M, N, K, path):
     g = torch.Generator(device="cuda"); g.manual_seed(M * 7 + N * 3 + K)
