@@ -13,6 +13,7 @@
 // The per-token extra KV rows (the token's own tuple's drafted codes, at most L-1 of them) are folded in afterwards
 // straight from global memory.  Every barrier wait is bounded (abort flag + error status + return).
 #include <math.h>
+#include <stdlib.h>
 
 #include "tma.cuh"
 
@@ -394,6 +395,8 @@ void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cud
 
 }  // namespace
 
+void launch_attention_umma(const AttnArgs& a, const CUtensorMap* tk, const CUtensorMap* tv, cudaStream_t st);
+
 bool attention_tc_supported(const AttnArgs& a) {
   if (!a.status || !a.req_info || a.n_rows <= 0 || a.max_tokens_per_row <= 0) return false;
   if (a.hd != 64 && a.hd != 128) return false;
@@ -417,6 +420,8 @@ void launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
     if (a.hd == 64) launch<64, 1, 2>(tk, tv, a, st); else launch<128, 1, 2>(tk, tv, a, st);
     return;
   }
+  static const bool umma = getenv("NEZHA_NO_UMMA_ATTENTION") == nullptr;
+  if (umma && r >= 64) { launch_attention_umma(a, tk, tv, st); return; }   // many rows: the tcgen05 kernel, 128 rows per CTA
   // otherwise the fewest CTAs of at most 128 rows, each as short as covers the rows: little padding, K/V streamed
   // as few times as possible
   const int groups = (int)((r + 15) / 16), n_ctas = (groups + 7) / 8;

@@ -1,0 +1,367 @@
+// KV-cache attention on the Blackwell tensor path (tcgen05 + TMEM), for many query rows per (request, KV head).
+//
+// One CTA = (request, KV head, tile of 128 query rows): the rows are the request's tokens of this pass times the G query
+// heads of the group, so the context K/V is streamed once per 128 rows.  Per 64-position K/V tile (brought in by TMA,
+// 128-byte swizzle, 3-slot ring):
+//   S = Q K^T      tcgen05.mma M128 N64 K16 x hd/16, Q resident in shared memory, S in one of two 64-column TMEM buffers
+//   softmax        4 warps, one thread per row (a TMEM lane is a row, so row maximum and row sum need no shuffles):
+//                  tcgen05.ld the row's 64 scores, base-2 exponentials against a running reference maximum that is only
+//                  raised when the true maximum has grown by more than 8 (then the O accumulator in TMEM is rescaled
+//                  with tcgen05.ld / st); P goes to shared memory as the bf16 A operand of the second product
+//   O += P V       tcgen05.mma M128 N=hd K16 x 4, V taken as it lies in the cache ([position][hd] = N-major operand)
+// The S product of tile j+1 is issued before the softmax of tile j is awaited, so the tensor pipe works under the
+// softmax.  At the end each thread folds in its row's extra KV rows (the token's own drafted codes) from global
+// memory, normalises and stores its row.  Every mbarrier wait is bounded (abort flag, error status, TMEM freed).
+#include <math.h>
+
+#include "gemm_epilogue.cuh"
+
+namespace nz {
+
+namespace {
+
+using namespace gemm_detail;
+
+constexpr int kPosU = 64;          // KV positions per tile
+constexpr int kRowsU = 128;        // query rows per CTA
+constexpr int kStagesU = 3;
+constexpr int kThreadsU = 192;     // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: softmax (one thread per row)
+constexpr float kRaise = 8.f;      // the reference maximum follows the true one only in steps larger than this (log2 units)
+
+template <int HD> struct UmmaCfg {
+  static constexpr int kQBytes = kRowsU * HD * 2;
+  static constexpr int kPBytes = kRowsU * kPosU * 2;
+  static constexpr int kTileBytes = kPosU * HD * 2;            // one K (or V) tile
+  static constexpr int kStageBytes = 2 * kTileBytes;
+  static constexpr int kSmemBytes = kQBytes + kPBytes + kStagesU * kStageBytes + 1024 + 256;
+  static constexpr int kTmemCols = HD == 64 ? 256 : 256;       // S: 2 x 64 columns, O: HD columns; a power of two
+  static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kPosU >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
+  static constexpr uint32_t kIdescPV =
+      (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) /* B is N-major */ | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
+};
+
+// N-major (MN-major) operand tile with the 128-byte swizzle: rows of 64 elements along N, 8-row groups along K 1024 B
+// apart (SBO), 64-element groups along N `lbo` bytes apart (LBO).
+__device__ __forceinline__ uint64_t smem_desc_nmajor(uint32_t addr, uint32_t lbo) {
+  return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((lbo >> 4) & 0x3FFF) << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]),
+        "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]),
+        "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]),
+        "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31]) : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2u(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+template <int HD>
+__global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                             const __grid_constant__ CUtensorMap tmV, AttnArgs a, int* status) {
+  using C = UmmaCfg<HD>;
+  constexpr int S = kStagesU;
+  constexpr int NH = HD / 64;                       // 64-column sub-tiles of a K / V / Q tile
+  constexpr int KS = HD / 16;                       // k-steps of Q K^T
+  constexpr uint32_t kColS = 0, kColO = 128;        // TMEM columns: S buffers at 0 and 64, O at 128
+
+  pdl_wait();                                       // before the first global read and before any exit
+  pdl_launch();
+  const int req_local = blockIdx.z, kvh = blockIdx.y, tile = blockIdx.x;
+  const int G = a.Hq / a.Hkv;
+  const int4 info = a.req_info[req_local];          // {first token, token count, cache row, context length or -1}
+  const int tok0 = info.x, n_tok = info.y, request = info.z;
+  const int R = n_tok * G;
+  const int r0 = tile * kRowsU;
+  if (r0 >= R) return;
+  const int max_ctx = info.w >= 0 ? info.w : min((r0 + kRowsU - 1) / G, n_tok - 1) + 1;
+  const int n_tiles = (max_ctx + kPosU - 1) / kPosU;
+  const int kv_row0 = (int)(((long long)request * a.Hkv + kvh) * (a.ctx_head_stride / HD));
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_base = base, p_base = base + C::kQBytes, kv_base = p_base + C::kPBytes;
+  const uint32_t bar_base = kv_base + S * C::kStageBytes;
+  auto kv_full = [&](int s) { return bar_base + 8u * s; };
+  auto kv_empty = [&](int s) { return bar_base + 8u * (S + s); };
+  auto s_full = [&](int b) { return bar_base + 8u * (2 * S + b); };
+  auto s_free = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
+  const uint32_t p_full = bar_base + 8u * (2 * S + 4), pv_done = bar_base + 8u * (2 * S + 5);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - base) + 8 * (2 * S + 6));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(s_free(b), 4); }
+    mbar_init(p_full, 4); mbar_init(pv_done, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(C::kTmemCols));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  // the softmax threads bring their own query row into shared memory (K-major, 128-byte swizzle), zeros for dead rows
+  int row = -1, tok = 0, head = 0, ctx = 0;
+  bool live = false;
+  if (warp >= 2) {
+    row = (warp & 3) * 32 + lane;                   // = the TMEM lane this thread may read
+    live = r0 + row < R;
+    const int rr = live ? r0 + row : r0;
+    tok = tok0 + rr / G; head = kvh * G + rr % G;
+    ctx = !live ? 0 : (info.w >= 0 ? info.w : rr / G + 1);
+    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) + (long long)tok * a.q_stride +
+                                                      (long long)head * HD);
+#pragma unroll
+    for (int c = 0; c < HD / 8; ++c) {
+      const uint4 v = live ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t dst = (c >> 3) * (kRowsU * 128) + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+      *reinterpret_cast<uint4*>(gen_base + dst) = v;
+    }
+    fence_async_smem();                             // generic-proxy writes, read by the tensor core through the async proxy
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const float sc = a.scale * 1.4426950408889634f;   // scores in base 2
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int t = 0;
+      bool ok = true;
+      for (; t < n_tiles; ++t) {
+        const int s = t % S;
+        if (t >= S && !mbar_wait_or_abort(kv_empty(s), ((t / S) - 1) & 1, abort_flag)) { ok = false; break; }
+        mbar_expect_tx(kv_full(s), C::kStageBytes);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          tma_load_2d(kv_base + s * C::kStageBytes + h * (kPosU * 128), &tmK, h * 64, kv_row0 + t * kPosU, kv_full(s));
+          tma_load_2d(kv_base + s * C::kStageBytes + C::kTileBytes + h * (kPosU * 128), &tmV, h * 64, kv_row0 + t * kPosU, kv_full(s));
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        for (int j = max(0, t - S); j < t; ++j) mbar_wait(kv_full(j % S), (j / S) & 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      auto issue_s = [&](int j) {                    // S_j = Q K_j^T into S buffer j & 1
+        const int s = j % S, b = j & 1;
+        if (!mbar_wait_or_abort(kv_full(s), (j / S) & 1, abort_flag)) return false;
+        if (j >= 2 && !mbar_wait_or_abort(s_free(b), ((j >> 1) - 1) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t kt = kv_base + s * C::kStageBytes;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+          tc_mma(tmem_base + kColS + (uint32_t)(b * kPosU), smem_desc(q_base + (ks >> 2) * (kRowsU * 128) + (ks & 3) * 32),
+                 smem_desc(kt + (ks >> 2) * (kPosU * 128) + (ks & 3) * 32), C::kIdescS, ks > 0 ? 1u : 0u);
+        tc_commit(s_full(b));
+        return true;
+      };
+      if (n_tiles > 0) ok = issue_s(0);
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        if (j + 1 < n_tiles && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
+        if (!mbar_wait_or_abort(p_full, j & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t vt = kv_base + (j % S) * C::kStageBytes + C::kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < kPosU / 16; ++ks)
+          tc_mma(tmem_base + kColO, smem_desc(p_base + ks * 32), smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128), C::kIdescPV,
+                 (j > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(kv_empty(j % S));                  // K_j and V_j are no longer needed
+        tc_commit(pv_done);                          // O holds tiles 0..j
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax, one thread per row
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    float m_ref = -INFINITY, l_run = 0.f;           // reference maximum (scaled log2 domain) and row sum against it
+    bool ok = true;
+    const int ctx_min = __reduce_min_sync(0xffffffffu, ctx);
+    for (int j = 0; j < n_tiles; ++j) {
+      const int b = j & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full(b), (j >> 1) & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      float sv[kPosU];
+      tmem_ld32(tmem_base + lane_addr + kColS + (uint32_t)(b * kPosU), sv);
+      tmem_ld32(tmem_base + lane_addr + kColS + (uint32_t)(b * kPosU + 32), sv + 32);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_free(b));         // the scores are in registers: the buffer may take tile j + 2
+      if ((j + 1) * kPosU > ctx_min) {
+#pragma unroll
+        for (int c = 0; c < kPosU; ++c)
+          if (j * kPosU + c >= ctx) sv[c] = -INFINITY;
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < kPosU; ++c) mx = fmaxf(mx, sv[c]);
+      mx *= sc;
+      // raise the reference only when the true maximum has run away from it: p stays below 2^8 otherwise
+      const bool raise = mx > m_ref + kRaise || (m_ref == -INFINITY && mx > -INFINITY);
+      const float m_new = raise ? mx : m_ref;
+      const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+      const float corr = raise ? ex2u(m_ref - m_safe) : 1.f;     // ex2(-inf) = 0 the first time
+      float rs = 0.f;
+      uint32_t pk[kPosU / 2];
+#pragma unroll
+      for (int c = 0; c < kPosU; c += 2) {
+        const float p0 = ex2u(fmaf(sv[c], sc, -m_safe)), p1 = ex2u(fmaf(sv[c + 1], sc, -m_safe));
+        rs += p0 + p1;
+        __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+        pk[c >> 1] = *reinterpret_cast<uint32_t*>(&pb);
+      }
+      l_run = l_run * corr + rs;
+      m_ref = m_new;
+      if (j > 0) {                                   // O (tiles 0..j-1) must be complete before it is rescaled or P replaced
+        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, (j - 1) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, raise)) {
+#pragma unroll 1
+          for (int c = 0; c < HD / 32; ++c) {
+            float ov[32];
+            tmem_ld32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ov[i] *= corr;
+            tmem_st32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
+          }
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        *reinterpret_cast<uint4*>(gen_base + (p_base - base) + row * 128 + ((c ^ (row & 7)) << 4)) =
+            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full);
+    }
+    if (ok && n_tiles > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, (n_tiles - 1) & 1, abort_flag));
+      tc_fence_after();
+    }
+    if (!ok) { if (lane == 0) *abort_flag = 1; }
+    else {
+      // ---- the row's own extra KV rows, then normalise and store (thread = row)
+      constexpr int E = kMaxLevels;
+      const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(a.q) + (long long)tok * a.q_stride + (long long)head * HD;
+      const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
+      const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
+      long long off[E]; float se[E];
+      float m_fin = m_ref;
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        off[e] = (live && e < a.n_ext_max) ? a.tok_ext[(long long)tok * a.n_ext_max + e] : -1;
+        se[e] = -INFINITY;
+      }
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        if (off[e] < 0) continue;
+        const uint4* kp = reinterpret_cast<const uint4*>(ke + off[e] + (long long)kvh * a.ext_head_stride);
+        float d = 0.f;
+        for (int c = 0; c < HD / 8; ++c) {
+          const uint4 qv = reinterpret_cast<const uint4*>(qp)[c], kv = kp[c];
+          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
+          const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 qf = __bfloat1622float2(q2[i]), kf = __bfloat1622float2(k2[i]);
+            d = fmaf(qf.x, kf.x, d); d = fmaf(qf.y, kf.y, d);
+          }
+        }
+        se[e] = d * sc;
+        m_fin = fmaxf(m_fin, se[e]);
+      }
+      const float m_safe = m_fin == -INFINITY ? 0.f : m_fin;
+      const float c0 = ex2u(m_ref - m_safe);
+      float l_tot = l_run * c0, pe[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) { pe[e] = off[e] >= 0 ? ex2u(se[e] - m_safe) : 0.f; l_tot += pe[e]; }
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      __nv_bfloat16* op = reinterpret_cast<__nv_bfloat16*>(a.out) + (long long)tok * a.out_stride + (long long)head * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD / 32; ++c) {
+        float ov[32];
+        tmem_ld32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);   // warp-collective: dead rows take part too
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ov[i] *= c0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          if (off[e] < 0) continue;
+          const uint4* vp = reinterpret_cast<const uint4*>(ve + off[e] + (long long)kvh * a.ext_head_stride + c * 32);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint4 vv = vp[u];
+            const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vv);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 vf = __bfloat1622float2(v2[i]);
+              ov[u * 8 + 2 * i] = fmaf(pe[e], vf.x, ov[u * 8 + 2 * i]);
+              ov[u * 8 + 2 * i + 1] = fmaf(pe[e], vf.y, ov[u * 8 + 2 * i + 1]);
+            }
+          }
+        }
+        if (live && l_tot > 0.f) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              __nv_bfloat162 t = __floats2bfloat162_rn(ov[u * 8 + 2 * i] * inv, ov[u * 8 + 2 * i + 1] * inv);
+              w[i] = *reinterpret_cast<uint32_t*>(&t);
+            }
+            reinterpret_cast<uint4*>(op + c * 32)[u] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols));
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(status, kStInternal);
+}
+
+template <int HD>
+void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cudaStream_t st) {
+  using C = UmmaCfg<HD>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    configured = true;
+  }
+  const int G = a.Hq / a.Hkv;
+  dim3 grid((a.max_tokens_per_row * G + kRowsU - 1) / kRowsU, a.Hkv, a.n_rows);
+  launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, a, a.status);
+}
+
+}  // namespace
+
+// tk / tv: tensor maps of the layer's context K and V caches with boxes of 64 positions x 64 columns.
+void launch_attention_umma(const AttnArgs& a, const CUtensorMap* tk, const CUtensorMap* tv, cudaStream_t st) {
+  if (a.hd == 64) launch_umma<64>(tk, tv, a, st);
+  else launch_umma<128>(tk, tv, a, st);
+}
+
+}  // namespace nz
