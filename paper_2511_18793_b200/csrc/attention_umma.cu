@@ -7,7 +7,8 @@
 //   softmax        4 warps, one thread per row (a TMEM lane is a row, so row maximum and row sum need no shuffles):
 //                  tcgen05.ld the row's 64 scores, base-2 exponentials against a running reference maximum that is only
 //                  raised when the true maximum has grown by more than 8 (then the O accumulator in TMEM is rescaled
-//                  with tcgen05.ld / st); P goes to shared memory as the bf16 A operand of the second product
+//                  with tcgen05.ld / st); P goes to one of two shared-memory buffers as the bf16 A operand of the
+//                  second product, so the softmax of tile j + 1 does not wait for the product of tile j
 //   O += P V       tcgen05.mma M128 N=hd K16 x 4, V taken as it lies in the cache ([position][hd] = N-major operand)
 // The S product of tile j+1 is issued before the softmax of tile j is awaited, so the tensor pipe works under the
 // softmax.  At the end each thread folds in its row's extra KV rows (the token's own drafted codes) from global
@@ -33,7 +34,7 @@ template <int HD> struct UmmaCfg {
   static constexpr int kPBytes = kRowsU * kPosU * 2;
   static constexpr int kTileBytes = kPosU * HD * 2;            // one K (or V) tile
   static constexpr int kStageBytes = 2 * kTileBytes;
-  static constexpr int kSmemBytes = kQBytes + kPBytes + kStagesU * kStageBytes + 1024 + 256;
+  static constexpr int kSmemBytes = kQBytes + 2 * kPBytes + kStagesU * kStageBytes + 1024 + 256;
   static constexpr int kTmemCols = HD == 64 ? 256 : 256;       // S: 2 x 64 columns, O: HD columns; a power of two
   static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kPosU >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
   static constexpr uint32_t kIdescPV =
@@ -88,21 +89,22 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_base = base, p_base = base + C::kQBytes, kv_base = p_base + C::kPBytes;
+  const uint32_t q_base = base, p_base = base + C::kQBytes, kv_base = p_base + 2 * C::kPBytes;   // two P buffers
   const uint32_t bar_base = kv_base + S * C::kStageBytes;
   auto kv_full = [&](int s) { return bar_base + 8u * s; };
   auto kv_empty = [&](int s) { return bar_base + 8u * (S + s); };
   auto s_full = [&](int b) { return bar_base + 8u * (2 * S + b); };
   auto s_free = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
-  const uint32_t p_full = bar_base + 8u * (2 * S + 4), pv_done = bar_base + 8u * (2 * S + 5);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - base) + 8 * (2 * S + 6));
+  auto p_full = [&](int b) { return bar_base + 8u * (2 * S + 4 + b); };
+  auto pv_done = [&](int b) { return bar_base + 8u * (2 * S + 6 + b); };   // PV of tile j commits to pv_done(j & 1)
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - base) + 8 * (2 * S + 8));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(s_free(b), 4); }
-    mbar_init(p_full, 4); mbar_init(pv_done, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(p_full(b), 4); mbar_init(pv_done(b), 1); }
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -176,15 +178,15 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       if (n_tiles > 0) ok = issue_s(0);
       for (int j = 0; j < n_tiles && ok; ++j) {
         if (j + 1 < n_tiles && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
-        if (!mbar_wait_or_abort(p_full, j & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_or_abort(p_full(j & 1), (j >> 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vt = kv_base + (j % S) * C::kStageBytes + C::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < kPosU / 16; ++ks)
-          tc_mma(tmem_base + kColO, smem_desc(p_base + ks * 32), smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128), C::kIdescPV,
+          tc_mma(tmem_base + kColO, smem_desc(p_base + (j & 1) * C::kPBytes + ks * 32), smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128), C::kIdescPV,
                  (j > 0 || ks > 0) ? 1u : 0u);
         tc_commit(kv_empty(j % S));                  // K_j and V_j are no longer needed
-        tc_commit(pv_done);                          // O holds tiles 0..j
+        tc_commit(pv_done(j & 1));                   // O holds tiles 0..j
       }
       if (!ok) *abort_flag = 1;
     }
@@ -230,32 +232,34 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       }
       l_run = l_run * corr + rs;
       m_ref = m_new;
-      if (j > 0) {                                   // O (tiles 0..j-1) must be complete before it is rescaled or P replaced
-        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, (j - 1) & 1, abort_flag));
+      if (j >= 2) {                                  // P buffer b was read by the PV product of tile j - 2
+        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done(b), ((j >> 1) - 1) & 1, abort_flag));
+        if (!ok) break;
+      }
+      if (j > 0 && __any_sync(0xffffffffu, raise)) { // rescale O: it must hold every earlier tile first
+        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done(b ^ 1), ((j - 1) >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, raise)) {
 #pragma unroll 1
-          for (int c = 0; c < HD / 32; ++c) {
-            float ov[32];
-            tmem_ld32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
+        for (int c = 0; c < HD / 32; ++c) {
+          float ov[32];
+          tmem_ld32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) ov[i] *= corr;
-            tmem_st32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
-          }
+          for (int i = 0; i < 32; ++i) ov[i] *= corr;
+          tmem_st32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
         }
       }
 #pragma unroll
       for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(gen_base + (p_base - base) + row * 128 + ((c ^ (row & 7)) << 4)) =
+        *reinterpret_cast<uint4*>(gen_base + (p_base - base) + b * C::kPBytes + row * 128 + ((c ^ (row & 7)) << 4)) =
             make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full);
+      if (lane == 0) mbar_arrive(p_full(b));
     }
     if (ok && n_tiles > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, (n_tiles - 1) & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done((n_tiles - 1) & 1), ((n_tiles - 1) >> 1) & 1, abort_flag));
       tc_fence_after();
     }
     if (!ok) { if (lane == 0) *abort_flag = 1; }
