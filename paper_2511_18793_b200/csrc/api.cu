@@ -76,6 +76,9 @@ struct nezha_ctx {
   // fused tensor-core path: RMSNorm split around the GEMMs (partial sums of squares per output tile), SwiGLU and
   // rotary embedding + KV append in GEMM epilogues; weights of q/k heads and gate/up re-laid-out to match
   bool fused; float *ss_a, *ss_b, *ss_e;
+  // draft head with merged products (fused path, default options): [W_logit_l ; W_s] per level, U = E W_e^T for every
+  // code token, H_l = W_logit_l h_l per request, the level's states as a bf16 A operand, the level's product
+  void* draft_wcat[kMaxLevels]; float* draft_u; float* draft_hl; void* draft_sact; float* draft_g;
   int* h_rows; unsigned long long* n_unique_dev;
   EngineState es;
   int* host_counters;       // pinned
@@ -212,7 +215,14 @@ size_t carve(nezha_ctx* c) {
   c->h_rows = cv.take<int>((size_t)c->Bmax * (c->L + 1));
   c->fused = c->bf16 && (c->hd == 64 || c->hd == 128) && c->d % 64 == 0 && c->F % 64 == 0;
   c->ss_a = c->ss_b = c->ss_e = nullptr;
+  c->draft_u = c->draft_hl = c->draft_g = nullptr; c->draft_sact = nullptr;
+  for (int l = 0; l < kMaxLevels; ++l) c->draft_wcat[l] = nullptr;
   if (c->fused) {
+    for (int l = 0; l < c->L; ++l) c->draft_wcat[l] = cv.take_bytes((size_t)(g.T[l] + c->d) * c->d * esz);
+    c->draft_u = cv.take<float>((size_t)li.vocab_codes * c->d);
+    c->draft_hl = cv.take<float>((size_t)c->L * c->Bmax * c->Tmax);
+    c->draft_sact = cv.take_bytes((size_t)c->Bmax * c->Kmax * c->d * esz);
+    c->draft_g = cv.take<float>((size_t)c->Bmax * c->Kmax * (c->Tmax + c->d));
     c->ss_a = cv.take<float>((size_t)(c->d / 32) * c->Ms);      // one partial sum per 32 columns
     c->ss_b = cv.take<float>((size_t)(c->d / 32) * c->Ms);
     c->ss_e = cv.take<float>((size_t)c->Ms);
@@ -396,17 +406,41 @@ SelectArgs select_base(nezha_ctx* c, int batch, int K) {
   return s;
 }
 
+// The draft head with its two per-level products merged into one (fused path, default options).  Eq. 2 is linear:
+// W_l (h_l + s_l) = W_l h_l + W_l s_l, and W_l h_l is a per-request constant (draft_hl, computed after the prefill);
+// Eq. 3's W_e e_l is a table look-up (draft_u) and its W_s s_l does not depend on which code gets chosen.  So one
+// product per level, s_l [W_l ; W_s]^T, yields the logits (before the selection) and the state term (used after it).
+bool draft_fast(const nezha_ctx* c) {
+  return c->fused && c->opt_transition == 0 && c->opt_inputs == 0;
+}
+void draft_level_product(nezha_ctx* c, int batch, int l, bool with_state) {
+  const int T = c->cfg.T[l - 1];
+  gemm(c, c->draft_sact, c->d, c->draft_wcat[l - 1], c->d, c->draft_g, c->Tmax + c->d, (long long)batch * c->Kmax, nullptr,
+       T + (with_state ? c->d : 0), c->d, kEpiStoreF32);
+}
+void draft_level_step(nezha_ctx* c, int batch, int l) {
+  launch_draft_step(c->es, batch, l, c->draft_g, c->Tmax + c->d, c->cfg.T[l - 1], c->draft_u, (const float*)c->draft_b_f32, c->draft_sact,
+                    c->st);
+}
+
 // Algorithm 3's inference loop (from the empty beam), or its continuation from the true beams (Algorithm 2's drafting step).
 // `first_level` = smallest level any request can still need drafting at (levels below are teacher-forced only).
 void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_level, bool filter) {
   const EngineState& e = c->es;
   launch_draft_init(e, batch, from_scratch ? 1 : 0, c->st);
+  const bool fast = draft_fast(c);
+  if (fast) launch_draft_state_init(e, batch, c->draft_sact, c->st);
   for (int l = 1; l <= c->L; ++l) {
+    if (fast && (l >= first_level || l < c->L)) draft_level_product(c, batch, l, l < c->L);
     if (l >= first_level) {
-      draft_logits_level(c, batch, l);
+      if (!fast) draft_logits_level(c, batch, l);
       SelectArgs s = select_base(c, batch, K);
       const size_t lv_in = (size_t)(l - 1) * c->Bmax * c->Kmax, lv_out = (size_t)l * c->Bmax * c->Kmax;
       s.logits = c->logits_d; s.row_stride = c->cfg.T[l - 1]; s.col_off = 0; s.src_row = nullptr; s.src_mul = c->Kmax;
+      if (fast) {
+        s.logits = c->draft_g; s.row_stride = c->Tmax + c->d;
+        s.logit_bias = c->draft_hl + (size_t)(l - 1) * c->Bmax * c->Tmax; s.bias_stride = c->Tmax;
+      }
       s.in_codes = e.dw_codes + lv_in * c->L; s.in_score = e.dw_score + lv_in; s.in_count = e.dw_count + (size_t)(l - 1) * c->Bmax;
       s.n = l - 1; s.T = c->cfg.T[l - 1]; s.per_beam = K < s.T ? K : s.T; s.filter = (filter && l == c->L) ? 1 : 0;
       s.gate = e.d_m; s.gate_mode = 2; s.gate_value = l;
@@ -414,7 +448,7 @@ void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_le
       s.out_token = nullptr; s.out_count = e.dw_count + (size_t)l * c->Bmax;
       launch_select(s, c->st);
     }
-    if (l < c->L) draft_transition_level(c, batch, l);
+    if (l < c->L) { if (fast) draft_level_step(c, batch, l); else draft_transition_level(c, batch, l); }
   }
 }
 
@@ -651,6 +685,14 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
     ok = cudaMemcpyAsync(c->es.n_tokens, &zero, sizeof(int), cudaMemcpyHostToDevice, st) == cudaSuccess;
     launch_embed(w->draft_b, c->bf16, c->es.n_tokens, 1, nullptr, c->d, (float*)c->draft_b_f32, st);
   }
+  if (ok && c->fused) {
+    // [W_logit_l ; W_s] per level, and U = E W_e^T (fp32) for every code token: Eq. 3's input term of a chosen code
+    for (int l = 0; ok && l < c->L; ++l)
+      ok = cp(c->draft_wcat[l], w->draft_logit[l], (size_t)cfg->T[l] * c->d * esz) &&
+           cp((char*)c->draft_wcat[l] + (size_t)cfg->T[l] * c->d * esz, w->draft_ws, (size_t)c->d * c->d * esz);
+    gemm(c, c->embed, c->d, (char*)c->draft_wse + (size_t)c->d * esz, 2 * c->d, c->draft_u, c->d, c->es.li.vocab_codes, nullptr,
+         c->d, c->d, kEpiStoreF32);
+  }
   // rotary tables in double precision on the host
   if (ok) {
     const int half = c->hd / 2, np = c->S + c->L;
@@ -722,6 +764,10 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
     const size_t ho = (size_t)b0 * (c->L + 1) * c->d;
     launch_rmsnorm(c->resid, c->d, c->h_rows, c->final_norm, c->bf16, (char*)c->h_act + ho * c->esz, c->h_f32 + ho,
                    rows * (c->L + 1), nullptr, c->d, c->cfg.rms_eps, c->st);
+    if (c->fused)                  // the request-constant half of Eq. 2: W_logit_l h_l for every level
+      for (int l = 1; l <= c->L; ++l)
+        gemm(c, (char*)c->h_act + (ho + (size_t)l * c->d) * c->esz, (long long)(c->L + 1) * c->d, c->draft_logit[l - 1], c->d,
+             c->draft_hl + ((size_t)(l - 1) * c->Bmax + b0) * c->Tmax, c->Tmax, rows, nullptr, c->cfg.T[l - 1], c->d, kEpiStoreF32);
   }
   NZ_CUDA(c, cudaGetLastError());
   c->batch = batch;
@@ -808,9 +854,17 @@ nezha_status nezha_draft_logits(nezha_ctx* c, int32_t batch, int32_t n_beams, in
                                    prefixes + (size_t)b * n_beams * level, (size_t)level * sizeof(int),
                                    (size_t)level * sizeof(int), (size_t)n_beams, cudaMemcpyDeviceToDevice, c->st));
   }
-  for (int l = 1; l <= level; ++l) draft_transition_level(c, batch, l);
-  draft_logits_level(c, batch, level + 1);
-  launch_copy_logits(c->logits_d, c->cfg.T[level], 0, nullptr, c->Kmax, 1, batch, n_beams, 0, c->cfg.T[level], logits, c->st);
+  if (draft_fast(c)) {
+    launch_draft_state_init(e, batch, c->draft_sact, c->st);
+    for (int l = 1; l <= level; ++l) { draft_level_product(c, batch, l, true); draft_level_step(c, batch, l); }
+    draft_level_product(c, batch, level + 1, false);
+    launch_copy_logits_bias(c->draft_g, c->Tmax + c->d, c->Kmax, batch, n_beams, c->cfg.T[level],
+                            c->draft_hl + (size_t)level * c->Bmax * c->Tmax, c->Tmax, logits, c->st);
+  } else {
+    for (int l = 1; l <= level; ++l) draft_transition_level(c, batch, l);
+    draft_logits_level(c, batch, level + 1);
+    launch_copy_logits(c->logits_d, c->cfg.T[level], 0, nullptr, c->Kmax, 1, batch, n_beams, 0, c->cfg.T[level], logits, c->st);
+  }
   NZ_CUDA(c, cudaGetLastError());
   return NEZHA_OK;
 }

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int t = lane + 32 * j;
-      key[j] = (t < a.T) ? z[t] : -INFINITY;
+      key[j] = (t < a.T) ? z[t] + (a.logit_bias ? a.logit_bias[(long long)b * a.bias_stride + t] : 0.f) : -INFINITY;
       mx = fmaxf(mx, key[j]);
     }
     mx = warp_max(mx);
@@ -357,6 +357,57 @@ __global__ void trans_gather_kernel(EngineState e, int batch, int l, const T* em
     if (ADD) { nxt[c] = s[c] + to_f32(emb[c]); }
     else { dst[c] = from_f32<T>(s[c]); dst[e.d + c] = emb[c]; }
   }
+}
+
+// ---- the draft head with merged products ---------------------------------------------------------------------
+// s_1 = h_0 (Eq. 1) for every beam slot of every request, as the bf16 A operand of the level's product.
+__global__ void draft_state_init_kernel(EngineState e, int batch, __nv_bfloat16* s_act) {
+  pdl_wait();
+  pdl_launch();
+  const int bk = blockIdx.x, b = bk / e.Kmax;
+  if (b >= batch) return;
+  const float* h0 = e.h_f32 + (long long)b * (e.L + 1) * e.d;
+  for (int c = threadIdx.x; c < e.d; c += blockDim.x) s_act[(long long)bk * e.d + c] = __float2bfloat16_rn(h0[c]);
+}
+
+// Eq. 3 after the product: s_{l+1}[k] = tanh((W_s s_l)[parent] + (W_e E)[code] + b).  G holds [logits | W_s s_l] of
+// every beam slot of level l (W_s s_l from column t_cols on), U = W_e E for every code token.  Which (parent, code) a
+// slot takes is decided exactly as in trans_gather_kernel.
+__global__ void draft_step_kernel(EngineState e, int batch, int l, const float* __restrict__ G, long long g_stride, int t_cols,
+                                  const float* __restrict__ U, const float* __restrict__ bias, __nv_bfloat16* s_act) {
+  pdl_wait();
+  pdl_launch();
+  const int bk = blockIdx.x;
+  const int b = bk / e.Kmax, k = bk - b * e.Kmax;
+  if (b >= batch) return;
+  __nv_bfloat16* dst = s_act + (long long)bk * e.d;
+  const int dm = e.d_m[b];
+  int src_level, parent;
+  bool live = dm < e.L || e.row_m[b] < e.L;
+  if (dm >= l) { src_level = min(dm, e.L); parent = k; }
+  else { src_level = l; parent = -2; }
+  const long long s_idx = lvl_bk(e, src_level, b, k);
+  live = live && k < e.dw_count[src_level * e.Bmax + b];
+  if (live && parent == -2) parent = e.dw_parent[s_idx];
+  const int code = live ? e.dw_codes[s_idx * e.L + (l - 1)] : -1;
+  live = live && code >= 0 && parent >= 0;
+  if (!live) {
+    for (int c = threadIdx.x; c < e.d; c += blockDim.x) dst[c] = __float2bfloat16_rn(0.f);
+    return;
+  }
+  const float* z = G + ((long long)b * e.Kmax + parent) * g_stride + t_cols;
+  const float* u = U + (long long)(e.li.off[l - 1] + code) * e.d;
+  for (int c = threadIdx.x; c < e.d; c += blockDim.x) dst[c] = __float2bfloat16_rn(tanhf(z[c] + u[c] + bias[c]));
+}
+
+// dst[b, r, :] = src[(b * row_mul + r), 0 : T] + bias[b, :]
+__global__ void copy_logits_bias_kernel(const float* src, long long row_stride, int row_mul, int n_beams, int T,
+                                        const float* bias, long long bias_stride, float* dst) {
+  pdl_wait();
+  pdl_launch();
+  const int b = blockIdx.x / n_beams, r = blockIdx.x % n_beams;
+  const float* z = src + ((long long)b * row_mul + r) * row_stride;
+  for (int t = threadIdx.x; t < T; t += blockDim.x) dst[(long long)blockIdx.x * T + t] = z[t] + bias[(long long)b * bias_stride + t];
 }
 
 // ----------------------------------------------------------------------------------------------------
@@ -706,6 +757,22 @@ void launch_trans_add(const EngineState& e, int batch, int l, const void* embed,
   else
     launch_pdl(trans_gather_kernel<float, true>, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, (const float*)embed,
                (float*)nullptr);
+}
+void launch_draft_state_init(const EngineState& e, int batch, void* s_act, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
+  launch_pdl(draft_state_init_kernel, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, (__nv_bfloat16*)s_act);
+}
+void launch_draft_step(const EngineState& e, int batch, int l, const float* G, long long g_stride, int t_cols, const float* U,
+                       const float* bias, void* s_act, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
+  launch_pdl(draft_step_kernel, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, G, g_stride, t_cols, U, bias,
+             (__nv_bfloat16*)s_act);
+}
+void launch_copy_logits_bias(const float* src, long long row_stride, int row_mul, int batch, int n_beams, int T,
+                             const float* bias, long long bias_stride, float* dst, cudaStream_t st) {
+  LaunchScope ls(kcMisc, st);
+  launch_pdl(copy_logits_bias_kernel, dim3(batch * n_beams), dim3(128), 0, st, src, row_stride, row_mul, n_beams, T, bias,
+             bias_stride, dst);
 }
 void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st) {
   LaunchScope ls(kcNodes, st, 2);

@@ -58,6 +58,7 @@ struct SelectArgs {
   int n;                                // codes the input beams have; the level's codebook is T[n]
   int T, K, per_beam, filter;
   const int* gate; int gate_mode, gate_value;   // 0: none, 1: run iff gate[b] == value, 2: run iff gate[b] < value
+  const float* logit_bias; long long bias_stride;   // optional: logits of request b get logit_bias[b * bias_stride + t] added
   int* out_codes; int* out_token; float* out_score; int* out_parent; int* out_count; int out_stride;
   int tuple_len;                        // row length of in_codes / out_codes (L)
   int batch;
@@ -74,6 +75,12 @@ void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, 
 void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
                          cudaStream_t st);
 void launch_trans_add(const EngineState& e, int batch, int l, const void* embed, bool bf16, cudaStream_t st);
+// The draft head with its two per-level products merged (see DraftFast in api.cu)
+void launch_draft_state_init(const EngineState& e, int batch, void* s_act, cudaStream_t st);
+void launch_draft_step(const EngineState& e, int batch, int l, const float* G, long long g_stride, int t_cols, const float* U,
+                       const float* bias, void* s_act, cudaStream_t st);
+void launch_copy_logits_bias(const float* src, long long row_stride, int row_mul, int batch, int n_beams, int T,
+                             const float* bias, long long bias_stride, float* dst, cudaStream_t st);
 void launch_build_nodes(const EngineState& e, int batch, cudaStream_t st);
 void launch_nodes_from_prefixes(const EngineState& e, int batch, int n_beams, int level, const int* prefixes,
                                 cudaStream_t st);
