@@ -196,10 +196,20 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
     float m_ref = -INFINITY, l_run = 0.f;           // reference maximum (scaled log2 domain) and row sum against it
     bool ok = true;
     const int ctx_min = __reduce_min_sync(0xffffffffu, ctx);
+    const bool warp_dead = r0 + (warp & 3) * 32 >= R;   // none of this warp's 32 rows exists: it only keeps the barriers going
     for (int j = 0; j < n_tiles; ++j) {
       const int b = j & 1;
       ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full(b), (j >> 1) & 1, abort_flag));
       if (!ok) break;
+      if (warp_dead) {                               // (its P rows stay whatever they are: O rows nobody reads)
+        if (lane == 0) mbar_arrive(s_free(b));
+        if (j >= 2) {
+          ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done(b), ((j >> 1) - 1) & 1, abort_flag));
+          if (!ok) break;
+        }
+        if (lane == 0) mbar_arrive(p_full(b));
+        continue;
+      }
       tc_fence_after();
       float sv[kPosU];
       tmem_ld32(tmem_base + lane_addr + kColS + (uint32_t)(b * kPosU), sv);

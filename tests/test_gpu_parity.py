@@ -6,7 +6,7 @@ import torch
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
 from helpers import codes_of
-from gpu_helpers import Case, assert_topk_matches, tolerance
+from gpu_helpers import Case, assert_topk_matches, check_levels, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -306,3 +306,74 @@ def test_draft_head_variants(name, variant):
         case.eng.set_option(7, 0)
     with pytest.raises(case.binding.NezhaError):
         case.eng.set_option(1, 3)
+
+
+# ---------------------------------------------------------------------------------------- the library's size limits
+def test_maximum_beam_and_codebook_sizes():
+    """Beam 128 over codebooks of 1024 codes (both the largest the library takes): every mode against the oracle."""
+    w = synth.scaled(synth.WORKLOADS["tiny"], L=2, T=(1024, 1024), n_items=30_000, batch=2, beam=128, n_hist=6)
+    case = Case(w).prefill()
+    model, head, V = case.oracle
+    tol = tolerance(w)
+    ar = case.eng.decode(w.beam, mode=2)
+    sp = case.eng.decode(w.beam, mode=1)
+    dr = case.eng.decode(w.beam, mode=0)
+    assert torch.equal(ar["codes"], sp["codes"]) and torch.equal(ar["count"], sp["count"])
+    for b in range(w.batch):
+        ref = O.ar_beam_search(model, case.req(b), w.beam, V)[-1]
+        assert_topk_matches(*(ar[k][b].cpu().numpy() for k in ("codes", "scores", "count")), ref, w.beam, tol)
+        ref = O.nezha_draft(head, case.req(b), w.beam, V)[-1]
+        assert_topk_matches(*(dr[k][b].cpu().numpy() for k in ("codes", "scores", "count")), ref, w.beam, tol)
+    assert int(ar["count"].min()) == w.beam                        # 30 000 items: every request fills its beam
+
+
+def test_maximum_number_of_levels():
+    """L = 8 codes per item (NEZHA_MAX_LEVELS) over codebooks of 4: seven verification levels, Eq. 4 with eight digits."""
+    w = synth.scaled(synth.WORKLOADS["tiny"], L=8, T=(4,) * 8, n_items=9_000, batch=3, beam=6, n_hist=5)
+    case = Case(w).prefill()
+    model, head, V = case.oracle
+    probe = synth.probe_keys_mix(w, case.catalog, 20_000)
+    keys = case.eng.pack(torch.from_numpy(probe).cuda())
+    assert np.array_equal(keys.cpu().numpy().view(np.uint64), O.pack_keys(probe, w.T))
+    assert np.array_equal(case.eng.probe(keys).cpu().numpy().astype(bool), V.contains(probe))
+    ar = case.eng.decode(w.beam, mode=2)
+    sp = case.eng.decode(w.beam, mode=1, trace=True)
+    dr = case.eng.decode(w.beam, mode=0)
+    assert torch.equal(ar["codes"], sp["codes"]) and torch.equal(ar["count"], sp["count"])
+    assert 1 <= sp["stats"].rounds <= w.L - 1
+    beams, scores = sp["trace"]["beams"].cpu().numpy(), sp["trace"]["beam_scores"].cpu().numpy()
+    for b in range(w.batch):
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam)
+        ref = O.ar_beam_search(model, case.req(b), w.beam, V)[-1]
+        assert_topk_matches(*(ar[k][b].cpu().numpy() for k in ("codes", "scores", "count")), ref, w.beam, tolerance(w))
+        ref = O.nezha_draft(head, case.req(b), w.beam, V)[-1]
+        assert_topk_matches(*(dr[k][b].cpu().numpy() for k in ("codes", "scores", "count")), ref, w.beam, tolerance(w))
+
+
+def test_one_item_catalogue_and_beam_wider_than_it():
+    """A catalogue of one item under a beam that keeps every prefix (64 beams over 8 x 8 x 8 codes): every mode returns
+    that item alone (count 1, the other beam slots -1).  Under a narrow beam the item's prefix may be pruned before the
+    last level, where alone validity is checked, so the result may be empty: it must equal the oracle's.  A single level
+    L = 1 has no prefix to verify at all."""
+    catalog = np.array([[3, 1, 4]], dtype=np.int32)
+    for beam in (64, 3):
+        w = synth.scaled(synth.WORKLOADS["tiny"], T=(8, 8, 8), n_items=1, batch=2, beam=beam)
+        hist = np.tile(catalog[None], (w.batch, 5, 1)).astype(np.int32)
+        case = Case(w, catalog=catalog, hist=hist).prefill()
+        model, head, V = case.oracle
+        assert case.n_unique == 1
+        for mode in (0, 1, 2):
+            out = case.eng.decode(w.beam, mode=mode)
+            codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
+            for b in range(w.batch):
+                ref = (O.nezha_draft(head, case.req(b), beam, V) if mode == 0 else O.ar_beam_search(model, case.req(b), beam, V))[-1]
+                assert count[b] == len(ref) and (beam == 3 or count[b] == 1)
+                assert np.all(codes[b, : count[b]] == catalog[0]) and np.all(codes[b, count[b]:] == -1)
+    w1 = synth.scaled(synth.WORKLOADS["tiny"], L=1, T=(32,), n_items=20, batch=2, beam=5)
+    c1 = Case(w1).prefill()
+    model, head, V = c1.oracle
+    for mode in (0, 1, 2):
+        out = c1.eng.decode(w1.beam, mode=mode)
+        for b in range(w1.batch):
+            ref = (O.nezha_draft(head, c1.req(b), w1.beam, V) if mode == 0 else O.ar_beam_search(model, c1.req(b), w1.beam, V))[-1]
+            assert_topk_matches(*(out[k][b].cpu().numpy() for k in ("codes", "scores", "count")), ref, w1.beam, tolerance(w1))
