@@ -152,7 +152,11 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
 
   pdl_wait();                                       // before the first global read and before any exit
   pdl_launch();
-  const int req_local = blockIdx.z, kvh = blockIdx.y, tile = blockIdx.x;
+  // the row tile is the slowest grid index: tiles beyond a request's rows (the grid covers the largest row count a
+  // call may have) are scheduled after every tile that has work, instead of holding its place in the first wave
+  // (a causal prefill has no such tiles to speak of, and its last tiles see the most context: those go first)
+  const int req_local = blockIdx.y, kvh = blockIdx.x;
+  const int tile = a.n_ext_max > 0 ? (int)blockIdx.z : (int)(gridDim.z - 1 - blockIdx.z);
   const int G = a.Hq / a.Hkv;
   const int4 info = a.req_info[req_local];          // {first token, token count, cache row, context length or -1}
   const int tok0 = info.x, n_tok = info.y, request = info.z;
@@ -389,7 +393,7 @@ void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cud
     configured = true;
   }
   const int G = a.Hq / a.Hkv;
-  dim3 grid((a.max_tokens_per_row * G + 16 * RW - 1) / (16 * RW), a.Hkv, a.n_rows);
+  dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + 16 * RW - 1) / (16 * RW));
   launch_pdl(attn_tc_kernel<HD, RW, KW>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *tk, *tv, a, a.status);
 }
 
@@ -398,7 +402,7 @@ void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cud
 void launch_attention_umma(const AttnArgs& a, const CUtensorMap* tk, const CUtensorMap* tv, cudaStream_t st);
 
 bool attention_tc_supported(const AttnArgs& a) {
-  if (!a.status || !a.req_info || a.n_rows <= 0 || a.max_tokens_per_row <= 0) return false;
+  if (!a.status || !a.req_info || a.n_rows <= 0 || a.n_rows > 65535 || a.max_tokens_per_row <= 0) return false;
   if (a.hd != 64 && a.hd != 128) return false;
   if (!tma_encode_fn()) return false;
   if (a.ctx_head_stride % a.hd || a.ctx_row_stride != a.ctx_head_stride * a.Hkv) return false;

@@ -75,7 +75,11 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
 
   pdl_wait();                                       // before the first global read and before any exit
   pdl_launch();
-  const int req_local = blockIdx.z, kvh = blockIdx.y, tile = blockIdx.x;
+  // the row tile is the slowest grid index: tiles beyond a request's rows (the grid covers the largest row count a
+  // call may have) are scheduled after every tile that has work, instead of holding its place in the first wave
+  // (a causal prefill has no such tiles to speak of, and its last tiles see the most context: those go first)
+  const int req_local = blockIdx.y, kvh = blockIdx.x;
+  const int tile = a.n_ext_max > 0 ? (int)blockIdx.z : (int)(gridDim.z - 1 - blockIdx.z);
   const int G = a.Hq / a.Hkv;
   const int4 info = a.req_info[req_local];          // {first token, token count, cache row, context length or -1}
   const int tok0 = info.x, n_tok = info.y, request = info.z;
@@ -366,7 +370,7 @@ void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a
     configured = true;
   }
   const int G = a.Hq / a.Hkv;
-  dim3 grid((a.max_tokens_per_row * G + kRowsU - 1) / kRowsU, a.Hkv, a.n_rows);
+  dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + kRowsU - 1) / kRowsU);
   launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, a, a.status);
 }
 

@@ -63,6 +63,8 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kEpiWarps); }
     *abort_flag = 0;
     mbar_fence_init();
+    tma_prefetch_map(&tmA);
+    tma_prefetch_map(&tmB);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
@@ -84,15 +86,19 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int it = 0;                                // k-iterations issued so far, over all tiles
+      int s = 0;                                 // it % STAGES, and the parity of slot s's current round
+      uint32_t round = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
         for (int k = 0; k < k_iters; ++k, ++it) {
-          const int s = it % STAGES;
-          if (it >= STAGES && !mbar_wait_or_abort(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), C::kStageBytes);
-          tma_load_2d(base + s * C::kStageBytes, &tmA, k * BK, m0, full_bar(s));
-          tma_load_2d(base + s * C::kStageBytes + kTileBytesA, &tmB, k * BK, n0, full_bar(s));
+          // (waiting for the parity before the first one succeeds at once on a fresh barrier: round 0 never waits)
+          if (!mbar_wait_or_abort(empty_bar(s), round ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = full_bar(s), dst = base + s * C::kStageBytes;
+          mbar_expect_tx(fb, C::kStageBytes);
+          tma_load_2d(dst, &tmA, k * BK, m0, fb);
+          tma_load_2d(dst + kTileBytesA, &tmB, k * BK, n0, fb);
+          if (++s == STAGES) { s = 0; round ^= 1u; }
         }
       }
       if (!ok) {                                 // drain: wait (bounded) for the copies still in flight
@@ -103,22 +109,24 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int it = 0, t_local = 0;
+      int t_local = 0, s = 0;
+      uint32_t round = 0;
       bool ok = true;
+      // descriptors of slot 0; a slot further on adds its byte offset / 16 to the address field (shared memory
+      // addresses stay below 2^18, so the 14-bit field never carries)
+      const uint64_t da0 = smem_desc(base), db0 = smem_desc(base + kTileBytesA);
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
         const int b = t_local & 1;
         if (t_local >= 2 && !mbar_wait_or_abort(acc_empty(b), ((t_local >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_acc = tmem_base + (uint32_t)(b * BN);
-        for (int k = 0; k < k_iters; ++k, ++it) {
-          const int s = it % STAGES;
-          if (!mbar_wait_or_abort(full_bar(s), (it / STAGES) & 1, abort_flag)) { ok = false; break; }
+        for (int k = 0; k < k_iters; ++k) {
+          if (!mbar_wait_or_abort(full_bar(s), round, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + s * C::kStageBytes, sb = sa + kTileBytesA;
-#pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            tc_mma(tmem_acc, smem_desc(sa + kk * 32), smem_desc(sb + kk * 32), C::kInstrDesc, (k > 0 || kk > 0) ? 1u : 0u);
+          const uint64_t so = (uint64_t)(s * (C::kStageBytes >> 4));
+          tc_mma_kstep(tmem_acc, da0 + so, db0 + so, C::kInstrDesc, k > 0 ? 1u : 0u);
           tc_commit(empty_bar(s));               // slot free once these MMAs have read it
+          if (++s == STAGES) { s = 0; round ^= 1u; }
         }
         if (ok) tc_commit(acc_full(b));          // accumulator complete
       }

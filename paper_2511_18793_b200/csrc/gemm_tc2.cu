@@ -40,12 +40,20 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(leader_bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+// The four MMAs (K = 16 each) of one 64-deep k-step over the pair, in one statement (see tc_mma_kstep).
+__device__ __forceinline__ void tc_mma_pair_kstep(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate_first) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, t;\n\t.reg .b64 a1, b1, a2, b2, a3, b3;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(kInstrDesc2), "r"(accumulate) : "memory");
+      "setp.eq.b32 t, %4, %4;\n\t"
+      "add.s64 a1, %1, 2;\n\tadd.s64 b1, %2, 2;\n\t"
+      "add.s64 a2, %1, 4;\n\tadd.s64 b2, %2, 4;\n\t"
+      "add.s64 a3, %1, 6;\n\tadd.s64 b3, %2, 6;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, t;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a2, b2, %3, t;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a3, b3, %3, t;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(kInstrDesc2), "r"(accumulate_first) : "memory");
 }
 // Arrives (once the MMAs issued so far have completed) on the barrier at this offset in BOTH CTAs of the pair.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
@@ -84,6 +92,8 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_pair_kernel(const __grid_con
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 2 * kEpiWarps); }
     *abort_flag = 0;
     mbar_fence_init();
+    tma_prefetch_map(&tmA);
+    tma_prefetch_map(&tmB);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
@@ -105,17 +115,20 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_pair_kernel(const __grid_con
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
-      int it = 0;
+      int s = 0;
+      uint32_t round = 0;
       bool ok = true;
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
         const int m0 = (tile % tiles_m) * (2 * BM) + rank * BM;          // this CTA's rows
         const int nb0 = (tile / tiles_m) * kBN2 + rank * (kBN2 / 2);     // this CTA's half of the W tile
-        for (int k = 0; k < k_iters; ++k, ++it) {
-          const int s = it % STAGES;
-          if (it >= STAGES && !mbar_wait_or_abort(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag)) { ok = false; break; }
+        for (int k = 0; k < k_iters; ++k) {
+          // (round 0 never waits: the parity before a fresh barrier's first one counts as complete)
+          if (!mbar_wait_or_abort(empty_bar(s), round ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t dst = base + s * kStageBytes2, fb = full_bar(s) & kLeaderMask;
           if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStageBytes2);  // the bytes of both CTAs' copies
-          tma_load_2d_pair(base + s * kStageBytes2, &tmA, k * BK, m0, full_bar(s) & kLeaderMask);
-          tma_load_2d_pair(base + s * kStageBytes2 + kTileBytesA, &tmB, k * BK, nb0, full_bar(s) & kLeaderMask);
+          tma_load_2d_pair(dst, &tmA, k * BK, m0, fb);
+          tma_load_2d_pair(dst + kTileBytesA, &tmB, k * BK, nb0, fb);
+          if (++s == STAGES) { s = 0; round ^= 1u; }
         }
       }
       if (!ok) *abort_flag = 1;
@@ -123,22 +136,22 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_pair_kernel(const __grid_con
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
     if (lane == 0 && rank == 0) {
-      int it = 0, t_local = 0;
+      int t_local = 0, s = 0;
+      uint32_t round = 0;
       bool ok = true;
+      const uint64_t da0 = smem_desc(base), db0 = smem_desc(base + kTileBytesA);   // slot 0; later slots add to the address field
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++t_local) {
         const int b = t_local & 1;
         if (t_local >= 2 && !mbar_wait_or_abort(acc_empty(b), ((t_local >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_acc = tmem_base + (uint32_t)(b * kBN2);
-        for (int k = 0; k < k_iters; ++k, ++it) {
-          const int s = it % STAGES;
-          if (!mbar_wait_or_abort(full_bar(s), (it / STAGES) & 1, abort_flag)) { ok = false; break; }
+        for (int k = 0; k < k_iters; ++k) {
+          if (!mbar_wait_or_abort(full_bar(s), round, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + s * kStageBytes2, sb = sa + kTileBytesA;
-#pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            tc_mma_pair(tmem_acc, smem_desc(sa + kk * 32), smem_desc(sb + kk * 32), (k > 0 || kk > 0) ? 1u : 0u);
+          const uint64_t so = (uint64_t)(s * (kStageBytes2 >> 4));
+          tc_mma_pair_kstep(tmem_acc, da0 + so, db0 + so, k > 0 ? 1u : 0u);
           tc_commit_pair(empty_bar(s));          // slot free in both CTAs once these MMAs have read it
+          if (++s == STAGES) { s = 0; round ^= 1u; }
         }
         if (ok) tc_commit_pair(acc_full(b));     // accumulator complete, in both CTAs
       }
