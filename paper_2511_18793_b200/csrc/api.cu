@@ -427,9 +427,8 @@ void draft_level_step(nezha_ctx* c, int batch, int l) {
 // `first_level` = smallest level any request can still need drafting at (levels below are teacher-forced only).
 void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_level, bool filter) {
   const EngineState& e = c->es;
-  launch_draft_init(e, batch, from_scratch ? 1 : 0, c->st);
   const bool fast = draft_fast(c);
-  if (fast) launch_draft_state_init(e, batch, c->draft_sact, c->st);
+  launch_draft_init(e, batch, from_scratch ? 1 : 0, fast ? c->draft_sact : nullptr, c->st);
   for (int l = 1; l <= c->L; ++l) {
     if (fast && (l >= first_level || l < c->L)) draft_level_product(c, batch, l, l < c->L);
     if (l >= first_level) {
@@ -446,6 +445,11 @@ void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_le
       s.gate = e.d_m; s.gate_mode = 2; s.gate_value = l;
       s.out_codes = e.dw_codes + lv_out * c->L; s.out_score = e.dw_score + lv_out; s.out_parent = e.dw_parent + lv_out;
       s.out_token = nullptr; s.out_count = e.dw_count + (size_t)l * c->Bmax;
+      if (fast && l < c->L) {                      // the selection and the state update it feeds, in one launch
+        launch_select_step(s, e, l, c->draft_g, c->Tmax + c->d, c->cfg.T[l - 1], c->draft_u, (const float*)c->draft_b_f32,
+                           c->draft_sact, c->st);
+        continue;
+      }
       launch_select(s, c->st);
     }
     if (l < c->L) { if (fast) draft_level_step(c, batch, l); else draft_transition_level(c, batch, l); }
@@ -561,7 +565,6 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     // drafts are mostly rejected or mostly accepted in a steady workload, so the round's token count repeats: tile for it
     c->m_expected = c->m_seen[round];
     rs = run_segment(c, key_of(round), [&] {
-      launch_fill_i32(e.counters, 8, 0, c->st);
       if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
       else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
       else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, c->opt_filter != 0);
@@ -577,8 +580,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
         s.gate = e.row_cur; s.gate_mode = 1; s.gate_value = n;
         s.out_codes = e.tb_codes + lv_out * L; s.out_score = e.tb_score + lv_out; s.out_parent = e.tb_parent + lv_out;
         s.out_count = e.tb_count + (size_t)(n + 1) * c->Bmax;
-        launch_select(s, c->st);
-        launch_advance(e, batch, n, K, out_codes, out_scores, out_count, c->st);
+        launch_select_advance(s, e, n, K, out_codes, out_scores, out_count, c->st);
       }
       launch_round_end(e, batch, K, round, tr, c->st);
       cudaMemcpyAsync(c->host_counters, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st);

@@ -38,9 +38,7 @@ __device__ __forceinline__ float from_ordered_bits(unsigned o) {
 constexpr unsigned kOrderedNegInf = 0x007fffffu;          // ordered_bits(-inf)
 
 template <int VPL>
-__global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
-  pdl_wait();
-  pdl_launch();
+__device__ __forceinline__ void select_body(const SelectArgs& a) {
   const int b = blockIdx.x;
   if (a.gate_mode == 1 && a.gate[b] != a.gate_value) return;
   if (a.gate_mode == 2 && !(a.gate[b] < a.gate_value)) return;
@@ -202,7 +200,16 @@ __global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
   if (lane == 0) a.out_count[b] = n_out;
 }
 
+template <int VPL>
+__global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
+  pdl_wait();
+  pdl_launch();
+  select_body<VPL>(a);
+}
+
 }  // namespace
+
+cudaError_t select_step_configure(int bytes);
 
 size_t select_smem_bytes(int in_stride, int K) {
   return (size_t)in_stride * K * (sizeof(float) + sizeof(int)) + (size_t)in_stride * sizeof(int);
@@ -214,7 +221,8 @@ cudaError_t select_configure(int max_beam) {
   if ((e = cudaFuncSetAttribute(select_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
   if ((e = cudaFuncSetAttribute(select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
   if ((e = cudaFuncSetAttribute(select_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
-  return cudaFuncSetAttribute(select_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if ((e = cudaFuncSetAttribute(select_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  return select_step_configure(bytes);
 }
 
 void launch_select(const SelectArgs& a, cudaStream_t st) {
@@ -267,11 +275,22 @@ __global__ void init_decode_kernel(EngineState e, int batch) {
 
 // Start of a round's drafting (Algorithm 2's drafting step): the draft head continues from the true beams B_m, or from
 // the empty beam in the first round (Algorithm 3's initialisation).
-__global__ void draft_init_kernel(EngineState e, int batch, int from_scratch) {
+// Also clears the round's counters (this is the first kernel of a drafting round) and, when s_act is given, starts
+// every beam slot's draft state at s_1 = h_0 (Eq. 1).
+__global__ void draft_init_kernel(EngineState e, int batch, int from_scratch, __nv_bfloat16* s_act) {
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x;
+  if (b == 0 && threadIdx.x < 8) e.counters[threadIdx.x] = 0;
   if (b >= batch) return;
+  if (s_act) {
+    const float* h0 = e.h_f32 + (long long)b * (e.L + 1) * e.d;
+    __nv_bfloat16* dst = s_act + (long long)b * e.Kmax * e.d;
+    for (int c = threadIdx.x; c < e.d; c += blockDim.x) {
+      const __nv_bfloat16 v = __float2bfloat16_rn(h0[c]);
+      for (int k = 0; k < e.Kmax; ++k) dst[(long long)k * e.d + c] = v;
+    }
+  }
   const int m = e.row_m[b];
   if (m >= e.L) { if (threadIdx.x == 0) { e.d_m[b] = e.L; e.dw_count[(long long)e.L * e.Bmax + b] = 0; } return; }
   const int mm = from_scratch ? 0 : m;
@@ -291,6 +310,7 @@ __global__ void draft_set_kernel(EngineState e, int batch, int K, const int* dra
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x;
+  if (b == 0 && threadIdx.x < 8) e.counters[threadIdx.x] = 0;      // first kernel of the round: clear its counters
   if (b >= batch) return;
   const int cnt = (drafts && e.row_m[b] < e.L) ? max(0, min(n_draft[b], K)) : 0;
   for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
@@ -373,14 +393,10 @@ __global__ void draft_state_init_kernel(EngineState e, int batch, __nv_bfloat16*
 // Eq. 3 after the product: s_{l+1}[k] = tanh((W_s s_l)[parent] + (W_e E)[code] + b).  G holds [logits | W_s s_l] of
 // every beam slot of level l (W_s s_l from column t_cols on), U = W_e E for every code token.  Which (parent, code) a
 // slot takes is decided exactly as in trans_gather_kernel.
-__global__ void draft_step_kernel(EngineState e, int batch, int l, const float* __restrict__ G, long long g_stride, int t_cols,
-                                  const float* __restrict__ U, const float* __restrict__ bias, __nv_bfloat16* s_act) {
-  pdl_wait();
-  pdl_launch();
-  const int bk = blockIdx.x;
-  const int b = bk / e.Kmax, k = bk - b * e.Kmax;
-  if (b >= batch) return;
-  __nv_bfloat16* dst = s_act + (long long)bk * e.d;
+__device__ __forceinline__ void draft_step_slot(const EngineState& e, int b, int k, int l, const float* __restrict__ G,
+                                                long long g_stride, int t_cols, const float* __restrict__ U,
+                                                const float* __restrict__ bias, __nv_bfloat16* s_act, int tid, int n_thr) {
+  __nv_bfloat16* dst = s_act + ((long long)b * e.Kmax + k) * e.d;
   const int dm = e.d_m[b];
   int src_level, parent;
   bool live = dm < e.L || e.row_m[b] < e.L;
@@ -392,12 +408,34 @@ __global__ void draft_step_kernel(EngineState e, int batch, int l, const float* 
   const int code = live ? e.dw_codes[s_idx * e.L + (l - 1)] : -1;
   live = live && code >= 0 && parent >= 0;
   if (!live) {
-    for (int c = threadIdx.x; c < e.d; c += blockDim.x) dst[c] = __float2bfloat16_rn(0.f);
+    for (int c = tid; c < e.d; c += n_thr) dst[c] = __float2bfloat16_rn(0.f);
     return;
   }
   const float* z = G + ((long long)b * e.Kmax + parent) * g_stride + t_cols;
   const float* u = U + (long long)(e.li.off[l - 1] + code) * e.d;
-  for (int c = threadIdx.x; c < e.d; c += blockDim.x) dst[c] = __float2bfloat16_rn(tanhf(z[c] + u[c] + bias[c]));
+  for (int c = tid; c < e.d; c += n_thr) dst[c] = __float2bfloat16_rn(tanhf(z[c] + u[c] + bias[c]));
+}
+__global__ void draft_step_kernel(EngineState e, int batch, int l, const float* __restrict__ G, long long g_stride, int t_cols,
+                                  const float* __restrict__ U, const float* __restrict__ bias, __nv_bfloat16* s_act) {
+  pdl_wait();
+  pdl_launch();
+  const int bk = blockIdx.x;
+  const int b = bk / e.Kmax, k = bk - b * e.Kmax;
+  if (b >= batch) return;
+  draft_step_slot(e, b, k, l, G, g_stride, t_cols, U, bias, s_act, threadIdx.x, blockDim.x);
+}
+// The selection of draft level l and the state update that follows it, in one launch: a block selects its request's
+// beams (or skips that when the request's level is already settled) and then advances the states of its own slots.
+template <int VPL>
+__global__ void __launch_bounds__(512) select_step_kernel(SelectArgs a, EngineState e, int l, const float* __restrict__ G,
+                                                          long long g_stride, int t_cols, const float* __restrict__ U,
+                                                          const float* __restrict__ bias, __nv_bfloat16* s_act) {
+  pdl_wait();
+  pdl_launch();
+  select_body<VPL>(a);
+  __syncthreads();                                 // the block's own selection (global writes) is visible to all its threads
+  for (int k = threadIdx.x >> 5; k < e.Kmax; k += blockDim.x >> 5)          // a warp per beam slot
+    draft_step_slot(e, blockIdx.x, k, l, G, g_stride, t_cols, U, bias, s_act, threadIdx.x & 31, 32);
 }
 
 // dst[b, r, :] = src[(b * row_mul + r), 0 : T] + bias[b, :]
@@ -564,9 +602,7 @@ __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams
 //                KV rows simply become unreachable) and is matched against the alive drafts.  If every beam is
 //                the (n+1)-prefix of a draft, its hidden state is already in the pass and selection goes on;
 //                else level n+1 is the rejection level and the request waits for the next round.
-__global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count) {
-  pdl_wait();
-  pdl_launch();
+__device__ __forceinline__ void advance_body(const EngineState& e, int n, int K, int* out_codes, float* out_score, int* out_count) {
   const int b = blockIdx.x;
   if (e.row_cur[b] != n) return;
   const int L = e.L, Kmax = e.Kmax;
@@ -618,6 +654,21 @@ __global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_
       out_count[b] = 0;
     }
   }
+}
+__global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count) {
+  pdl_wait();
+  pdl_launch();
+  advance_body(e, n, K, out_codes, out_score, out_count);
+}
+// The selection of B_{n+1} and the step above in one launch (both act on the requests whose current level is n).
+template <int VPL>
+__global__ void __launch_bounds__(512) select_advance_kernel(SelectArgs a, EngineState e, int n, int K, int* out_codes,
+                                                             float* out_score, int* out_count) {
+  pdl_wait();
+  pdl_launch();
+  select_body<VPL>(a);
+  __syncthreads();                                 // the block's own selection (global writes) is visible to all its threads
+  advance_body(e, n, K, out_codes, out_score, out_count);
 }
 
 // End of a round: accepted length of every draft = the largest i <= (level reached) with D[k][0..i) in B_i;
@@ -728,9 +779,9 @@ void launch_init_decode(const EngineState& e, int batch, cudaStream_t st) {
   LaunchScope ls(kcMisc, st);
   launch_pdl(init_decode_kernel, dim3((batch + 127) / 128), dim3(128), 0, st, e, batch);
 }
-void launch_draft_init(const EngineState& e, int batch, int from_scratch, cudaStream_t st) {
+void launch_draft_init(const EngineState& e, int batch, int from_scratch, void* s_act, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
-  launch_pdl(draft_init_kernel, dim3(batch), dim3(64), 0, st, e, batch, from_scratch);
+  launch_pdl(draft_init_kernel, dim3(batch), dim3(128), 0, st, e, batch, from_scratch, (__nv_bfloat16*)s_act);
 }
 void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
@@ -768,6 +819,30 @@ void launch_draft_step(const EngineState& e, int batch, int l, const float* G, l
   launch_pdl(draft_step_kernel, dim3(batch * e.Kmax), dim3(128), 0, st, e, batch, l, G, g_stride, t_cols, U, bias,
              (__nv_bfloat16*)s_act);
 }
+cudaError_t select_step_configure(int bytes) {
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(select_advance_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_advance_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_advance_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_advance_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_step_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_step_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  if ((e = cudaFuncSetAttribute(select_step_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
+  return cudaFuncSetAttribute(select_step_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+void launch_select_step(const SelectArgs& a, const EngineState& e, int l, const float* G, long long g_stride, int t_cols,
+                        const float* U, const float* bias, void* s_act, cudaStream_t st) {
+  if (a.batch <= 0) return;
+  const size_t smem = select_smem_bytes(a.in_stride, a.K);
+  LaunchScope ls(kcSelect, st);
+  const int warps = a.in_stride < 8 ? 8 : a.in_stride > 16 ? 16 : a.in_stride;
+  const dim3 block(32 * warps), grid(a.batch);
+  __nv_bfloat16* s = (__nv_bfloat16*)s_act;
+  if (a.T <= 32) launch_pdl(select_step_kernel<1>, grid, block, smem, st, a, e, l, G, g_stride, t_cols, U, bias, s);
+  else if (a.T <= 256) launch_pdl(select_step_kernel<8>, grid, block, smem, st, a, e, l, G, g_stride, t_cols, U, bias, s);
+  else if (a.T <= 512) launch_pdl(select_step_kernel<16>, grid, block, smem, st, a, e, l, G, g_stride, t_cols, U, bias, s);
+  else launch_pdl(select_step_kernel<32>, grid, block, smem, st, a, e, l, G, g_stride, t_cols, U, bias, s);
+}
 void launch_copy_logits_bias(const float* src, long long row_stride, int row_mul, int batch, int n_beams, int T,
                              const float* bias, long long bias_stride, float* dst, cudaStream_t st) {
   LaunchScope ls(kcMisc, st);
@@ -788,6 +863,18 @@ void launch_advance(const EngineState& e, int batch, int n, int K, int* out_code
                     cudaStream_t st) {
   LaunchScope ls(kcAccept, st);
   launch_pdl(advance_kernel, dim3(batch), dim3(64), 0, st, e, batch, n, K, out_codes, out_score, out_count);
+}
+void launch_select_advance(const SelectArgs& a, const EngineState& e, int n, int K, int* out_codes, float* out_score,
+                           int* out_count, cudaStream_t st) {
+  if (a.batch <= 0) return;
+  const size_t smem = select_smem_bytes(a.in_stride, a.K);
+  LaunchScope ls(kcSelect, st);
+  const int warps = a.in_stride < 8 ? 8 : a.in_stride > 16 ? 16 : a.in_stride;
+  const dim3 block(32 * warps), grid(a.batch);
+  if (a.T <= 32) launch_pdl(select_advance_kernel<1>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
+  else if (a.T <= 256) launch_pdl(select_advance_kernel<8>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
+  else if (a.T <= 512) launch_pdl(select_advance_kernel<16>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
+  else launch_pdl(select_advance_kernel<32>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
 }
 void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, cudaStream_t st) {
   LaunchScope ls(kcAccept, st);

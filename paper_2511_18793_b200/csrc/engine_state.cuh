@@ -65,11 +65,17 @@ struct SelectArgs {
   LevelInfo li; HashSetView hs;
 };
 void launch_select(const SelectArgs& a, cudaStream_t st);
+// launch_select (gated on row_cur == n) followed, in the same launch, by launch_advance of level n
+void launch_select_advance(const SelectArgs& a, const EngineState& e, int n, int K, int* out_codes, float* out_score,
+                           int* out_count, cudaStream_t st);
+// launch_select followed, in the same launch, by launch_draft_step of level l (same arguments as there)
+void launch_select_step(const SelectArgs& a, const EngineState& e, int l, const float* G, long long g_stride, int t_cols,
+                        const float* U, const float* bias, void* s_act, cudaStream_t st);
 size_t select_smem_bytes(int in_stride, int K);
 cudaError_t select_configure(int max_beam);
 
 void launch_init_decode(const EngineState& e, int batch, cudaStream_t st);
-void launch_draft_init(const EngineState& e, int batch, int from_scratch, cudaStream_t st);
+void launch_draft_init(const EngineState& e, int batch, int from_scratch, void* s_act, cudaStream_t st);   // s_act may be null
 void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st);
 void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st);
 void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
