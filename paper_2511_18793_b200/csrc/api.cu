@@ -89,6 +89,7 @@ struct nezha_ctx {
   int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
+  int rounds_seen[3];       // rounds the last decode call of each mode needed: that many are launched without waiting
   int state;                // 0 created, 1 hash set built, 2 prefilled
   int batch;                // prefilled batch
   std::string err;
@@ -583,19 +584,29 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
         launch_select_advance(s, e, n, K, out_codes, out_scores, out_count, c->st);
       }
       launch_round_end(e, batch, K, round, tr, c->st);
-      cudaMemcpyAsync(c->host_counters, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st);
+      cudaMemcpyAsync(c->host_counters + 16 + 8 * round, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st);
     });
-    if (rs != NEZHA_OK) { c->m_expected = 0; return rs; }
+    c->m_expected = 0;
+    if (rs != NEZHA_OK) return rs;
+    // Whether another round is needed is known only from this round's counters.  A steady workload needs the same
+    // number of rounds call after call, so the rounds the last call needed are queued without waiting in between;
+    // a round queued for nothing finds every request finished and each of its kernels returns at once.
+    if (round < R && round < c->rounds_seen[mode]) continue;
     NZ_CUDA(c, cudaStreamSynchronize(c->st));
     NZ_CUDA(c, cudaGetLastError());
-    c->m_expected = 0;
-    c->m_seen[round] = (c->host_counters[1] + 127) / 128 * 128;
-    sd.rounds = round;
-    sd.primary_tokens += c->host_counters[1];
-    sd.accepted_levels += c->host_counters[2];
-    if (round == 1) sd.drafted = c->host_counters[3];
-    if (c->host_counters[0] == 0) break;
+    bool finished = false;
+    for (int r = sd.rounds + 1; r <= round && !finished; ++r) {
+      const int* hc = c->host_counters + 16 + 8 * r;
+      c->m_seen[r] = (hc[1] + 127) / 128 * 128;
+      sd.rounds = r;
+      sd.primary_tokens += hc[1];
+      sd.accepted_levels += hc[2];
+      if (r == 1) sd.drafted = hc[3];
+      finished = hc[0] == 0;
+    }
+    if (finished) break;
   }
+  c->rounds_seen[mode] = sd.rounds;
   if (tr.beams || tr.beam_scores) launch_trace_beams(e, batch, K, tr, c->st);
   nezha_status ps = pending_device_error(c);
   if (stats) *stats = sd;
@@ -632,6 +643,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   c->use_graphs = cuda_stream != nullptr && !getenv("NEZHA_NO_GRAPHS");
   c->m_expected = 0;
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
+  for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
   c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
@@ -639,7 +651,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   carve(c);
   auto bail = [&](nezha_status s) { if (c->host_counters) cudaFreeHost(c->host_counters); delete c; return s; };
   c->host_counters = nullptr;
-  if (cudaMallocHost((void**)&c->host_counters, 16 * sizeof(int)) != cudaSuccess) return bail(NEZHA_ERR_CUDA);
+  if (cudaMallocHost((void**)&c->host_counters, (16 + 8 * (kMaxLevels + 1)) * sizeof(int)) != cudaSuccess) return bail(NEZHA_ERR_CUDA);
   if (select_configure(c->Kmax) != cudaSuccess) return bail(NEZHA_ERR_CUDA);
   if (c->fused) {                  // needs the tensor-core GEMM (TMA descriptors) for every projection
     GemmArgs probe{c->xn, c->d, c->layers[0].wqkv, c->d, c->qkv, c->qkv_dim, 128, nullptr, c->qkv_dim, c->d, kEpiStoreAct, nullptr,

@@ -37,31 +37,93 @@ __device__ __forceinline__ float from_ordered_bits(unsigned o) {
 }
 constexpr unsigned kOrderedNegInf = 0x007fffffu;          // ordered_bits(-inf)
 
+// Sorts v in descending order with Batcher's odd-even merge network (N a power of two; every index is a compile-time
+// constant once unrolled, so v stays in registers).
+template <int N>
+__device__ __forceinline__ void sort_desc(unsigned long long (&v)[N]) {
+#pragma unroll
+  for (int p = 1; p < N; p <<= 1) {
+#pragma unroll
+    for (int k = p; k >= 1; k >>= 1) {
+#pragma unroll
+      for (int j = k % p; j + k < N; j += 2 * k) {
+#pragma unroll
+        for (int i = 0; i < k; ++i) {
+          if (i + j + k < N && (i + j) / (2 * p) == (i + j + k) / (2 * p)) {
+            const unsigned long long x = v[i + j], y = v[i + j + k];
+            v[i + j] = x > y ? x : y;
+            v[i + j + k] = x > y ? y : x;
+          }
+        }
+      }
+    }
+  }
+}
+
+// One block per request.  Stage 1, a warp per input beam: log-softmax of the beam's logits row (+ Eq. 5 on every
+// extension at the last level), then its `want` best codes in order into shared memory.  Stage 2: the K best of those
+// lists (score, then parent rank, then code).  Stage 3, all threads: the output beams.  The kernel is a chain of
+// dependent steps on a few warps, so its time is the sum of their latencies: loads whose address needs no other load
+// go out together at the top; each lane keeps its keys sorted, so one survivor costs two redux and a shift; small
+// merges are a rank count with no serial loop at all.
 template <int VPL>
 __device__ __forceinline__ void select_body(const SelectArgs& a) {
   const int b = blockIdx.x;
-  if (a.gate_mode == 1 && a.gate[b] != a.gate_value) return;
-  if (a.gate_mode == 2 && !(a.gate[b] < a.gate_value)) return;
   extern __shared__ unsigned char smem_raw[];
   const int nb_cap = a.in_stride;
   float* l_score = reinterpret_cast<float*>(smem_raw);              // [nb_cap][K]
   int* l_tok = reinterpret_cast<int*>(l_score + (size_t)nb_cap * a.K);   // [nb_cap][K]
   int* l_cnt = l_tok + (size_t)nb_cap * a.K;                         // [nb_cap]
+  float* sel_s = reinterpret_cast<float*>(l_cnt + nb_cap);           // [K] the selected (score, parent, code)
+  int* sel_r = reinterpret_cast<int*>(sel_s + a.K);
+  int* sel_t = sel_r + a.K;
+  int* s_nout = sel_t + a.K;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
-  const int nb = min(a.in_count[b], nb_cap);
+
+  // ---- first wave of loads (none of these addresses depends on a loaded value)
+  const int gate_v = a.gate_mode ? a.gate[b] : 0;
+  const int nb_raw = a.in_count[b];
+  const bool has0 = warp < nb_cap;                                   // this warp's first beam slot exists in the arrays
+  const long long slot0 = (long long)b * a.in_stride + warp;
+  const bool direct0 = has0 && !a.src_row && warp < a.src_mul;       // its logits row is known without a look-up
+  long long row0 = 0;
+  if (has0) row0 = a.src_row ? (long long)a.src_row[slot0] : (long long)b * a.src_mul + warp;
+  const float base0 = has0 ? a.in_score[slot0] : 0.f;
+  unsigned long long pk0 = 0;
+  if (has0)
+    for (int l = 0; l < a.n; ++l) pk0 += (unsigned long long)a.in_codes[slot0 * a.tuple_len + l] * a.li.mult[l];
+  float bias[VPL], z0[VPL];
+#pragma unroll
+  for (int j = 0; j < VPL; ++j) {
+    const int t = lane + 32 * j;
+    bias[j] = (a.logit_bias && t < a.T) ? a.logit_bias[(long long)b * a.bias_stride + t] : 0.f;
+    z0[j] = (direct0 && t < a.T) ? a.logits[row0 * a.row_stride + a.col_off + t] : 0.f;
+  }
+  if (a.gate_mode == 1 && gate_v != a.gate_value) return;
+  if (a.gate_mode == 2 && !(gate_v < a.gate_value)) return;
+  const int nb = min(nb_raw, nb_cap);
   const bool all_codes = a.per_beam >= a.T;
   const int want = all_codes ? min(a.K, a.T) : min(a.per_beam, a.K);
+  const unsigned long long mult_n = a.li.mult[a.n];
 
   for (int r = warp; r < nb; r += n_warps) {
-    const long long row = a.src_row ? a.src_row[(long long)b * a.in_stride + r] : (long long)b * a.src_mul + r;
+    const bool first = r == warp;
+    const long long slot = (long long)b * a.in_stride + r;
+    const long long row = first ? row0 : (a.src_row ? (long long)a.src_row[slot] : (long long)b * a.src_mul + r);
     const float* z = a.logits + row * a.row_stride + a.col_off;
     float key[VPL];
     float mx = -INFINITY;
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int t = lane + 32 * j;
-      key[j] = (t < a.T) ? z[t] + (a.logit_bias ? a.logit_bias[(long long)b * a.bias_stride + t] : 0.f) : -INFINITY;
+      key[j] = (t < a.T) ? ((first && direct0) ? z0[j] : z[t]) + bias[j] : -INFINITY;
       mx = fmaxf(mx, key[j]);
+    }
+    const float base = first ? base0 : a.in_score[slot];
+    unsigned long long prefix_key = pk0;
+    if (!first) {
+      prefix_key = 0;
+      for (int l = 0; l < a.n; ++l) prefix_key += (unsigned long long)a.in_codes[slot * a.tuple_len + l] * a.li.mult[l];
     }
     mx = warp_max(mx);
     float sum = 0.f;
@@ -69,11 +131,6 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
     for (int j = 0; j < VPL; ++j) sum += (lane + 32 * j < a.T) ? expf(key[j] - mx) : 0.f;
     sum = warp_sum(sum);
     const float lse = mx + logf(sum);
-    const float base = a.in_score[(long long)b * a.in_stride + r];
-    unsigned long long prefix_key = 0;
-    for (int l = 0; l < a.n; ++l)
-      prefix_key += (unsigned long long)a.in_codes[((long long)b * a.in_stride + r) * a.tuple_len + l] * a.li.mult[l];
-    const unsigned long long mult_n = a.li.mult[a.n];
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       if (lane + 32 * j < a.T) {
@@ -97,25 +154,26 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
           if (want_probe[j] && !ok[j]) key[j0 + j] = -INFINITY;
       }
     }
-    // ordered extraction: one warp arg-max per survivor (two redux instructions; ties go to the smaller code)
+    // this lane's keys in descending order: (ordered score bits, then the smaller code first); 0 = used up
+    unsigned long long sk[VPL];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) sk[j] = ((unsigned long long)ordered_bits(key[j]) << 32) | (unsigned)(VPL - 1 - j);
+    sort_desc<VPL>(sk);
+    // ordered extraction: the warp's best head (ties go to the smaller code), whose lane then shifts its list
     int cnt = 0;
     for (int it = 0; it < want; ++it) {
-      unsigned bo = 0u; int bt = 0x7fffffff;
-#pragma unroll
-      for (int j = 0; j < VPL; ++j) {
-        const unsigned o = ordered_bits(key[j]);
-        if (o > bo) { bo = o; bt = lane + 32 * j; }
-      }
-      const unsigned mo = __reduce_max_sync(0xffffffffu, bo);
+      const unsigned ho = (unsigned)(sk[0] >> 32);
+      const int ht = lane + 32 * (VPL - 1 - (int)(unsigned)sk[0]);
+      const unsigned mo = __reduce_max_sync(0xffffffffu, ho);
       if (mo <= kOrderedNegInf) break;
-      bt = __reduce_min_sync(0xffffffffu, bo == mo ? bt : 0x7fffffff);
-      const float bv = from_ordered_bits(mo);
+      const int bt = (int)__reduce_min_sync(0xffffffffu, ho == mo ? (unsigned)ht : 0x7fffffffu);
       if ((bt & 31) == lane) {
 #pragma unroll
-        for (int j = 0; j < VPL; ++j)
-          if (j == (bt >> 5)) key[j] = -INFINITY;
+        for (int j = 0; j + 1 < VPL; ++j) sk[j] = sk[j + 1];
+        sk[VPL - 1] = 0ull;
       }
       if (lane == 0) {
+        const float bv = from_ordered_bits(mo);
         l_score[(size_t)r * a.K + cnt] = all_codes ? bv : base + bv;
         l_tok[(size_t)r * a.K + cnt] = bt;
       }
@@ -126,16 +184,16 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
       int kept = 0;
       for (int c0 = 0; c0 < cnt; c0 += 32) {
         const int c = c0 + lane;
-        bool ok = false; float s = 0.f; int t = 0;
+        bool ok = false; float sv = 0.f; int t = 0;
         if (c < cnt) {
-          s = l_score[(size_t)r * a.K + c]; t = l_tok[(size_t)r * a.K + c];
+          sv = l_score[(size_t)r * a.K + c]; t = l_tok[(size_t)r * a.K + c];
           ok = hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
         }
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         __syncwarp();
         if (ok) {
           const int dst = kept + __popc(m & ((1u << lane) - 1u));
-          l_score[(size_t)r * a.K + dst] = s; l_tok[(size_t)r * a.K + dst] = t;
+          l_score[(size_t)r * a.K + dst] = sv; l_tok[(size_t)r * a.K + dst] = t;
         }
         kept += __popc(m);
         __syncwarp();
@@ -145,59 +203,83 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
     if (lane == 0) l_cnt[r] = cnt;
   }
   __syncthreads();
-  if (warp != 0) return;
 
-  // merge the sorted lists
-  constexpr int RPL = 4;                                 // lists per lane: in_stride <= 128
-  int ptr[RPL];
-#pragma unroll
-  for (int q = 0; q < RPL; ++q) ptr[q] = 0;
-  int n_out = 0;
-  for (int k = 0; k < a.K; ++k) {
-    float bs = -INFINITY; int br = 0x7fffffff, bt = 0x7fffffff;
-#pragma unroll
-    for (int q = 0; q < RPL; ++q) {
-      const int r = lane + 32 * q;
-      if (r < nb && ptr[q] < l_cnt[r]) {
-        const float s = l_score[(size_t)r * a.K + ptr[q]];
-        const int t = l_tok[(size_t)r * a.K + ptr[q]];
-        if (br == 0x7fffffff || cand_better(s, r, t, bs, br, bt)) { bs = s; br = r; bt = t; }
+  // ---- stage 2: the K best candidates of the nb lists into sel_*[0 .. n_out)
+  if (nb * a.K <= 1024) {
+    // few candidates: a candidate's output position is the number of candidates that beat it (the order is strict)
+    if (threadIdx.x == 0) {
+      int tot = 0;
+      for (int r = 0; r < nb; ++r) tot += l_cnt[r];
+      *s_nout = min(tot, a.K);
+    }
+    for (int i = threadIdx.x; i < nb * a.K; i += blockDim.x) {
+      const int r = i / a.K, c = i - r * a.K;
+      if (c >= l_cnt[r]) continue;
+      const float sv = l_score[i];
+      const int t = l_tok[i];
+      int rank = c;                                        // its own list is sorted: c of its entries come before it
+      for (int r2 = 0; r2 < nb; ++r2) {
+        if (r2 == r) continue;
+        const int n2 = l_cnt[r2];
+        for (int c2 = 0; c2 < n2; ++c2)
+          rank += cand_better(l_score[(size_t)r2 * a.K + c2], r2, l_tok[(size_t)r2 * a.K + c2], sv, r, t) ? 1 : 0;
       }
+      if (rank < a.K) { sel_s[rank] = sv; sel_r[rank] = r; sel_t[rank] = t; }
     }
-    // warp arg-best: maximum score, then the smallest (parent rank, code) among the lanes that hold it
-    const unsigned bo = br == 0x7fffffff ? 0u : ordered_bits(bs);
-    const unsigned mo = __reduce_max_sync(0xffffffffu, bo);
-    if (mo == 0u) break;                                   // every list is exhausted
-    const unsigned pick = __reduce_min_sync(0xffffffffu, bo == mo ? ((unsigned)br << 16 | (unsigned)bt) : 0xffffffffu);
-    bs = from_ordered_bits(mo); br = (int)(pick >> 16); bt = (int)(pick & 0xffffu);
+  } else if (warp == 0) {
+    constexpr int RPL = 4;                                 // lists per lane: in_stride <= 128
+    int ptr[RPL];
 #pragma unroll
-    for (int q = 0; q < RPL; ++q)
-      if (lane + 32 * q == br) ++ptr[q];
-    const long long o = (long long)b * a.out_stride + k;
-    if (lane == 0) {
-      a.out_score[o] = bs;
-      if (a.out_parent) a.out_parent[o] = br;
-      if (a.out_token) a.out_token[o] = bt;
-    }
-    if (a.out_codes) {
-      for (int l = lane; l < a.tuple_len; l += 32) {
-        int c = -1;
-        if (l < a.n) c = a.in_codes[((long long)b * a.in_stride + br) * a.tuple_len + l];
-        else if (l == a.n) c = bt;
-        a.out_codes[o * a.tuple_len + l] = c;
+    for (int q = 0; q < RPL; ++q) ptr[q] = 0;
+    int n_out = 0;
+    for (int k = 0; k < a.K; ++k) {
+      float bs = -INFINITY; int br = 0x7fffffff, bt = 0x7fffffff;
+#pragma unroll
+      for (int q = 0; q < RPL; ++q) {
+        const int r = lane + 32 * q;
+        if (r < nb && ptr[q] < l_cnt[r]) {
+          const float sv = l_score[(size_t)r * a.K + ptr[q]];
+          const int t = l_tok[(size_t)r * a.K + ptr[q]];
+          if (br == 0x7fffffff || cand_better(sv, r, t, bs, br, bt)) { bs = sv; br = r; bt = t; }
+        }
       }
+      // warp arg-best: maximum score, then the smallest (parent rank, code) among the lanes that hold it
+      const unsigned bo = br == 0x7fffffff ? 0u : ordered_bits(bs);
+      const unsigned mo = __reduce_max_sync(0xffffffffu, bo);
+      if (mo == 0u) break;                                   // every list is exhausted
+      const unsigned pick = __reduce_min_sync(0xffffffffu, bo == mo ? ((unsigned)br << 16 | (unsigned)bt) : 0xffffffffu);
+      br = (int)(pick >> 16); bt = (int)(pick & 0xffffu);
+#pragma unroll
+      for (int q = 0; q < RPL; ++q)
+        if (lane + 32 * q == br) ++ptr[q];
+      if (lane == 0) { sel_s[k] = from_ordered_bits(mo); sel_r[k] = br; sel_t[k] = bt; }
+      ++n_out;
     }
-    ++n_out;
+    if (lane == 0) *s_nout = n_out;
   }
-  for (int k = n_out + lane; k < a.K; k += 32) {
+  __syncthreads();
+
+  // ---- stage 3: the output beams, all threads
+  const int n_out = *s_nout;
+  for (int k = threadIdx.x; k < a.K; k += blockDim.x) {
     const long long o = (long long)b * a.out_stride + k;
-    a.out_score[o] = -INFINITY;
-    if (a.out_parent) a.out_parent[o] = -1;
-    if (a.out_token) a.out_token[o] = -1;
-    if (a.out_codes)
-      for (int l = 0; l < a.tuple_len; ++l) a.out_codes[o * a.tuple_len + l] = -1;
+    const bool live = k < n_out;
+    a.out_score[o] = live ? sel_s[k] : -INFINITY;
+    if (a.out_parent) a.out_parent[o] = live ? sel_r[k] : -1;
+    if (a.out_token) a.out_token[o] = live ? sel_t[k] : -1;
   }
-  if (lane == 0) a.out_count[b] = n_out;
+  if (a.out_codes) {
+    for (int i = threadIdx.x; i < a.K * a.tuple_len; i += blockDim.x) {
+      const int k = i / a.tuple_len, l = i - k * a.tuple_len;
+      int c = -1;
+      if (k < n_out) {
+        if (l < a.n) c = a.in_codes[((long long)b * a.in_stride + sel_r[k]) * a.tuple_len + l];
+        else if (l == a.n) c = sel_t[k];
+      }
+      a.out_codes[((long long)b * a.out_stride + k) * a.tuple_len + l] = c;
+    }
+  }
+  if (threadIdx.x == 0) a.out_count[b] = n_out;
 }
 
 template <int VPL>
@@ -212,7 +294,8 @@ __global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
 cudaError_t select_step_configure(int bytes);
 
 size_t select_smem_bytes(int in_stride, int K) {
-  return (size_t)in_stride * K * (sizeof(float) + sizeof(int)) + (size_t)in_stride * sizeof(int);
+  return (size_t)in_stride * K * (sizeof(float) + sizeof(int)) + (size_t)in_stride * sizeof(int) +
+         (size_t)K * (sizeof(float) + 2 * sizeof(int)) + sizeof(int);
 }
 
 cudaError_t select_configure(int max_beam) {
