@@ -59,6 +59,26 @@ __device__ __forceinline__ uint32_t kv_addr(uint32_t tile, int pos, int chunk) {
 // softmax state of the thread's two rows (m in the scaled log2 domain).  The loads of all (row, entry) pairs are
 // issued together -- offsets, then every K row, then every V row -- so the chain of dependent memory round trips is
 // three long whatever the number of entries.  E = compile-time bound of the entries per token (n_ext_max <= E).
+// Asks for the extra K and V rows of one token (and, by loading it, the token's offset list) to be brought into L1.
+// Called before the context tiles are streamed, so that the three dependent round trips of fold_extra_rows (offsets, K
+// rows, V rows) happen under the wait for the first tiles instead of after the last one.
+template <int HD>
+__device__ __forceinline__ void prefetch_extra_rows(const AttnArgs& a, int tok, int kvh) {
+  const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
+  const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
+  for (int e = 0; e < a.n_ext_max; ++e) {
+    const long long off = a.tok_ext[(long long)tok * a.n_ext_max + e];
+    if (off < 0) continue;
+    const __nv_bfloat16* kp = ke + off + (long long)kvh * a.ext_head_stride;
+    const __nv_bfloat16* vp = ve + off + (long long)kvh * a.ext_head_stride;
+#pragma unroll
+    for (int c = 0; c < HD; c += 64) {              // 128-byte lines
+      asm volatile("prefetch.global.L1 [%0];" ::"l"(kp + c));
+      asm volatile("prefetch.global.L1 [%0];" ::"l"(vp + c));
+    }
+  }
+}
+
 template <int HD, int E>
 __device__ __forceinline__ void fold_extra_rows(const AttnArgs& a, const int* tok, const int* head, const bool* live, int kvh,
                                                 int qc, float sc, float* m_run, float* l_run, float (*o)[4]) {
@@ -242,6 +262,11 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
 #pragma unroll
     for (int j = 0; j < NB; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
     const int ctx_min = __reduce_min_sync(0xffffffffu, min(ctx[0], ctx[1]));   // tiles below it need no masking
+    if (a.n_ext_max > 0 && qc == 0) {               // one lane per row
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+        if (live[i]) prefetch_extra_rows<HD>(a, tok[i], kvh);
+    }
 
     for (int t = g; t < n_tiles; t += KW) {
       const int s = t % S;

@@ -201,6 +201,19 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
     bool ok = true;
     const int ctx_min = __reduce_min_sync(0xffffffffu, ctx);
     const bool warp_dead = r0 + (warp & 3) * 32 >= R;   // none of this warp's 32 rows exists: it only keeps the barriers going
+    if (live && a.n_ext_max > 0) {                  // the row's extra K and V rows into L1 while the context streams
+      const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
+      const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
+      for (int e = 0; e < a.n_ext_max; ++e) {
+        const long long off = a.tok_ext[(long long)tok * a.n_ext_max + e];
+        if (off < 0) continue;
+#pragma unroll
+        for (int c = 0; c < HD; c += 64) {
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(ke + off + (long long)kvh * a.ext_head_stride + c));
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(ve + off + (long long)kvh * a.ext_head_stride + c));
+        }
+      }
+    }
     for (int j = 0; j < n_tiles; ++j) {
       const int b = j & 1;
       ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full(b), (j >> 1) & 1, abort_flag));
