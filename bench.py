@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -27,11 +28,12 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 METRIC, UNIT = "items_per_s_decoded", "items/s"
 # bumped whenever a kernel of the class changes in a way that can change its DRAM traffic: a traffic figure taken
 # from an older revision is reported as null
-KERNEL_REV = {"gemm": 4, "attention": 2}
+KERNEL_REV = {"gemm": 4, "attention": 2, "probe": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the launches of the class in one decode step
 # (ncu, eager launches, L2 flushed before the step)
 NCU_TRAFFIC = {
     "gemm@small": {"kernel_rev": 4, "dram_bytes_per_launch": 3.18e6, "source": "profiles/gemm_tc_kernel_ncu.md, section A2"},
+    "probe@0.5b@67108864": {"kernel_rev": 2, "dram_bytes_per_launch": 5.10e9, "source": "profiles/hs_probe_kernel.md"},
     "attention@small": {"kernel_rev": 2, "dram_bytes_per_launch": 29.6e6, "source": "profiles/attn_tc_kernel_ncu.md, traffic section"},
 }
 
@@ -146,6 +148,51 @@ def algorithmic_work(w, stats_tokens_per_step, rounds):
     return {"gemm_flops": gemm_flops, "attention_bytes": attn_bytes, "attention_flops": attn_flops}
 
 
+def probe_bench(args, w, eng, cat_dev, config, dev):
+    """The hash-set probe alone: n keys (half catalogue items drawn at random, half uniform random tuples, shuffled),
+    already packed and resident in HBM.  Algorithmic bytes per key: the 8-byte key, the 1-byte answer and one 32-byte
+    bucket (at load factor 0.5 a probe sequence almost always ends in its first bucket)."""
+    import torch
+    n = args.probe_keys
+    g = torch.Generator(device=dev); g.manual_seed(1234)
+    half = n // 2
+    idx = torch.randint(0, w.n_items, (half,), device=dev, generator=g)
+    hits = cat_dev[idx]
+    rnd = torch.stack([torch.randint(0, w.T[l], (n - half,), device=dev, generator=g, dtype=torch.int32) for l in range(w.L)], dim=1)
+    codes = torch.cat([hits, rnd], dim=0)[torch.randperm(n, device=dev, generator=g)].contiguous()
+    keys = eng.pack(codes)
+    del codes, hits, rnd, idx
+    found = torch.empty(n, dtype=torch.uint8, device=dev)
+    for _ in range(max(args.warmup, 3)):
+        eng.probe(keys, out=found)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(int(dev.split(":")[1]))
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        eng.probe(keys, out=found)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / args.steps
+    peaks = load_peaks()
+    gbs = n * 41.0 / (ms / 1e3) / 1e9
+    rec = NCU_TRAFFIC.get(f"probe@{w.name}@{n}")
+    traffic = rec["dram_bytes_per_launch"] if rec and rec["kernel_rev"] == KERNEL_REV.get("probe") else None
+    slots = 4 * max(2, math.ceil(math.ceil(max(1, w.n_items) / w.load_factor) / 4))      # buckets of four 8-byte slots
+    print(json.dumps({"metric": "hash_probes_per_s", "value": n / (ms / 1e3), "unit": "probes/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "u64", "data": "synthetic",
+                      "config": {"workload": config["workload"], "keys": n, "hit_fraction": float(found.float().mean()),
+                                 "table_bytes": slots * 8, "l2": "keys alone (8 bytes each) exceed L2"},
+                      "clocks": clocks, "gpu_launches": args.steps,
+                      "roofline": {"kernel": "hs_probe_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": traffic,
+                                   "of": peaks.get("source", "measured"),
+                                   "algorithmic_bytes_per_key": 41}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -158,6 +205,9 @@ def main():
                     help="mode 1 only: 'natural' = the (random-init) draft head's own drafts; 'perfect' = the true top-k "
                          "tuples injected as round-1 drafts (best case: one round, everything accepted)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (requests per decode call)")
+    ap.add_argument("--probe-keys", type=int, default=0,
+                    help="instead of the decode step, time the stand-alone hash-set probe (Eq. 5) on this many keys, "
+                         "half of them catalogue items, and print its own JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
     args = ap.parse_args()
@@ -227,6 +277,9 @@ def main():
     eng = binding.Engine(binding.make_config(w), weights, cat_dev, w.load_factor, stream=torch.cuda.current_stream())
     n_unique = eng.build_hashset()
     assert n_unique == w.n_items
+    if args.probe_keys > 0:
+        probe_bench(args, w, eng, cat_dev, config, dev)
+        return
     hist_pinned = torch.from_numpy(hist).pin_memory()
     nh_pinned = torch.full((w.batch,), w.n_hist, dtype=torch.int32).pin_memory()
     hist_dev = hist_pinned.to(dev, non_blocking=True)
