@@ -302,6 +302,8 @@ void run_layers_fused(nezha_ctx* c, long long M, const int* M_dev, bool verify, 
     t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
     t.rows_expected = (c->m_expected > 0 && n_rows > 0) ? (c->m_expected + n_rows - 1) / n_rows * (c->Hq / c->Hkv) : 0;
     t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
+    t.ext_positions = (c->L > 1 ? c->L - 1 : 1) * c->Kmax; t.ext_pos_stride = (long long)c->Hkv * c->hd;
+    t.ext_req_stride = t.ext_positions * t.ext_pos_stride; t.ext_rows_total = (long long)c->Bmax * t.ext_positions;
     if (attention_tc_supported(t)) launch_attention_tc(t, c->st);
     else launch_attention_simt(t, true, c->st);
     GemmFuse fo{};
@@ -349,6 +351,8 @@ void run_layers(nezha_ctx* c, long long M, const int* M_dev, bool verify, int n_
     t.req_info = verify ? e.req_info : e.pf_req_info;
     t.n_rows = n_rows; t.max_tokens_per_row = max_tok_per_row;
     t.ctx_rows_total = (long long)c->Bmax * c->Hkv * c->S; t.status = e.status;
+    t.ext_positions = (c->L > 1 ? c->L - 1 : 1) * c->Kmax; t.ext_pos_stride = (long long)c->Hkv * c->hd;
+    t.ext_req_stride = t.ext_positions * t.ext_pos_stride; t.ext_rows_total = (long long)c->Bmax * t.ext_positions;
     if (c->bf16 && attention_tc_supported(t)) launch_attention_tc(t, c->st);
     else launch_attention_simt(t, c->bf16, c->st);
     gemm(c, c->attn, (long long)c->Hq * c->hd, w.wo, (long long)c->Hq * c->hd, c->resid, c->d, M, M_dev, c->d,

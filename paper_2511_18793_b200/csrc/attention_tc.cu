@@ -10,8 +10,11 @@
 //   RW = 1, KW = 4   16 rows per CTA, the four warps take every fourth tile and their   (few rows: one beam set of a
 //                    softmax states are merged through shared memory at the end          small model, plain decode)
 // Ring slots are handed back to the producer with per-slot "empty" mbarriers, so warps never wait for each other.
-// The per-token extra KV rows (the token's own tuple's drafted codes, at most L-1 of them) are folded in afterwards
-// straight from global memory.  Every barrier wait is bounded (abort flag + error status + return).
+// The draft-token KV rows (a token sees its own tuple's drafted codes, at most L of them) are not gathered per token:
+// the request's whole block of draft positions -- every beam's, every level's, contiguous in the cache for one KV head --
+// follows the context as one or more further tiles of the same loop, and each query row masks them with the bit set
+// of the positions it may see (tree attention over the drafted tuples).  Every barrier wait is bounded (abort flag +
+// error status + return).
 #include <math.h>
 #include <stdlib.h>
 
@@ -55,98 +58,6 @@ __device__ __forceinline__ uint32_t kv_addr(uint32_t tile, int pos, int chunk) {
   return tile + sub * (kPos * 128) + pos * 128 + ((c ^ (pos & 7)) << 4);
 }
 
-// The token's own extra KV rows (drafted codes of its tuple), straight from global memory, folded into the running
-// softmax state of the thread's two rows (m in the scaled log2 domain).  The loads of all (row, entry) pairs are
-// issued together -- offsets, then every K row, then every V row -- so the chain of dependent memory round trips is
-// three long whatever the number of entries.  E = compile-time bound of the entries per token (n_ext_max <= E).
-// Asks for the extra K and V rows of one token (and, by loading it, the token's offset list) to be brought into L1.
-// Called before the context tiles are streamed, so that the three dependent round trips of fold_extra_rows (offsets, K
-// rows, V rows) happen under the wait for the first tiles instead of after the last one.
-template <int HD>
-__device__ __forceinline__ void prefetch_extra_rows(const AttnArgs& a, int tok, int kvh) {
-  const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
-  const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
-  for (int e = 0; e < a.n_ext_max; ++e) {
-    const long long off = a.tok_ext[(long long)tok * a.n_ext_max + e];
-    if (off < 0) continue;
-    const __nv_bfloat16* kp = ke + off + (long long)kvh * a.ext_head_stride;
-    const __nv_bfloat16* vp = ve + off + (long long)kvh * a.ext_head_stride;
-#pragma unroll
-    for (int c = 0; c < HD; c += 64) {              // 128-byte lines
-      asm volatile("prefetch.global.L1 [%0];" ::"l"(kp + c));
-      asm volatile("prefetch.global.L1 [%0];" ::"l"(vp + c));
-    }
-  }
-}
-
-template <int HD, int E>
-__device__ __forceinline__ void fold_extra_rows(const AttnArgs& a, const int* tok, const int* head, const bool* live, int kvh,
-                                                int qc, float sc, float* m_run, float* l_run, float (*o)[4]) {
-  constexpr int NB = HD / 8;
-  const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
-  const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
-  const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
-  long long off[2][E];
-#pragma unroll
-  for (int i = 0; i < 2; ++i)
-#pragma unroll
-    for (int e = 0; e < E; ++e)
-      off[i][e] = (live[i] && e < a.n_ext_max) ? a.tok_ext[(long long)tok[i] * a.n_ext_max + e] : -1;
-  // the 4 lanes of a quad own the same rows, so `off` is uniform inside the quad shuffles below
-  float sdot[2][E];
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    const __nv_bfloat16* qp = q + (long long)tok[i] * a.q_stride + (long long)head[i] * HD + qc * 2;
-    __nv_bfloat162 qq[NB];
-#pragma unroll
-    for (int j = 0; j < NB; ++j) qq[j] = *reinterpret_cast<const __nv_bfloat162*>(qp + j * 8);
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-      float sd = 0.f;
-      if (off[i][e] >= 0) {
-        const __nv_bfloat16* kp = ke + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
-#pragma unroll
-        for (int j = 0; j < NB; ++j) {
-          const __nv_bfloat162 kk = *reinterpret_cast<const __nv_bfloat162*>(kp + j * 8);
-          sd += __bfloat162float(qq[j].x) * __bfloat162float(kk.x) + __bfloat162float(qq[j].y) * __bfloat162float(kk.y);
-        }
-      }
-      sdot[i][e] = sd;
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    float m_new = m_run[i];
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-      float sd = sdot[i][e];
-      sd += __shfl_xor_sync(0xffffffffu, sd, 1);
-      sd += __shfl_xor_sync(0xffffffffu, sd, 2);
-      sdot[i][e] = off[i][e] >= 0 ? sd * sc : -INFINITY;
-      m_new = fmaxf(m_new, sdot[i][e]);
-    }
-    if (m_new == -INFINITY) continue;              // nothing visible at all (dead row)
-    const float c = ex2(m_run[i] - m_new);
-    l_run[i] *= c;
-#pragma unroll
-    for (int j = 0; j < NB; ++j) { o[j][i * 2] *= c; o[j][i * 2 + 1] *= c; }
-    m_run[i] = m_new;
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-      if (off[i][e] < 0) continue;
-      const float p = ex2(sdot[i][e] - m_new);
-      l_run[i] += (qc == 0 ? p : 0.f);             // row sums are per-lane partials, reduced at the end
-      const __nv_bfloat16* vp = ve + off[i][e] + (long long)kvh * a.ext_head_stride + qc * 2;
-#pragma unroll
-      for (int j = 0; j < NB; ++j) {
-        const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162*>(vp + j * 8);
-        o[j][i * 2] += p * __bfloat162float(vv.x);
-        o[j][i * 2 + 1] += p * __bfloat162float(vv.y);
-      }
-    }
-  }
-}
-
 template <int HD, int RW, int KW>
 struct AttnCfg {
   static constexpr int kStages = KW == 1 ? 3 : KW;                // a multiple of KW: slot s always serves warp group s % KW
@@ -162,6 +73,8 @@ struct AttnCfg {
 template <int HD, int RW, int KW>
 __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                                const __grid_constant__ CUtensorMap tmV,
+                                                                               const __grid_constant__ CUtensorMap tmKx,
+                                                                               const __grid_constant__ CUtensorMap tmVx,
                                                                                AttnArgs a, int* status) {
   using C = AttnCfg<HD, RW, KW>;
   constexpr int S = C::kStages;
@@ -186,6 +99,12 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
   // context positions this tile needs: all of them, or (causal prefill) up to its last token's own position
   const int max_ctx = info.w >= 0 ? info.w : min((r0 + kRows - 1) / G, n_tok - 1) + 1;
   const int n_tiles = (max_ctx + kPos - 1) / kPos;
+  // The draft-token KV rows of the request (every beam's, every level's: ext_positions of them, contiguous for one KV
+  // head) follow the context as n_xt more tiles of the same loop; a query row sees only its own ancestors and itself
+  // among them, through a per-row bit mask.  Rows nobody sees are finite (the cache is zeroed when the engine is made),
+  // so their P = 0 contributes exactly nothing.
+  const int n_xt = a.n_ext_max > 0 ? (a.ext_positions + kPos - 1) / kPos : 0;
+  const int NT = n_tiles + n_xt;
   const int kv_row0 = (int)(((long long)request * a.Hkv + kvh) * (a.ctx_head_stride / HD));   // first cache row
 
   extern __shared__ uint8_t smem_raw[];
@@ -218,14 +137,21 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
     if (lane == 0) {
       int t = 0;
       bool ok = true;
-      for (; t < n_tiles; ++t) {
+      for (; t < NT; ++t) {
         const int s = t % S;
         if (t >= S && !mbar_wait_or_abort(empty_bar(s), ((t / S) - 1) & 1, abort_flag)) { ok = false; break; }
         mbar_expect_tx(full_bar(s), C::kStageBytes);
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
-          tma_load_2d(base + s * C::kStageBytes + h * (kPos * 128), &tmK, h * 64, kv_row0 + t * kPos, full_bar(s));
-          tma_load_2d(base + s * C::kStageBytes + C::kTileBytes + h * (kPos * 128), &tmV, h * 64, kv_row0 + t * kPos, full_bar(s));
+          const uint32_t kd = base + s * C::kStageBytes + h * (kPos * 128), vd = kd + C::kTileBytes;
+          if (t < n_tiles) {
+            tma_load_2d(kd, &tmK, h * 64, kv_row0 + t * kPos, full_bar(s));
+            tma_load_2d(vd, &tmV, h * 64, kv_row0 + t * kPos, full_bar(s));
+          } else {                                   // [positions, kv heads * hd]: this head's columns of 64 draft positions
+            const int y = request * a.ext_positions + (t - n_tiles) * kPos;
+            tma_load_2d(kd, &tmKx, kvh * HD + h * 64, y, full_bar(s));
+            tma_load_2d(vd, &tmVx, kvh * HD + h * 64, y, full_bar(s));
+          }
         }
       }
       if (!ok) {                                     // drain the copies still in flight before the CTA's smem goes away
@@ -262,13 +188,17 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
 #pragma unroll
     for (int j = 0; j < NB; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
     const int ctx_min = __reduce_min_sync(0xffffffffu, min(ctx[0], ctx[1]));   // tiles below it need no masking
-    if (a.n_ext_max > 0 && qc == 0) {               // one lane per row
+    int xpos[2][kMaxLevels];                        // the rows' visible draft positions inside the request's block, or -1
 #pragma unroll
-      for (int i = 0; i < 2; ++i)
-        if (live[i]) prefetch_extra_rows<HD>(a, tok[i], kvh);
-    }
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int e = 0; e < kMaxLevels; ++e) {
+        long long off = -1;
+        if (live[i] && e < a.n_ext_max) off = a.tok_ext[(long long)tok[i] * a.n_ext_max + e];
+        xpos[i][e] = off >= 0 ? (int)((off - (long long)request * a.ext_req_stride) / a.ext_pos_stride) : -1;
+      }
 
-    for (int t = g; t < n_tiles; t += KW) {
+    for (int t = g; t < NT; t += KW) {
       const int s = t % S;
       const bool got = mbar_wait_or_abort(full_bar(s), (t / S) & 1, abort_flag);
       if (!__all_sync(0xffffffffu, got)) { if (lane == 0) *abort_flag = 1; break; }
@@ -293,7 +223,21 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
       }
       // ---- mask (only tiles that reach past some row's context), online softmax in base 2
       // rows qr and qr+8; columns j*8 + qc*2 + {0,1}
-      if ((t + 1) * kPos > ctx_min) {
+      if (t >= n_tiles) {                            // a tile of draft positions: each row's own mask
+        unsigned long long mk[2] = {0ull, 0ull};
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+          for (int e = 0; e < kMaxLevels; ++e) {
+            const int p = xpos[i][e] - (t - n_tiles) * kPos;
+            if (xpos[i][e] >= 0 && p >= 0 && p < kPos) mk[i] |= 1ull << p;
+          }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (!((mk[e >> 1] >> (j * 8 + qc * 2 + (e & 1))) & 1ull)) sacc[j][e] = -INFINITY;
+      } else if ((t + 1) * kPos > ctx_min) {
         const int p_base = t * kPos + qc * 2;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -389,10 +333,6 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
     }
   }
 
-  // ---- the token's own extra KV rows (drafted codes of its tuple)
-  if (a.n_ext_max > 4) fold_extra_rows<HD, kMaxLevels>(a, tok, head, live, kvh, qc, sc, m_run, l_run, o);
-  else if (a.n_ext_max > 0) fold_extra_rows<HD, 4>(a, tok, head, live, kvh, qc, sc, m_run, l_run, o);
-
   // ---- normalise and store
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out);
 #pragma unroll
@@ -419,7 +359,16 @@ void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cud
   }
   const int G = a.Hq / a.Hkv;
   dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + 16 * RW - 1) / (16 * RW));
-  launch_pdl(attn_tc_kernel<HD, RW, KW>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *tk, *tv, a, a.status);
+  // the layer's draft-token caches as [positions of all requests, kv heads * hd] (a prefill has none: any valid map)
+  const CUtensorMap* tkx = tk;
+  const CUtensorMap* tvx = tv;
+  if (a.n_ext_max > 0) {
+    const long long rows = a.ext_rows_total, cols = (long long)a.Hkv * HD;
+    tkx = tma_map_bf16(a.k_ext, rows, cols, cols, kPos);
+    tvx = tma_map_bf16(a.v_ext, rows, cols, cols, kPos);
+    if (!tkx || !tvx) { static const int flag = kStInternal; cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st); return; }
+  }
+  launch_pdl(attn_tc_kernel<HD, RW, KW>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *tk, *tv, *tkx, *tvx, a, a.status);
 }
 
 }  // namespace

@@ -11,8 +11,10 @@
 //                  second product, so the softmax of tile j + 1 does not wait for the product of tile j
 //   O += P V       tcgen05.mma M128 N=hd K16 x 4, V taken as it lies in the cache ([position][hd] = N-major operand)
 // The S product of tile j+1 is issued before the softmax of tile j is awaited, so the tensor pipe works under the
-// softmax.  At the end each thread folds in its row's extra KV rows (the token's own drafted codes) from global
-// memory, normalises and stores its row.  Every mbarrier wait is bounded (abort flag, error status, TMEM freed).
+// softmax.  The request's block of draft-token KV rows (every beam's, every level's) follows the context as further
+// tiles of the same loop; a row masks them with the bit set of the positions it may see (its own tuple's codes).  At
+// the end each thread normalises and stores its row.  Every mbarrier wait is bounded (abort flag, error status, TMEM
+// freed).
 #include <math.h>
 
 #include "gemm_epilogue.cuh"
@@ -66,7 +68,9 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 
 template <int HD>
 __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                             const __grid_constant__ CUtensorMap tmV, AttnArgs a, int* status) {
+                                                             const __grid_constant__ CUtensorMap tmV,
+                                                             const __grid_constant__ CUtensorMap tmKx,
+                                                             const __grid_constant__ CUtensorMap tmVx, AttnArgs a, int* status) {
   using C = UmmaCfg<HD>;
   constexpr int S = kStagesU;
   constexpr int NH = HD / 64;                       // 64-column sub-tiles of a K / V / Q tile
@@ -88,6 +92,12 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
   if (r0 >= R) return;
   const int max_ctx = info.w >= 0 ? info.w : min((r0 + kRowsU - 1) / G, n_tok - 1) + 1;
   const int n_tiles = (max_ctx + kPosU - 1) / kPosU;
+  // The draft-token KV rows of the request (every beam's, every level's: ext_positions of them, contiguous for one KV
+  // head) follow the context as n_xt more tiles of the same loop; a query row sees only its own ancestors and itself
+  // among them, through a per-row bit mask.  Rows nobody sees are finite (the cache is zeroed when the engine is made),
+  // so their P = 0 contributes exactly nothing.
+  const int n_xt = a.n_ext_max > 0 ? (a.ext_positions + kPosU - 1) / kPosU : 0;
+  const int NT = n_tiles + n_xt;
   const int kv_row0 = (int)(((long long)request * a.Hkv + kvh) * (a.ctx_head_stride / HD));
 
   extern __shared__ uint8_t smem_raw[];
@@ -147,14 +157,21 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
     if (lane == 0) {
       int t = 0;
       bool ok = true;
-      for (; t < n_tiles; ++t) {
+      for (; t < NT; ++t) {
         const int s = t % S;
         if (t >= S && !mbar_wait_or_abort(kv_empty(s), ((t / S) - 1) & 1, abort_flag)) { ok = false; break; }
         mbar_expect_tx(kv_full(s), C::kStageBytes);
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
-          tma_load_2d(kv_base + s * C::kStageBytes + h * (kPosU * 128), &tmK, h * 64, kv_row0 + t * kPosU, kv_full(s));
-          tma_load_2d(kv_base + s * C::kStageBytes + C::kTileBytes + h * (kPosU * 128), &tmV, h * 64, kv_row0 + t * kPosU, kv_full(s));
+          const uint32_t kd = kv_base + s * C::kStageBytes + h * (kPosU * 128), vd = kd + C::kTileBytes;
+          if (t < n_tiles) {
+            tma_load_2d(kd, &tmK, h * 64, kv_row0 + t * kPosU, kv_full(s));
+            tma_load_2d(vd, &tmV, h * 64, kv_row0 + t * kPosU, kv_full(s));
+          } else {                                   // [positions, kv heads * hd]: this head's columns of 64 draft positions
+            const int y = request * a.ext_positions + (t - n_tiles) * kPosU;
+            tma_load_2d(kd, &tmKx, kvh * HD + h * 64, y, kv_full(s));
+            tma_load_2d(vd, &tmVx, kvh * HD + h * 64, y, kv_full(s));
+          }
         }
       }
       if (!ok) {
@@ -179,9 +196,9 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
         tc_commit(s_full(b));
         return true;
       };
-      if (n_tiles > 0) ok = issue_s(0);
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        if (j + 1 < n_tiles && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
+      if (NT > 0) ok = issue_s(0);
+      for (int j = 0; j < NT && ok; ++j) {
+        if (j + 1 < NT && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
         if (!mbar_wait_or_abort(p_full(j & 1), (j >> 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vt = kv_base + (j % S) * C::kStageBytes + C::kTileBytes;
@@ -201,20 +218,14 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
     bool ok = true;
     const int ctx_min = __reduce_min_sync(0xffffffffu, ctx);
     const bool warp_dead = r0 + (warp & 3) * 32 >= R;   // none of this warp's 32 rows exists: it only keeps the barriers going
-    if (live && a.n_ext_max > 0) {                  // the row's extra K and V rows into L1 while the context streams
-      const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
-      const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
-      for (int e = 0; e < a.n_ext_max; ++e) {
-        const long long off = a.tok_ext[(long long)tok * a.n_ext_max + e];
-        if (off < 0) continue;
+    int xpos[kMaxLevels];                           // the row's visible draft positions inside the request's block, or -1
 #pragma unroll
-        for (int c = 0; c < HD; c += 64) {
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(ke + off + (long long)kvh * a.ext_head_stride + c));
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(ve + off + (long long)kvh * a.ext_head_stride + c));
-        }
-      }
+    for (int e = 0; e < kMaxLevels; ++e) {
+      long long off = -1;
+      if (live && e < a.n_ext_max) off = a.tok_ext[(long long)tok * a.n_ext_max + e];
+      xpos[e] = off >= 0 ? (int)((off - (long long)request * a.ext_req_stride) / a.ext_pos_stride) : -1;
     }
-    for (int j = 0; j < n_tiles; ++j) {
+    for (int j = 0; j < NT; ++j) {
       const int b = j & 1;
       ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full(b), (j >> 1) & 1, abort_flag));
       if (!ok) break;
@@ -234,7 +245,17 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(s_free(b));         // the scores are in registers: the buffer may take tile j + 2
-      if ((j + 1) * kPosU > ctx_min) {
+      if (j >= n_tiles) {                            // a tile of draft positions: the row's own mask
+        unsigned long long mk = 0ull;
+#pragma unroll
+        for (int e = 0; e < kMaxLevels; ++e) {
+          const int p = xpos[e] - (j - n_tiles) * kPosU;
+          if (xpos[e] >= 0 && p >= 0 && p < kPosU) mk |= 1ull << p;
+        }
+#pragma unroll
+        for (int c = 0; c < kPosU; ++c)
+          if (!((mk >> c) & 1ull)) sv[c] = -INFINITY;
+      } else if ((j + 1) * kPosU > ctx_min) {
 #pragma unroll
         for (int c = 0; c < kPosU; ++c)
           if (j * kPosU + c >= ctx) sv[c] = -INFINITY;
@@ -285,71 +306,20 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(p_full(b));
     }
-    if (ok && n_tiles > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done((n_tiles - 1) & 1), ((n_tiles - 1) >> 1) & 1, abort_flag));
+    if (ok && NT > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done((NT - 1) & 1), ((NT - 1) >> 1) & 1, abort_flag));
       tc_fence_after();
     }
     if (!ok) { if (lane == 0) *abort_flag = 1; }
     else {
-      // ---- the row's own extra KV rows, then normalise and store (thread = row)
-      constexpr int E = kMaxLevels;
-      const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(a.q) + (long long)tok * a.q_stride + (long long)head * HD;
-      const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(a.k_ext);
-      const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(a.v_ext);
-      long long off[E]; float se[E];
-      float m_fin = m_ref;
-#pragma unroll
-      for (int e = 0; e < E; ++e) {
-        off[e] = (live && e < a.n_ext_max) ? a.tok_ext[(long long)tok * a.n_ext_max + e] : -1;
-        se[e] = -INFINITY;
-      }
-#pragma unroll
-      for (int e = 0; e < E; ++e) {
-        if (off[e] < 0) continue;
-        const uint4* kp = reinterpret_cast<const uint4*>(ke + off[e] + (long long)kvh * a.ext_head_stride);
-        float d = 0.f;
-        for (int c = 0; c < HD / 8; ++c) {
-          const uint4 qv = reinterpret_cast<const uint4*>(qp)[c], kv = kp[c];
-          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
-          const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 qf = __bfloat1622float2(q2[i]), kf = __bfloat1622float2(k2[i]);
-            d = fmaf(qf.x, kf.x, d); d = fmaf(qf.y, kf.y, d);
-          }
-        }
-        se[e] = d * sc;
-        m_fin = fmaxf(m_fin, se[e]);
-      }
-      const float m_safe = m_fin == -INFINITY ? 0.f : m_fin;
-      const float c0 = ex2u(m_ref - m_safe);
-      float l_tot = l_run * c0, pe[E];
-#pragma unroll
-      for (int e = 0; e < E; ++e) { pe[e] = off[e] >= 0 ? ex2u(se[e] - m_safe) : 0.f; l_tot += pe[e]; }
+      // ---- normalise and store (thread = row)
+      const float l_tot = l_run;
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
       __nv_bfloat16* op = reinterpret_cast<__nv_bfloat16*>(a.out) + (long long)tok * a.out_stride + (long long)head * HD;
 #pragma unroll 1
       for (int c = 0; c < HD / 32; ++c) {
         float ov[32];
         tmem_ld32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);   // warp-collective: dead rows take part too
-#pragma unroll
-        for (int i = 0; i < 32; ++i) ov[i] *= c0;
-#pragma unroll
-        for (int e = 0; e < E; ++e) {
-          if (off[e] < 0) continue;
-          const uint4* vp = reinterpret_cast<const uint4*>(ve + off[e] + (long long)kvh * a.ext_head_stride + c * 32);
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const uint4 vv = vp[u];
-            const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vv);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float2 vf = __bfloat1622float2(v2[i]);
-              ov[u * 8 + 2 * i] = fmaf(pe[e], vf.x, ov[u * 8 + 2 * i]);
-              ov[u * 8 + 2 * i + 1] = fmaf(pe[e], vf.y, ov[u * 8 + 2 * i + 1]);
-            }
-          }
-        }
         if (live && l_tot > 0.f) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -384,7 +354,16 @@ void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a
   }
   const int G = a.Hq / a.Hkv;
   dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + kRowsU - 1) / kRowsU);
-  launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, a, a.status);
+  // the layer's draft-token caches as [positions of all requests, kv heads * hd] (a prefill has none: any valid map)
+  const CUtensorMap* tkx = tk;
+  const CUtensorMap* tvx = tv;
+  if (a.n_ext_max > 0) {
+    const long long rows = a.ext_rows_total, cols = (long long)a.Hkv * HD;
+    tkx = tma_map_bf16(a.k_ext, rows, cols, cols, kPosU);
+    tvx = tma_map_bf16(a.v_ext, rows, cols, cols, kPosU);
+    if (!tkx || !tvx) { static const int flag = kStInternal; cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st); return; }
+  }
+  launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, *tkx, *tvx, a, a.status);
 }
 
 }  // namespace

@@ -242,6 +242,9 @@ struct AttnArgs {
   int n_rows, max_tokens_per_row;
   int rows_expected;                            // 0, or the query rows per (request, kv head) the caller expects: tiling only
   long long ctx_rows_total;                     // requests * kv heads * positions of the layer's context cache
+  // the draft-token cache seen as positions: a request owns ext_positions consecutive positions (level-major, then beam
+  // slot), ext_pos_stride elements apart (all KV heads of a position are adjacent), ext_req_stride elements per request
+  int ext_positions; long long ext_pos_stride, ext_req_stride, ext_rows_total;
   int* status;
 };
 void launch_attention_simt(const AttnArgs& a, bool bf16, cudaStream_t st);
