@@ -2,19 +2,20 @@
 //
 // One CTA = (request, KV head, tile of 128 query rows): the rows are the request's tokens of this pass times the G query
 // heads of the group, so the context K/V is streamed once per 128 rows.  Per 64-position K/V tile (brought in by TMA,
-// 128-byte swizzle, 3-slot ring):
-//   S = Q K^T      tcgen05.mma M128 N64 K16 x hd/16, Q resident in shared memory, S in one of two 64-column TMEM buffers
+// 128-byte swizzle; K and V in rings of two slots each, because a K tile is free again right after S = Q K^T while
+// its V tile is needed until the end of the tile):
+//   S = Q K^T      tcgen05.mma M128 N64 K16 x hd/16, Q resident in shared memory, S in 64 TMEM columns
 //   softmax        4 warps, one thread per row (a TMEM lane is a row, so row maximum and row sum need no shuffles):
-//                  tcgen05.ld the row's 64 scores, base-2 exponentials against a running reference maximum that is only
-//                  raised when the true maximum has grown by more than 8 (then the O accumulator in TMEM is rescaled
-//                  with tcgen05.ld / st); P goes to one of two shared-memory buffers as the bf16 A operand of the
-//                  second product, so the softmax of tile j + 1 does not wait for the product of tile j
+//                  tcgen05.ld the row's 64 scores (after which S is free for the next tile's product, which therefore
+//                  runs under this tile's exponentials), base-2 exponentials against a running reference maximum that
+//                  is only raised when the true maximum has grown by more than 8 (then the O accumulator in TMEM is
+//                  rescaled with tcgen05.ld / st); P goes to shared memory as the bf16 A operand of the second product
 //   O += P V       tcgen05.mma M128 N=hd K16 x 4, V taken as it lies in the cache ([position][hd] = N-major operand)
-// The S product of tile j+1 is issued before the softmax of tile j is awaited, so the tensor pipe works under the
-// softmax.  The request's block of draft-token KV rows (every beam's, every level's) follows the context as further
-// tiles of the same loop; a row masks them with the bit set of the positions it may see (its own tuple's codes).  At
-// the end each thread normalises and stores its row.  Every mbarrier wait is bounded (abort flag, error status, TMEM
-// freed).
+// A CTA is a chain whose softmax takes most of a tile's time, so the kernel keeps every buffer single (65 KB of shared
+// memory and 128 TMEM columns at hd = 64, 113 KB and 256 at hd = 128) and lets three (two) CTAs share an SM instead.
+// The request's block of draft-token KV rows (every beam's, every level's) follows the context as further tiles of the
+// same loop; a row masks them with the bit set of the positions it may see (its own tuple's codes).  At the end each
+// thread normalises and stores its row.  Every mbarrier wait is bounded (abort flag, error status, TMEM freed).
 #include <math.h>
 
 #include "gemm_epilogue.cuh"
@@ -27,7 +28,8 @@ using namespace gemm_detail;
 
 constexpr int kPosU = 64;          // KV positions per tile
 constexpr int kRowsU = 128;        // query rows per CTA
-constexpr int kStagesU = 3;
+constexpr int kRingU = 2;          // K tiles in flight, and V tiles in flight (separate rings: K is free again after
+                                   // S = Q K^T, long before V, which waits for the end of the tile's softmax)
 constexpr int kThreadsU = 192;     // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: softmax (one thread per row)
 constexpr float kRaise = 8.f;      // the reference maximum follows the true one only in steps larger than this (log2 units)
 
@@ -35,9 +37,12 @@ template <int HD> struct UmmaCfg {
   static constexpr int kQBytes = kRowsU * HD * 2;
   static constexpr int kPBytes = kRowsU * kPosU * 2;
   static constexpr int kTileBytes = kPosU * HD * 2;            // one K (or V) tile
-  static constexpr int kStageBytes = 2 * kTileBytes;
-  static constexpr int kSmemBytes = kQBytes + 2 * kPBytes + kStagesU * kStageBytes + 1024 + 256;
-  static constexpr int kTmemCols = HD == 64 ? 256 : 256;       // S: 2 x 64 columns, O: HD columns; a power of two
+  // One S accumulator, one P buffer, two K and two V slots: 65 KB (hd 64) / 113 KB (hd 128) per CTA, so that three /
+  // two CTAs share an SM.  A CTA is a chain (S -> softmax -> P V per tile) whose softmax takes most of the tile's time;
+  // the S product of the next tile still runs under it (the scores leave TMEM at the start of the softmax), and
+  // concurrency comes from the CTAs that share the SM rather than from second buffers.
+  static constexpr int kSmemBytes = kQBytes + kPBytes + 2 * kRingU * kTileBytes + 1024 + 256;
+  static constexpr int kTmemCols = HD == 64 ? 128 : 256;       // S: 64 columns, O: HD columns; a power of two
   static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kPosU >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
   static constexpr uint32_t kIdescPV =
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) /* B is N-major */ | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
@@ -67,15 +72,15 @@ __device__ __forceinline__ float ex2u(float x) {
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 template <int HD>
-__global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
                                                              const __grid_constant__ CUtensorMap tmV,
                                                              const __grid_constant__ CUtensorMap tmKx,
                                                              const __grid_constant__ CUtensorMap tmVx, AttnArgs a, int* status) {
   using C = UmmaCfg<HD>;
-  constexpr int S = kStagesU;
+  constexpr int S = kRingU;
   constexpr int NH = HD / 64;                       // 64-column sub-tiles of a K / V / Q tile
   constexpr int KS = HD / 16;                       // k-steps of Q K^T
-  constexpr uint32_t kColS = 0, kColO = 128;        // TMEM columns: S buffers at 0 and 64, O at 128
+  constexpr uint32_t kColS = 0, kColO = 64;         // TMEM columns: S at 0, O at 64
 
   pdl_wait();                                       // before the first global read and before any exit
   pdl_launch();
@@ -103,22 +108,21 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_base = base, p_base = base + C::kQBytes, kv_base = p_base + 2 * C::kPBytes;   // two P buffers
-  const uint32_t bar_base = kv_base + S * C::kStageBytes;
-  auto kv_full = [&](int s) { return bar_base + 8u * s; };
-  auto kv_empty = [&](int s) { return bar_base + 8u * (S + s); };
-  auto s_full = [&](int b) { return bar_base + 8u * (2 * S + b); };
-  auto s_free = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
-  auto p_full = [&](int b) { return bar_base + 8u * (2 * S + 4 + b); };
-  auto pv_done = [&](int b) { return bar_base + 8u * (2 * S + 6 + b); };   // PV of tile j commits to pv_done(j & 1)
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - base) + 8 * (2 * S + 8));
+  const uint32_t q_base = base, p_base = base + C::kQBytes, k_base = p_base + C::kPBytes, v_base = k_base + S * C::kTileBytes;
+  const uint32_t bar_base = v_base + S * C::kTileBytes;
+  auto k_full = [&](int s) { return bar_base + 8u * s; };
+  auto k_empty = [&](int s) { return bar_base + 8u * (S + s); };
+  auto v_full = [&](int s) { return bar_base + 8u * (2 * S + s); };
+  auto v_empty = [&](int s) { return bar_base + 8u * (3 * S + s); };
+  // one phase per tile on each of these: tile j completes phase j (parity j & 1)
+  const uint32_t s_full = bar_base + 8u * (4 * S), s_free = s_full + 8u, p_full = s_full + 16u, pv_done = s_full + 24u;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - base) + 8 * (4 * S + 4));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(s_free(b), 4); }
-    for (int b = 0; b < 2; ++b) { mbar_init(p_full(b), 4); mbar_init(pv_done(b), 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
+    mbar_init(s_full, 1); mbar_init(s_free, 4); mbar_init(p_full, 4); mbar_init(pv_done, 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -155,59 +159,64 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int t = 0;
+      int t = 0, k_issued = 0, v_issued = 0;
       bool ok = true;
       for (; t < NT; ++t) {
         const int s = t % S;
-        if (t >= S && !mbar_wait_or_abort(kv_empty(s), ((t / S) - 1) & 1, abort_flag)) { ok = false; break; }
-        mbar_expect_tx(kv_full(s), C::kStageBytes);
+        const uint32_t par = (uint32_t)((t / S) - 1) & 1u;
+        const bool ctx_tile = t < n_tiles;
+        const int y = ctx_tile ? kv_row0 + t * kPosU : request * a.ext_positions + (t - n_tiles) * kPosU;
+        const int x0 = ctx_tile ? 0 : kvh * HD;      // the draft cache is [positions, kv heads * hd]: this head's columns
+        if (t >= S && !mbar_wait_or_abort(k_empty(s), par, abort_flag)) { ok = false; break; }
+        mbar_expect_tx(k_full(s), C::kTileBytes);
 #pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          const uint32_t kd = kv_base + s * C::kStageBytes + h * (kPosU * 128), vd = kd + C::kTileBytes;
-          if (t < n_tiles) {
-            tma_load_2d(kd, &tmK, h * 64, kv_row0 + t * kPosU, kv_full(s));
-            tma_load_2d(vd, &tmV, h * 64, kv_row0 + t * kPosU, kv_full(s));
-          } else {                                   // [positions, kv heads * hd]: this head's columns of 64 draft positions
-            const int y = request * a.ext_positions + (t - n_tiles) * kPosU;
-            tma_load_2d(kd, &tmKx, kvh * HD + h * 64, y, kv_full(s));
-            tma_load_2d(vd, &tmVx, kvh * HD + h * 64, y, kv_full(s));
-          }
-        }
+        for (int h = 0; h < NH; ++h)
+          tma_load_2d(k_base + s * C::kTileBytes + h * (kPosU * 128), ctx_tile ? &tmK : &tmKx, x0 + h * 64, y, k_full(s));
+        ++k_issued;
+        if (t >= S && !mbar_wait_or_abort(v_empty(s), par, abort_flag)) { ok = false; break; }
+        mbar_expect_tx(v_full(s), C::kTileBytes);
+#pragma unroll
+        for (int h = 0; h < NH; ++h)
+          tma_load_2d(v_base + s * C::kTileBytes + h * (kPosU * 128), ctx_tile ? &tmV : &tmVx, x0 + h * 64, y, v_full(s));
+        ++v_issued;
       }
-      if (!ok) {
+      if (!ok) {                                     // drain the copies still in flight before the CTA's memory goes away
         *abort_flag = 1;
-        for (int j = max(0, t - S); j < t; ++j) mbar_wait(kv_full(j % S), (j / S) & 1);
+        for (int j = max(0, k_issued - S); j < k_issued; ++j) mbar_wait(k_full(j % S), (j / S) & 1);
+        for (int j = max(0, v_issued - S); j < v_issued; ++j) mbar_wait(v_full(j % S), (j / S) & 1);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = true;
-      auto issue_s = [&](int j) {                    // S_j = Q K_j^T into S buffer j & 1
-        const int s = j % S, b = j & 1;
-        if (!mbar_wait_or_abort(kv_full(s), (j / S) & 1, abort_flag)) return false;
-        if (j >= 2 && !mbar_wait_or_abort(s_free(b), ((j >> 1) - 1) & 1, abort_flag)) return false;
+      auto issue_s = [&](int j) {                    // S_j = Q K_j^T (the one S accumulator)
+        const int s = j % S;
+        if (!mbar_wait_or_abort(k_full(s), (uint32_t)(j / S) & 1u, abort_flag)) return false;
+        if (j >= 1 && !mbar_wait_or_abort(s_free, (uint32_t)(j - 1) & 1u, abort_flag)) return false;   // scores of tile j - 1 are in registers
         tc_fence_after();
-        const uint32_t kt = kv_base + s * C::kStageBytes;
+        const uint32_t kt = k_base + s * C::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks)
-          tc_mma(tmem_base + kColS + (uint32_t)(b * kPosU), smem_desc(q_base + (ks >> 2) * (kRowsU * 128) + (ks & 3) * 32),
+          tc_mma(tmem_base + kColS, smem_desc(q_base + (ks >> 2) * (kRowsU * 128) + (ks & 3) * 32),
                  smem_desc(kt + (ks >> 2) * (kPosU * 128) + (ks & 3) * 32), C::kIdescS, ks > 0 ? 1u : 0u);
-        tc_commit(s_full(b));
+        tc_commit(k_empty(s));                       // K_j may be overwritten
+        tc_commit(s_full);
         return true;
       };
       if (NT > 0) ok = issue_s(0);
       for (int j = 0; j < NT && ok; ++j) {
         if (j + 1 < NT && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
-        if (!mbar_wait_or_abort(p_full(j & 1), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_or_abort(p_full, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_or_abort(v_full(j % S), (uint32_t)(j / S) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t vt = kv_base + (j % S) * C::kStageBytes + C::kTileBytes;
+        const uint32_t vt = v_base + (j % S) * C::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < kPosU / 16; ++ks)
-          tc_mma(tmem_base + kColO, smem_desc(p_base + (j & 1) * C::kPBytes + ks * 32), smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128), C::kIdescPV,
+          tc_mma(tmem_base + kColO, smem_desc(p_base + ks * 32), smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128), C::kIdescPV,
                  (j > 0 || ks > 0) ? 1u : 0u);
-        tc_commit(kv_empty(j % S));                  // K_j and V_j are no longer needed
-        tc_commit(pv_done(j & 1));                   // O holds tiles 0..j
+        tc_commit(v_empty(j % S));                   // V_j may be overwritten
+        tc_commit(pv_done);                          // O holds tiles 0..j, and P may be overwritten
       }
       if (!ok) *abort_flag = 1;
     }
@@ -226,25 +235,25 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       xpos[e] = off >= 0 ? (int)((off - (long long)request * a.ext_req_stride) / a.ext_pos_stride) : -1;
     }
     for (int j = 0; j < NT; ++j) {
-      const int b = j & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full(b), (j >> 1) & 1, abort_flag));
+      const uint32_t par = (uint32_t)j & 1u, par_prev = par ^ 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full, par, abort_flag));
       if (!ok) break;
       if (warp_dead) {                               // (its P rows stay whatever they are: O rows nobody reads)
-        if (lane == 0) mbar_arrive(s_free(b));
-        if (j >= 2) {
-          ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done(b), ((j >> 1) - 1) & 1, abort_flag));
+        if (lane == 0) mbar_arrive(s_free);
+        if (j >= 1) {
+          ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, par_prev, abort_flag));
           if (!ok) break;
         }
-        if (lane == 0) mbar_arrive(p_full(b));
+        if (lane == 0) mbar_arrive(p_full);
         continue;
       }
       tc_fence_after();
       float sv[kPosU];
-      tmem_ld32(tmem_base + lane_addr + kColS + (uint32_t)(b * kPosU), sv);
-      tmem_ld32(tmem_base + lane_addr + kColS + (uint32_t)(b * kPosU + 32), sv + 32);
+      tmem_ld32(tmem_base + lane_addr + kColS, sv);
+      tmem_ld32(tmem_base + lane_addr + kColS + 32u, sv + 32);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(s_free(b));         // the scores are in registers: the buffer may take tile j + 2
+      if (lane == 0) mbar_arrive(s_free);            // the scores are in registers: S may take tile j + 1
       if (j >= n_tiles) {                            // a tile of draft positions: the row's own mask
         unsigned long long mk = 0ull;
 #pragma unroll
@@ -280,13 +289,11 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       }
       l_run = l_run * corr + rs;
       m_ref = m_new;
-      if (j >= 2) {                                  // P buffer b was read by the PV product of tile j - 2
-        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done(b), ((j >> 1) - 1) & 1, abort_flag));
+      if (j >= 1) {                                  // the PV product of tile j - 1 is done: P is free, O holds every earlier tile
+        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, par_prev, abort_flag));
         if (!ok) break;
       }
-      if (j > 0 && __any_sync(0xffffffffu, raise)) { // rescale O: it must hold every earlier tile first
-        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done(b ^ 1), ((j - 1) >> 1) & 1, abort_flag));
-        if (!ok) break;
+      if (j > 0 && __any_sync(0xffffffffu, raise)) { // rescale O
         tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < HD / 32; ++c) {
@@ -299,15 +306,15 @@ __global__ void __launch_bounds__(kThreadsU) attn_umma_kernel(const __grid_const
       }
 #pragma unroll
       for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(gen_base + (p_base - base) + b * C::kPBytes + row * 128 + ((c ^ (row & 7)) << 4)) =
+        *reinterpret_cast<uint4*>(gen_base + (p_base - base) + row * 128 + ((c ^ (row & 7)) << 4)) =
             make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full(b));
+      if (lane == 0) mbar_arrive(p_full);
     }
     if (ok && NT > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done((NT - 1) & 1), ((NT - 1) >> 1) & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, (uint32_t)(NT - 1) & 1u, abort_flag));
       tc_fence_after();
     }
     if (!ok) { if (lane == 0) *abort_flag = 1; }
