@@ -89,6 +89,7 @@ struct nezha_ctx {
   int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
+  int chains_now;           // GemmArgs::chains of the products being queued: 2 inside a decode call, 0 otherwise
   int rounds_seen[3];       // rounds the last decode call of each mode needed: that many are launched without waiting
   int state;                // 0 created, 1 hash set built, 2 prefilled
   int batch;                // prefilled batch
@@ -253,6 +254,7 @@ size_t carve(nezha_ctx* c) {
 void gemm(nezha_ctx* c, const void* A, long long lda, const void* W, long long ldw, void* C, long long ldc, long long M,
           const int* M_dev, int N, int K, int epi, const float* bias = nullptr) {
   GemmArgs a{A, lda, W, ldw, C, ldc, (int)M, M_dev, N, K, epi, bias, c->es.status};
+  a.chains = c->chains_now;
   if (c->bf16 && gemm_tc_supported(a)) launch_gemm_tc(a, c->st);
   else launch_gemm_simt(a, c->bf16, c->st);
 }
@@ -266,6 +268,7 @@ int gemm_fused(nezha_ctx* c, const void* A, long long lda, const void* W, void* 
   if (extra) a.f = *extra;
   a.f.ss_in = ss_in; a.f.ss_in_parts = ss_parts; a.f.ss_ld = c->Ms; a.f.inv_dim = 1.f / (float)c->d; a.f.eps = c->cfg.rms_eps;
   a.M_expected = c->m_expected;
+  a.chains = c->chains_now;
   launch_gemm_tc(a, c->st);
   return N / 32;
 }
@@ -516,6 +519,14 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     return fail(c, NEZHA_ERR_ARG, "nezha_decode: bad batch / beam_width / mode / output pointer");
   const EngineState& e = c->es;
   const int L = c->L;
+  // Every product of a decode call asks for the two-partial-sum order on narrow outputs (two MMA issuers): the
+  // choice is per call path, never per launch, so that the speculative and the autoregressive mode, whose passes differ
+  // in size, still compute the same bits.  The prefill keeps the plain order and the widest tiles.
+  struct ChainScope {
+    nezha_ctx* c;
+    explicit ChainScope(nezha_ctx* c_) : c(c_) { c->chains_now = 2; }
+    ~ChainScope() { c->chains_now = 0; }
+  } chain_scope(c);
   nezha_trace tr{};
   if (trace) tr = *trace;
   nezha_decode_stats sd{};
@@ -648,6 +659,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   c->m_expected = 0;
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
+  c->chains_now = 0;
   c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }

@@ -188,6 +188,11 @@ struct GemmArgs {
   int* status;           // device status word (bounded waits report here)
   GemmFuse f;            // zero-initialised unless a fused epilogue is asked for
   int M_expected;        // 0, or the row count the caller expects on the device (<= M): only shapes the tiling
+  // 0: the K range is accumulated in order.  2: products with N <= 1024 accumulate it in two interleaved partial sums
+  // (k-step k goes to sum k mod 2), added at the end, so that two MMA issuers can run the k-loop.  The two orders round
+  // differently: a caller that needs the same bits from launches of different sizes asks for the same value in all of
+  // them (the tiling itself never changes the result).
+  int chains;
 };
 
 void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);

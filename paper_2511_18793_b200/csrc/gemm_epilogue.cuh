@@ -204,7 +204,9 @@ __device__ __forceinline__ EpiRow epilogue_row(const GemmArgs& a, int row, int M
 // One epilogue warp's share of a finished accumulator: TMEM lanes [32 q, 32 q + 32) (= rows m0 + 32 q ..) and the
 // 32-column groups half, half + 2, ... of the BN columns starting at TMEM column `tmem_acc`.  er = epilogue_row of
 // the lane's own row (lane = row while the block comes out of TMEM).
-template <int BN, int EPI>
+// CHAINS > 1: the tile's K range was accumulated in that many partial accumulators, BN columns apart (one per MMA
+// issuer); they are added up here, in order, as the block leaves TMEM.
+template <int BN, int EPI, int CHAINS = 1>
 __device__ __forceinline__ void drain_accumulator(const GemmArgs& a, uint32_t tmem_acc, int q, int half, int lane,
                                                   float4* stg4, int m0, int n0, int M, const EpiRow& er) {
   const int row = m0 + q * 32 + lane;
@@ -215,6 +217,13 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& a, uint32_t tm
     if (n_chunk >= a.N) break;                               // ragged last tile (N is a multiple of 32)
     float v[32];
     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+#pragma unroll
+    for (int ch = 1; ch < CHAINS; ++ch) {
+      float w[32];
+      tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * BN + c * 32), w);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += w[j];
+    }
     // transpose through shared memory: from lane = row (how TMEM hands the block out) to 8 lanes per row
 #pragma unroll
     for (int j = 0; j < 8; ++j)

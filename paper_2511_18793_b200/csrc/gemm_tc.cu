@@ -36,11 +36,19 @@ template <int BN> struct Cfg {
 };
 
 
-template <int BN, int EPI>
-__global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                           const __grid_constant__ CUtensorMap tmB, GemmArgs a,
-                                                           int* status) {
+// ISS = number of MMA-issuing warps.  The tensor pipe takes a tcgen05.mma of M = 128 about every 76 cycles whatever
+// its N, and one issuing thread adds its own barrier wait, fence and commit to every k-step, during which the pipe
+// idles: the k-loop of a tile of at most 128 columns is bound by that chain, not by data or flops.  With ISS = 2 the
+// warps 1 and 2 take the k-steps alternately, each into an accumulator of its own (added up by the epilogue), so one
+// issuer's overhead runs under the other's MMAs.
+template <int BN, int EPI, int ISS>
+__global__ void __launch_bounds__(kThreads + 32 * (ISS - 1)) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                            const __grid_constant__ CUtensorMap tmB,
+                                                                            GemmArgs a, int* status) {
   using C = Cfg<BN>;
+  constexpr int kTmemCols = 2 * BN * ISS < 32 ? 32 : 2 * BN * ISS;   // two accumulators of ISS chains each
+  static_assert(2 * BN * ISS <= 512 && ISS <= C::kStages, "accumulator chains do not fit");
+  constexpr int kFirstEpiWarp = 1 + ISS;
   constexpr int STAGES = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -60,7 +68,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kEpiWarps); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), ISS); mbar_init(acc_empty(b), kEpiWarps); }
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_map(&tmA);
@@ -68,7 +76,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
-                 "r"(C::kTmemCols));
+                 "r"(kTmemCols));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
   tc_fence_before();
@@ -106,11 +114,11 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
         for (int j = max(0, it - STAGES); j < it; ++j) mbar_wait(full_bar(j % STAGES), (j / STAGES) & 1);
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp <= ISS) {
+    // ------------------------------------------------------------------ MMA issuers (warp i takes k-steps i-1, i-1+ISS, ...)
     if (lane == 0) {
-      int t_local = 0, s = 0;
-      uint32_t round = 0;
+      const int chain = warp - 1;
+      int t_local = 0;
       bool ok = true;
       // descriptors of slot 0; a slot further on adds its byte offset / 16 to the address field (shared memory
       // addresses stay below 2^18, so the 14-bit field never carries)
@@ -119,24 +127,28 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
         const int b = t_local & 1;
         if (t_local >= 2 && !mbar_wait_or_abort(acc_empty(b), ((t_local >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t tmem_acc = tmem_base + (uint32_t)(b * BN);
-        for (int k = 0; k < k_iters; ++k) {
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(b * BN * ISS + chain * BN);
+        const int it0 = t_local * k_iters + chain;   // this issuer's first k-step of the tile, counted over the CTA's tiles
+        int s = it0 % STAGES;
+        uint32_t round = (uint32_t)(it0 / STAGES) & 1u;
+        for (int k = chain; k < k_iters; k += ISS) {
           if (!mbar_wait_or_abort(full_bar(s), round, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint64_t so = (uint64_t)(s * (C::kStageBytes >> 4));
-          tc_mma_kstep(tmem_acc, da0 + so, db0 + so, C::kInstrDesc, k > 0 ? 1u : 0u);
+          tc_mma_kstep(tmem_acc, da0 + so, db0 + so, C::kInstrDesc, k >= ISS ? 1u : 0u);
           tc_commit(empty_bar(s));               // slot free once these MMAs have read it
-          if (++s == STAGES) { s = 0; round ^= 1u; }
+          s += ISS;
+          if (s >= STAGES) { s -= STAGES; round ^= 1u; }
         }
-        if (ok) tc_commit(acc_full(b));          // accumulator complete
+        if (ok) tc_commit(acc_full(b));          // this issuer's share of the accumulator is complete
       }
       if (!ok) *abort_flag = 1;
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // ------------------------------------------------------------------ epilogue (the last 8 warps)
     const int q = warp & 3;                      // TMEM lane quarter this warp may access
-    const int half = (warp - 2) >> 2;            // which half of the tile's 32-column groups this warp takes
-    float4* stg4 = reinterpret_cast<float4*>(gen_base + STAGES * C::kStageBytes + 256) + (warp - 2) * (32 * 8);
+    const int half = (warp - kFirstEpiWarp) >> 2;   // which half of the tile's 32-column groups this warp takes
+    float4* stg4 = reinterpret_cast<float4*>(gen_base + STAGES * C::kStageBytes + 256) + (warp - kFirstEpiWarp) * (32 * 8);
     int t_local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
@@ -147,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
       ok = __all_sync(0xffffffffu, mbar_wait_or_abort(acc_full(b), (t_local >> 1) & 1, abort_flag));   // warp-uniform
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator<BN, EPI>(a, tmem_base + (uint32_t)(b * BN), q, half, lane, stg4, m0, n0, M, er);
+      drain_accumulator<BN, EPI, ISS>(a, tmem_base + (uint32_t)(b * BN * ISS), q, half, lane, stg4, m0, n0, M, er);
       // this warp is done reading the accumulator: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
@@ -160,7 +172,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_kernel(const __grid_constant
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols));
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols));
   }
   if (threadIdx.x == 0 && *abort_flag) atomicOr(status, kStInternal);
 }
@@ -178,7 +190,7 @@ int sm_count() {
   return n;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int ISS>
 void launch(const GemmArgs& a, cudaStream_t st) {
   const CUtensorMap* ta = tma_map_bf16(a.A, a.M, a.K, a.lda, BM);
   const CUtensorMap* tb = tma_map_bf16(a.W, a.N, a.K, a.ldw, BN);
@@ -189,24 +201,24 @@ void launch(const GemmArgs& a, cudaStream_t st) {
   }
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
+    cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI, ISS>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
     configured = true;
   }
   const long long tiles = (long long)((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  launch_pdl(gemm_tc_kernel<BN, EPI>, dim3(grid), dim3(kThreads), Cfg<BN>::kSmemBytes, st, *ta, *tb, a, a.status);
+  launch_pdl(gemm_tc_kernel<BN, EPI, ISS>, dim3(grid), dim3(kThreads + 32 * (ISS - 1)), Cfg<BN>::kSmemBytes, st, *ta, *tb, a, a.status);
 }
 
-template <int BN>
+template <int BN, int ISS>
 void launch_bn(const GemmArgs& a, cudaStream_t st) {
   switch (a.epilogue) {
-    case kEpiStoreAct: launch<BN, kEpiStoreAct>(a, st); break;
-    case kEpiStoreF32: launch<BN, kEpiStoreF32>(a, st); break;
-    case kEpiAddF32: launch<BN, kEpiAddF32>(a, st); break;
-    case kEpiBiasTanhF32: launch<BN, kEpiBiasTanhF32>(a, st); break;
-    case kEpiSwiGLU: launch<BN, kEpiSwiGLU>(a, st); break;
-    case kEpiAddNorm: launch<BN, kEpiAddNorm>(a, st); break;
-    case kEpiRopeKV: launch<BN, kEpiRopeKV>(a, st); break;
+    case kEpiStoreAct: launch<BN, kEpiStoreAct, ISS>(a, st); break;
+    case kEpiStoreF32: launch<BN, kEpiStoreF32, ISS>(a, st); break;
+    case kEpiAddF32: launch<BN, kEpiAddF32, ISS>(a, st); break;
+    case kEpiBiasTanhF32: launch<BN, kEpiBiasTanhF32, ISS>(a, st); break;
+    case kEpiSwiGLU: launch<BN, kEpiSwiGLU, ISS>(a, st); break;
+    case kEpiAddNorm: launch<BN, kEpiAddNorm, ISS>(a, st); break;
+    case kEpiRopeKV: launch<BN, kEpiRopeKV, ISS>(a, st); break;
     default: break;
   }
 }
@@ -252,12 +264,35 @@ void launch_gemm_tc_pair(const GemmArgs& a, int n_sm, cudaStream_t st);
 
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
   LaunchScope ls(kcGemm, st);
-  switch (gemm_tc_plan(a.M_expected > 0 && a.M_expected < a.M ? a.M_expected : a.M, a.N)) {
+  const int m_plan = a.M_expected > 0 && a.M_expected < a.M ? a.M_expected : a.M;
+  // Narrow outputs (N <= 1024) never fill a 256-wide tile well and their k-loops are bound by the MMA issue chain:
+  // a caller that asks for two partial sums gets tiles of at most 128 columns with two issuers for them.  The rule
+  // looks at N and K only, never at M or at the tiling, so such a product keeps its summation order (and its bits)
+  // whatever the number of rows of a launch -- what lets two decode modes whose passes differ in size agree exactly.
+  static const bool one_issuer = getenv("NEZHA_ONE_MMA_ISSUER") != nullptr;
+  if (a.chains == 2 && a.N <= 1024 && a.K >= 2 * BK && !one_issuer) {
+    const long long tiles_m = (m_plan + BM - 1) / BM;
+    static const int widths[3] = {128, 64, 32}, wave_cost[3] = {400, 300, 250};
+    long long best = -1; int plan = 32;
+    for (int i = 0; i < 3; ++i) {
+      if (widths[i] > 32 && a.N < widths[i]) continue;
+      const long long tiles = tiles_m * ((a.N + widths[i] - 1) / widths[i]);
+      const long long cost = ((tiles + sm_count() - 1) / sm_count()) * wave_cost[i];
+      if (best < 0 || cost < best) { best = cost; plan = widths[i]; }
+    }
+    switch (plan) {
+      case 128: launch_bn<128, 2>(a, st); break;
+      case 64: launch_bn<64, 2>(a, st); break;
+      default: launch_bn<32, 2>(a, st); break;
+    }
+    return;
+  }
+  switch (gemm_tc_plan(m_plan, a.N)) {
     case kPlanPairs: launch_gemm_tc_pair(a, sm_count(), st); break;
-    case 256: launch_bn<256>(a, st); break;
-    case 128: launch_bn<128>(a, st); break;
-    case 64: launch_bn<64>(a, st); break;
-    default: launch_bn<32>(a, st); break;
+    case 256: launch_bn<256, 1>(a, st); break;
+    case 128: launch_bn<128, 1>(a, st); break;
+    case 64: launch_bn<64, 1>(a, st); break;
+    default: launch_bn<32, 1>(a, st); break;
   }
 }
 
