@@ -213,7 +213,9 @@ nezha_status nezha_select(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_
  * storage type (device pointers, row-major, leading dimensions = K for A and W, N for C).
  *   epilogue 0: C (storage type) = acc;  1: C (float) = acc;  2: C (float) += acc;  3: C (float) = tanh(acc + bias[n])
  *   path     0: the engine's own choice; 1: CUDA-core kernel; 2: tcgen05 kernel (NEZHA_ERR_UNSUPPORTED if the shape
- *               is not covered: bf16 storage, K % 64 == 0, N % 128 == 0)
+ *               is not covered: bf16 storage, K % 64 == 0, N % 32 == 0); 3: the tcgen05 kernel as the decode calls use
+ *               it: for N <= 1024 the K range is accumulated in two interleaved partial sums (two MMA issuers), which
+ *               rounds differently from path 2 in the last bits
  * Used by every projection of the primary model (Algorithm 1's model call), the LM head and the draft head
  * (Eq. 2-3).  Asynchronous. */
 nezha_status nezha_gemm(nezha_ctx* ctx, const void* A, const void* W, void* C, int32_t M, int32_t N, int32_t K,

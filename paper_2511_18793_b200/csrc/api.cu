@@ -925,11 +925,12 @@ nezha_status nezha_gemm(nezha_ctx* c, const void* A, const void* W, void* C, int
                         int32_t epilogue, const float* bias, int32_t path) {
   if (!c) return NEZHA_ERR_ARG;
   if (!A || !W || !C || M < 1 || N < 1 || K < 1 || epilogue < 0 || epilogue > 3 || (epilogue == 3 && !bias) || path < 0 ||
-      path > 2)
+      path > 3)
     return fail(c, NEZHA_ERR_ARG, "nezha_gemm: bad argument");
   GemmArgs a{A, K, W, K, C, N, M, nullptr, N, K, epilogue, bias, c->es.status};
+  a.chains = path == 3 ? 2 : 0;
   const bool tc_ok = c->bf16 && gemm_tc_supported(a);
-  if (path == 2 && !tc_ok) return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: shape not covered by the tcgen05 kernel");
+  if (path >= 2 && !tc_ok) return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: shape not covered by the tcgen05 kernel");
   if (path != 1 && tc_ok) launch_gemm_tc(a, c->st);
   else launch_gemm_simt(a, c->bf16, c->st);
   NZ_CUDA(c, cudaGetLastError());

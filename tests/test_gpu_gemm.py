@@ -23,7 +23,7 @@ def _ref(A, W):
                                     (1, 128, 64), (129, 128, 4864),
                                     # large enough for the CTA-pair kernel (256 x 256 tiles), ragged in M and in N
                                     (5000, 2304, 896), (18000, 1152, 512), (4100, 512, 2048)])
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 2, 3])
 def test_gemm_epilogues(ctx, M, N, K, path):
     g = torch.Generator(device="cuda"); g.manual_seed(M * 7 + N * 3 + K)
     A = (torch.randn(M, K, generator=g, device="cuda") * 0.5).bfloat16()
