@@ -217,12 +217,16 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
       if (c >= l_cnt[r]) continue;
       const float sv = l_score[i];
       const int t = l_tok[i];
-      int rank = c;                                        // its own list is sorted: c of its entries come before it
-      for (int r2 = 0; r2 < nb; ++r2) {
+      // Its own list is sorted: c of its entries come before it.  In another list the entries that beat it are a prefix
+      // (the list is sorted and the parent rank breaks ties), so the scan of a list stops at the first entry that does
+      // not, and the whole count stops once the candidate is known to miss the best K.
+      int rank = c;
+      for (int r2 = 0; r2 < nb && rank < a.K; ++r2) {
         if (r2 == r) continue;
         const int n2 = l_cnt[r2];
-        for (int c2 = 0; c2 < n2; ++c2)
-          rank += cand_better(l_score[(size_t)r2 * a.K + c2], r2, l_tok[(size_t)r2 * a.K + c2], sv, r, t) ? 1 : 0;
+        int c2 = 0;
+        while (c2 < n2 && cand_better(l_score[(size_t)r2 * a.K + c2], r2, l_tok[(size_t)r2 * a.K + c2], sv, r, t)) ++c2;
+        rank += c2;
       }
       if (rank < a.K) { sel_s[rank] = sv; sel_r[rank] = r; sel_t[rank] = t; }
     }
