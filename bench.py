@@ -145,7 +145,10 @@ def algorithmic_work(w, stats_tokens_per_step, rounds):
     # attention: the context KV of a request is read once per (request, layer, pass); queries and outputs once
     attn_bytes = rounds * nl * w.batch * (2 * Hkv * P * hd * esz) + stats_tokens_per_step * nl * 2 * Hq * hd * esz
     attn_flops = 4.0 * stats_tokens_per_step * nl * Hq * hd * (P + 2)
-    return {"gemm_flops": gemm_flops, "attention_bytes": attn_bytes, "attention_flops": attn_flops}
+    # the weights of every projection (and of the LM head rows used) are read once per pass
+    gemm_weight_bytes = rounds * (per_tok_params + lm) * esz
+    return {"gemm_flops": gemm_flops, "attention_bytes": attn_bytes, "attention_flops": attn_flops,
+            "gemm_weight_bytes": gemm_weight_bytes}
 
 
 def probe_bench(args, w, eng, cat_dev, config, dev):
@@ -395,6 +398,14 @@ def main():
     if rec and rec["kernel_rev"] == KERNEL_REV.get(dom):
         roof["traffic"] = rec["dram_bytes_per_launch"]
         roof["traffic_source"] = rec["source"]
+    # the whole step against its floor: per class the larger of (bytes / copy bandwidth) and (flops / tensor peak),
+    # summed over the GEMM and attention classes (the rest moves kilobytes), divided by the measured step time
+    if w.dtype == "bf16" and args.mode != 0:
+        tf, bw = peaks["bf16_tflops_sustained"] * 1e12, peaks["hbm_gbs"] * 1e9
+        floor_s = max(work["gemm_flops"] / tf, work["gemm_weight_bytes"] / bw) + \
+            max(work["attention_flops"] / tf, work["attention_bytes"] / bw)
+        roof["step_floor_ms"] = floor_s * 1e3
+        roof["step_frac"] = floor_s * 1e3 / (total_ms_max / args.steps)
     roof["classes"] = shares
     roof["attention_gbs"] = work["attention_bytes"] / (shares["attention"]["ms_per_step"] / 1e3) / 1e9 if "attention" in shares else None
     roof["gemm_tflops"] = work["gemm_flops"] / (shares["gemm"]["ms_per_step"] / 1e3) / 1e12 if "gemm" in shares else None
