@@ -19,6 +19,7 @@ void launch_hs_pack(const LevelInfo& li, const int* codes, unsigned long long n,
                     cudaStream_t st);
 void launch_hs_insert(const LevelInfo& li, HashSetView hs, const int* codes, unsigned long long n,
                       unsigned long long* n_unique, int* status, cudaStream_t st);
+void launch_pm_build(const LevelInfo& li, PrefixMapView pm, const int* codes, unsigned long long n, int* status, cudaStream_t st);
 void launch_hs_probe(HashSetView hs, const unsigned long long* keys, unsigned long long n, uint8_t* found,
                      cudaStream_t st);
 void launch_prefill_tokens(const EngineState& e, const int* hist, const int* n_hist, int b0, int rows, int max_n,
@@ -87,6 +88,7 @@ struct nezha_ctx {
   std::map<std::array<uintptr_t, 16>, Segment> segments;
   bool use_graphs;
   int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
+  int opt_mask;             // nezha_set_option: 0 = the last-level mask probes the hash set, 1 = it reads the prefix map
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
   int chains_now;           // GemmArgs::chains of the products being queued: 2 inside a decode call, 0 otherwise
@@ -173,6 +175,16 @@ size_t carve(nezha_ctx* c) {
   c->n_unique_dev = cv.take<unsigned long long>(1);
   e.hs.n_buckets = bucket_count(c->n_items, c->load_factor);
   e.hs.slots = cv.take<unsigned long long>(e.hs.n_buckets * kBucketSlots);
+  {  // prefix map: at most one slot per item and per possible prefix, at the hash set's load factor
+    double prefixes = 1.0;
+    for (int l = 0; l + 1 < g.L; ++l) prefixes *= (double)g.T[l];
+    const double n_pref = prefixes < (double)(c->n_items ? c->n_items : 1) ? prefixes : (double)(c->n_items ? c->n_items : 1);
+    e.pm.n_slots = (unsigned long long)ceil(n_pref / c->load_factor) + 1;
+    int words = 1 + (g.T[g.L - 1] + 63) / 64, stride = 2;
+    while (stride < words) stride *= 2;
+    e.pm.stride = stride;
+    e.pm.slots = cv.take<unsigned long long>(e.pm.n_slots * (unsigned long long)stride);
+  }
   // weights
   const size_t esz = c->esz;
   c->embed = cv.take_bytes((size_t)c->vocab * c->d * esz);
@@ -411,6 +423,7 @@ SelectArgs select_base(nezha_ctx* c, int batch, int K) {
   SelectArgs s{};
   s.in_stride = c->Kmax; s.out_stride = c->Kmax; s.K = K; s.tuple_len = c->L; s.batch = batch;
   s.li = c->es.li; s.hs = c->es.hs;
+  if (c->opt_mask == 1) s.pm = c->es.pm;
   return s;
 }
 
@@ -533,7 +546,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
   const int R = L - 1;
   auto key_of = [&](int segment) {
     std::array<uintptr_t, 16> k{};
-    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16);
+    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20);
     k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
     k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
     k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams; k[14] = (uintptr_t)tr.beam_scores;
@@ -660,7 +673,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
   c->chains_now = 0;
-  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1;
+  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 0;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;
@@ -746,6 +759,7 @@ nezha_status nezha_build_hashset(nezha_ctx* c, uint64_t* n_unique) {
   NZ_CUDA(c, cudaMemsetAsync(c->n_unique_dev, 0, sizeof(unsigned long long), c->st));
   launch_hs_clear(c->es.hs, c->st);
   launch_hs_insert(c->es.li, c->es.hs, c->catalog, c->n_items, c->n_unique_dev, c->es.status, c->st);
+  launch_pm_build(c->es.li, c->es.pm, c->catalog, c->n_items, c->es.status, c->st);
   unsigned long long nu = 0;
   NZ_CUDA(c, cudaMemcpyAsync(&nu, c->n_unique_dev, sizeof(nu), cudaMemcpyDeviceToHost, c->st));
   NZ_CUDA(c, cudaStreamSynchronize(c->st));
@@ -831,6 +845,9 @@ nezha_status nezha_set_option(nezha_ctx* c, int32_t option, int32_t value) {
     case NEZHA_OPT_DRAFT_FILTER:
       if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: filter must be 0 or 1");
       c->opt_filter = value; break;
+    case NEZHA_OPT_FINAL_MASK:
+      if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: final mask must be 0 or 1");
+      c->opt_mask = value; break;
     default: return fail(c, NEZHA_ERR_ARG, "nezha_set_option: unknown option");
   }
   return NEZHA_OK;

@@ -138,7 +138,14 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
         if (all_codes) key[j] += base;                   // rank by cumulative log-probability
       }
     }
-    if (all_codes && a.filter) {                         // Eq. 5 on every extension of the beam, 8 probes in flight
+    if (all_codes && a.filter && a.pm.slots) {           // Eq. 5 on every extension of the beam: the prefix's bit set
+      const unsigned long long* bits = pm_find(a.pm, prefix_key);
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) {
+        const int t = lane + 32 * j;
+        if (t < a.T && !pm_test(bits, t)) key[j] = -INFINITY;
+      }
+    } else if (all_codes && a.filter) {                  // Eq. 5 on every extension of the beam, 8 probes in flight
       constexpr int PB = VPL < 8 ? VPL : 8;
 #pragma unroll
       for (int j0 = 0; j0 < VPL; j0 += PB) {
@@ -187,7 +194,8 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
         bool ok = false; float sv = 0.f; int t = 0;
         if (c < cnt) {
           sv = l_score[(size_t)r * a.K + c]; t = l_tok[(size_t)r * a.K + c];
-          ok = hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
+          ok = a.pm.slots ? pm_test(pm_find(a.pm, prefix_key), t)
+                          : hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
         }
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         __syncwarp();

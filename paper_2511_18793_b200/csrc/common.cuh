@@ -132,6 +132,34 @@ __device__ __forceinline__ void hs_contains_many(const HashSetView& hs, const un
 }
 
 // --------------------------------------------------------------------------------------------------
+// prefix map: the same set V, regrouped as (prefix of L-1 codes) -> bit set of the valid last codes
+// --------------------------------------------------------------------------------------------------
+// Open addressing with linear probing over slots of `stride` words: word 0 = prefix key + 1 (0 = empty), words 1.. =
+// the bits of the last codes t with (prefix, t) in V.  The final-level mask of a beam then needs one look-up instead
+// of T_L hash probes; its answers are those of the hash set, bit for bit.
+struct PrefixMapView {
+  unsigned long long* slots;       // [n_slots * stride]; null = not in use
+  unsigned long long n_slots;
+  int stride;                      // words per slot: a power of two >= 1 + ceil(T_L / 64)
+};
+// The bit set of a prefix, or null if no item has it.  Every lane of a warp may call this with the same key (the
+// loads are then broadcasts).
+__device__ __forceinline__ const unsigned long long* pm_find(const PrefixMapView& pm, unsigned long long prefix_key) {
+  unsigned long long s = __umul64hi(hs_mix(prefix_key), pm.n_slots);
+  for (int step = 0; step < kMaxProbeBuckets; ++step) {
+    const unsigned long long* slot = pm.slots + s * pm.stride;
+    const unsigned long long k = __ldg(slot);
+    if (k == prefix_key + 1) return slot + 1;
+    if (k == 0ull) return nullptr;
+    if (++s == pm.n_slots) s = 0;
+  }
+  return nullptr;
+}
+__device__ __forceinline__ bool pm_test(const unsigned long long* bits, int t) {
+  return bits != nullptr && ((__ldg(bits + (t >> 6)) >> (t & 63)) & 1ull);
+}
+
+// --------------------------------------------------------------------------------------------------
 // model / engine description shared by the host code and the kernels
 // --------------------------------------------------------------------------------------------------
 struct LevelInfo {

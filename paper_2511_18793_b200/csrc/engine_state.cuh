@@ -12,6 +12,7 @@ struct EngineState {
   int Bmax, Kmax, L, d, Hkv, hd;
   LevelInfo li;
   HashSetView hs;
+  PrefixMapView pm;
   int* status;
   // draft-head variants (the ablations of Section 4.3); defaults 1, 1, 0 = Eq. 2 and Eq. 3 as printed
   int draft_use_h, draft_use_s, draft_additive;
@@ -63,6 +64,7 @@ struct SelectArgs {
   int tuple_len;                        // row length of in_codes / out_codes (L)
   int batch;
   LevelInfo li; HashSetView hs;
+  PrefixMapView pm;                     // slots == null: the last-level mask probes the hash set; else it reads the prefix's bit set
 };
 void launch_select(const SelectArgs& a, cudaStream_t st);
 // launch_select (gated on row_cur == n) followed, in the same launch, by launch_advance of level n

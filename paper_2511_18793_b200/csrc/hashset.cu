@@ -89,6 +89,40 @@ __global__ void __launch_bounds__(256) hs_probe_kernel(HashSetView hs, const uns
   }
 }
 
+// One thread per item: claims (or finds) the slot of the item's prefix, then sets the bit of its last code.
+__global__ void pm_insert_kernel(LevelInfo li, PrefixMapView pm, const int* __restrict__ codes, unsigned long long n, int* status) {
+  const unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  unsigned long long p = 0;
+  for (int l = 0; l + 1 < li.L; ++l) {
+    const int c = codes[i * li.L + l];
+    if (c < 0 || c >= li.T[l]) return;              // hs_insert_kernel has reported it
+    p += (unsigned long long)c * li.mult[l];
+  }
+  const int t = codes[i * li.L + li.L - 1];
+  if (t < 0 || t >= li.T[li.L - 1]) return;
+  unsigned long long s = __umul64hi(hs_mix(p), pm.n_slots);
+  for (int step = 0; step < kMaxProbeBuckets; ++step) {
+    unsigned long long* slot = pm.slots + s * pm.stride;
+    unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(slot);
+    if (cur == 0ull) cur = atomicCAS(slot, 0ull, p + 1);
+    if (cur == 0ull || cur == p + 1) {
+      atomicOr(slot + 1 + (t >> 6), 1ull << (t & 63));
+      return;
+    }
+    if (++s == pm.n_slots) s = 0;
+  }
+  atomicOr(status, kStHashFull);
+}
+
+void launch_pm_build(const LevelInfo& li, PrefixMapView pm, const int* codes, unsigned long long n, int* status, cudaStream_t st) {
+  if (!pm.slots) return;
+  cudaMemsetAsync(pm.slots, 0, (size_t)pm.n_slots * pm.stride * sizeof(unsigned long long), st);
+  if (!n) return;
+  LaunchScope ls(kcHash, st);
+  pm_insert_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(li, pm, codes, n, status);
+}
+
 void launch_hs_clear(HashSetView hs, cudaStream_t st) {
   LaunchScope ls(kcHash, st);
   hs_clear_kernel<<<148 * 8, 512, 0, st>>>(hs.slots, hs.n_buckets * kBucketSlots);

@@ -377,3 +377,29 @@ def test_one_item_catalogue_and_beam_wider_than_it():
         for b in range(w1.batch):
             ref = (O.nezha_draft(head, c1.req(b), w1.beam, V) if mode == 0 else O.ar_beam_search(model, c1.req(b), w1.beam, V))[-1]
             assert_topk_matches(*(out[k][b].cpu().numpy() for k in ("codes", "scores", "count")), ref, w1.beam, tolerance(w1))
+
+
+# ---------------------------------------------------------------------------------------- the last-level mask from the prefix map
+@pytest.mark.parametrize("name", ["tiny", "small_cut", "t512", "t1024", "one_level"])
+def test_final_mask_from_prefix_map_equals_hash_probes(name):
+    """NEZHA_OPT_FINAL_MASK = 1 answers Eq. 5 from the (prefix -> bit set of last codes) table instead of the hash set:
+    every mode must return the same bits as with the hash probes, whatever the codebook size (1, 2, 8 or 16 words of bits)."""
+    w = {"tiny": synth.WORKLOADS["tiny"],
+         "small_cut": synth.scaled(synth.WORKLOADS["small"], n_layers=2, n_items=100_000, batch=4, n_hist=20),
+         "t512": synth.scaled(synth.WORKLOADS["paper"], n_layers=1, batch=3),
+         "t1024": synth.scaled(synth.WORKLOADS["tiny"], L=2, T=(1024, 1024), n_items=30_000, batch=2, beam=16, n_hist=6),
+         "one_level": synth.scaled(synth.WORKLOADS["tiny"], L=1, T=(32,), n_items=20, batch=2, beam=5)}[name]
+    case = Case(w).prefill()
+    base = {m: case.eng.decode(w.beam, mode=m) for m in (0, 1, 2)}
+    case.eng.set_option(3, 1)
+    for m in (0, 1, 2):
+        got = case.eng.decode(w.beam, mode=m)
+        for k in ("codes", "scores", "count"):
+            assert torch.equal(got[k], base[m][k]), (name, m, k)
+    V = case.oracle[2]
+    codes, count = base[1]["codes"].cpu().numpy(), base[1]["count"].cpu().numpy()
+    live = np.arange(w.beam)[None, :] < count[:, None]
+    assert V.contains(codes[live]).all()
+    case.eng.set_option(3, 0)
+    again = case.eng.decode(w.beam, mode=1)
+    assert torch.equal(again["codes"], base[1]["codes"])
