@@ -199,8 +199,8 @@ def probe_bench(args, w, eng, cat_dev, config, dev):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="small")
     ap.add_argument("--mode", type=int, default=1, help="0 draft-only, 1 verified (default), 2 plain autoregressive")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
