@@ -208,8 +208,9 @@ def main():
                     help="mode 1 only: 'natural' = the (random-init) draft head's own drafts; 'perfect' = the true top-k "
                          "tuples injected as round-1 drafts (best case: one round, everything accepted)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (requests per decode call)")
-    ap.add_argument("--final-mask", default="hash", choices=["hash", "prefix"],
-                    help="how the last level's validity mask (Eq. 5) is answered: hash-set probes (default) or the prefix map")
+    ap.add_argument("--final-mask", default="prefix", choices=["hash", "prefix"],
+                    help="how the primary model's last-level validity mask (Eq. 5) is answered: the prefix map (the "
+                         "library's default) or one hash-set probe per candidate code")
     ap.add_argument("--probe-keys", type=int, default=0,
                     help="instead of the decode step, time the stand-alone hash-set probe (Eq. 5) on this many keys, "
                          "half of them catalogue items, and print its own JSON line")
@@ -285,9 +286,8 @@ def main():
     if args.probe_keys > 0:
         probe_bench(args, w, eng, cat_dev, config, dev)
         return
-    if args.final_mask == "prefix":
-        eng.set_option(binding.OPT_FINAL_MASK, 1)
-        config["final_mask"] = "prefix map (one look-up per beam)"
+    eng.set_option(binding.OPT_FINAL_MASK, 1 if args.final_mask == "prefix" else 0)
+    config["final_mask"] = "prefix map (one look-up per beam)" if args.final_mask == "prefix" else "hash-set probes"
     hist_pinned = torch.from_numpy(hist).pin_memory()
     nh_pinned = torch.full((w.batch,), w.n_hist, dtype=torch.int32).pin_memory()
     hist_dev = hist_pinned.to(dev, non_blocking=True)

@@ -169,11 +169,14 @@ nezha_status nezha_decode_with_drafts(nezha_ctx* ctx, int32_t batch, int32_t bea
  *   NEZHA_OPT_DRAFT_INPUTS      0: logits from h_l + s_l (Eq. 2)   1: from h_l alone, no context state (NEZHA-1)
  *                               2: from s_l alone (NEZHA-2)
  *   NEZHA_OPT_DRAFT_FILTER      1: hash-set filter at the last level (Eq. 5)        0: no filter              (NEZHA-4)
- *   NEZHA_OPT_FINAL_MASK        0: the validity mask of the last level (Eq. 5) probes the hash set once per candidate code
- *                               1: it looks the beam's prefix up in a second table, (first L-1 codes) -> bit set of the
- *                                  valid last codes, built by nezha_build_hashset from the same catalogue: one look-up per
- *                                  beam instead of T_L probes, the same answers bit for bit (the set V of Eq. 5 regrouped
- *                                  by prefix; the paper itself only describes the hash set)
+ *   NEZHA_OPT_FINAL_MASK        how the primary model's beam search (modes 1 and 2) answers the validity mask of the last
+ *                               level, where every one of the T_L extensions of every beam is tested (Eq. 5):
+ *                               0: one hash-set probe per candidate code
+ *                               1 (default): it looks the beam's prefix up in a second table, (first L-1 codes) -> bit
+ *                                  set of the valid last codes, built by nezha_build_hashset from the same catalogue: one
+ *                                  look-up per beam instead of T_L probes, the same answers bit for bit (the set V of
+ *                                  Eq. 5 regrouped by prefix; the paper itself only describes the hash set)
+ *                               The draft head's K chosen codes per beam (Algorithm 3) are always probed in the hash set.
  * Errors: NEZHA_ERR_ARG (unknown option or value). */
 #define NEZHA_OPT_DRAFT_TRANSITION 0
 #define NEZHA_OPT_DRAFT_INPUTS 1

@@ -88,7 +88,7 @@ struct nezha_ctx {
   std::map<std::array<uintptr_t, 16>, Segment> segments;
   bool use_graphs;
   int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
-  int opt_mask;             // nezha_set_option: 0 = the last-level mask probes the hash set, 1 = it reads the prefix map
+  int opt_mask;             // nezha_set_option: 0 = the primary model's last-level mask probes the hash set, 1 (default) = it reads the prefix map
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
   int chains_now;           // GemmArgs::chains of the products being queued: 2 inside a decode call, 0 otherwise
@@ -673,7 +673,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
   c->chains_now = 0;
-  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 0;
+  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 1;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;

@@ -194,8 +194,7 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
         bool ok = false; float sv = 0.f; int t = 0;
         if (c < cnt) {
           sv = l_score[(size_t)r * a.K + c]; t = l_tok[(size_t)r * a.K + c];
-          ok = a.pm.slots ? pm_test(pm_find(a.pm, prefix_key), t)
-                          : hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
+          ok = hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
         }
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         __syncwarp();

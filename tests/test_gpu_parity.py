@@ -382,7 +382,7 @@ def test_one_item_catalogue_and_beam_wider_than_it():
 # ---------------------------------------------------------------------------------------- the last-level mask from the prefix map
 @pytest.mark.parametrize("name", ["tiny", "small_cut", "t512", "t1024", "one_level"])
 def test_final_mask_from_prefix_map_equals_hash_probes(name):
-    """NEZHA_OPT_FINAL_MASK = 1 answers Eq. 5 from the (prefix -> bit set of last codes) table instead of the hash set:
+    """NEZHA_OPT_FINAL_MASK = 1 (the default) answers Eq. 5 from the (prefix -> bit set of last codes) table instead of the hash set:
     every mode must return the same bits as with the hash probes, whatever the codebook size (1, 2, 8 or 16 words of bits)."""
     w = {"tiny": synth.WORKLOADS["tiny"],
          "small_cut": synth.scaled(synth.WORKLOADS["small"], n_layers=2, n_items=100_000, batch=4, n_hist=20),
@@ -390,6 +390,7 @@ def test_final_mask_from_prefix_map_equals_hash_probes(name):
          "t1024": synth.scaled(synth.WORKLOADS["tiny"], L=2, T=(1024, 1024), n_items=30_000, batch=2, beam=16, n_hist=6),
          "one_level": synth.scaled(synth.WORKLOADS["tiny"], L=1, T=(32,), n_items=20, batch=2, beam=5)}[name]
     case = Case(w).prefill()
+    case.eng.set_option(3, 0)
     base = {m: case.eng.decode(w.beam, mode=m) for m in (0, 1, 2)}
     case.eng.set_option(3, 1)
     for m in (0, 1, 2):
