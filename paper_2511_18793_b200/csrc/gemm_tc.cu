@@ -26,7 +26,8 @@ template <int BN> struct Cfg {
   static constexpr int kTileBytesB = BN * BK * 2;
   static constexpr int kStageBytes = kTileBytesA + kTileBytesB;
   // as many stages as fit beside the transpose tiles: short-M launches are bound by bytes in flight per CTA
-  static constexpr int kStages = BN == 256 ? 4 : BN == 128 ? 6 : BN == 64 ? 8 : 9;
+  // (even, so that with two MMA issuers a ring slot always belongs to the same issuer: see the kernel)
+  static constexpr int kStages = BN == 256 ? 4 : BN == 128 ? 6 : 8;
   static constexpr int kSmemBytes =
       kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTransposeBytes;
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;       // two accumulators; a power of two >= 32
@@ -47,7 +48,11 @@ __global__ void __launch_bounds__(kThreads + 32 * (ISS - 1)) gemm_tc_kernel(cons
                                                                             GemmArgs a, int* status) {
   using C = Cfg<BN>;
   constexpr int kTmemCols = 2 * BN * ISS < 32 ? 32 : 2 * BN * ISS;   // two accumulators of ISS chains each
-  static_assert(2 * BN * ISS <= 512 && ISS <= C::kStages, "accumulator chains do not fit");
+  static_assert(2 * BN * ISS <= 512, "accumulator chains do not fit");
+  // A slot's `full` barrier must be waited for by ONE thread, phase after phase: a thread that asked for the phase after
+  // the one still in flight would be told "complete" (the parity it names is also that of the phase before).  With the
+  // k-steps dealt round-robin that holds exactly when the ring length is a multiple of the number of issuers.
+  static_assert(C::kStages % ISS == 0, "a ring slot must always be consumed by the same issuer");
   constexpr int kFirstEpiWarp = 1 + ISS;
   constexpr int STAGES = C::kStages;
   extern __shared__ uint8_t smem_raw[];
