@@ -56,3 +56,20 @@ def test_gemm_tc_rejects_uncovered_shapes(ctx):
     assert ei.value.status == 7
     ctx.eng.gemm(A, W, out, epilogue=1, path=0)          # falls back to the CUDA-core kernel
     ctx.eng.sync()
+
+
+@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("N,K", [(512, 2048), (768, 512), (1536, 512), (4096, 512), (896, 4864)])
+def test_gemm_rows_do_not_depend_on_the_number_of_rows(ctx, N, K, path):
+    """A row of the product must come out with the same bits whatever the launch's row count (which decides the tile
+    width, the kernel and the number of waves): the two decode modes run passes of different sizes and must agree exactly."""
+    g = torch.Generator(device="cuda"); g.manual_seed(N + K)
+    A = (torch.randn(5200, K, generator=g, device="cuda") * 0.5).bfloat16()
+    W = (torch.randn(N, K, generator=g, device="cuda") * 0.05).bfloat16()
+    full = torch.empty(5200, N, dtype=torch.float32, device="cuda")
+    ctx.eng.gemm(A, W, full, epilogue=1, path=path)
+    for M in (1, 77, 640, 1920):
+        part = torch.empty(M, N, dtype=torch.float32, device="cuda")
+        ctx.eng.gemm(A[:M].contiguous(), W, part, epilogue=1, path=path)
+        assert torch.equal(part, full[:M]), (N, K, path, M)
+    ctx.eng.sync()
