@@ -404,3 +404,24 @@ def test_final_mask_from_prefix_map_equals_hash_probes(name):
     case.eng.set_option(3, 0)
     again = case.eng.decode(w.beam, mode=1)
     assert torch.equal(again["codes"], base[1]["codes"])
+
+
+def test_nearly_full_tables():
+    """Load factor 0.95: long probe walks in the hash set and in the prefix map; membership stays exact, and both
+    last-level masks still agree with each other and with the oracle's set."""
+    w = synth.scaled(synth.WORKLOADS["small"], n_layers=1, n_items=200_000, batch=3, n_hist=10, load_factor=0.95)
+    case = Case(w).prefill()
+    V = case.oracle[2]
+    assert case.n_unique == w.n_items
+    probe = synth.probe_keys_mix(w, case.catalog, 300_000)
+    keys = case.eng.pack(torch.from_numpy(probe).cuda())
+    assert np.array_equal(case.eng.probe(keys).cpu().numpy().astype(bool), V.contains(probe))
+    outs = {}
+    for mask in (0, 1):
+        case.eng.set_option(3, mask)
+        outs[mask] = case.eng.decode(w.beam, mode=2)
+    for k in ("codes", "scores", "count"):
+        assert torch.equal(outs[0][k], outs[1][k])
+    codes, count = outs[1]["codes"].cpu().numpy(), outs[1]["count"].cpu().numpy()
+    live = np.arange(w.beam)[None, :] < count[:, None]
+    assert V.contains(codes[live]).all()
