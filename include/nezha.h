@@ -249,7 +249,7 @@ nezha_status nezha_gemm(nezha_ctx* ctx, const void* A, const void* W, void* C, i
  *   codes  device int32 [n, L]      found  device uint8 [n]      n <= NEZHA_NOALLOC_MAX_TUPLES
  *
  * Asynchronous on the context's stream.  Errors: NEZHA_ERR_ARG (null pointer; n above the maximum, with a message
- * saying so), NEZHA_ERR_STATE (before nezha_build_hashset), NEZHA_ERR_CUDA.  A code outside [0, T_l) sets
+ * saying so; another GPU than the context's is the current device), NEZHA_ERR_STATE (before nezha_build_hashset), NEZHA_ERR_CUDA.  A code outside [0, T_l) sets
  * NEZHA_ERR_CATALOG, reported by the next synchronising call; that tuple reads as not found.
  *
  * The first call on a device looks up the device address of the built-in buffer (the GPU of the context must be

@@ -207,6 +207,8 @@ class Engine:
         return int(n.value)
 
     def pack(self, codes: torch.Tensor) -> torch.Tensor:
+        assert codes.dtype == torch.int32 and codes.dim() == 2 and codes.shape[1] == self.L
+        assert codes.device == self.arena.device
         codes = codes.contiguous()
         keys = torch.empty(codes.shape[0], dtype=torch.int64, device=codes.device)   # bit pattern of uint64
         self._check(lib.nezha_pack(self._h, _ptr(codes), codes.shape[0], _ptr(keys)))
@@ -221,6 +223,8 @@ class Engine:
         """nezha_contains_noalloc: validity of code tuples with no allocation anywhere; `codes` (int32 [n, L],
         contiguous) and `found` (uint8 [n]) are the caller's, and this method creates no tensor either."""
         assert codes.dtype == torch.int32 and found.dtype == torch.uint8 and found.shape[0] == codes.shape[0]
+        assert codes.dim() == 2 and codes.shape[1] == self.L and codes.is_contiguous() and found.is_contiguous()
+        assert codes.device == self.arena.device and found.device == self.arena.device
         self._check(lib.nezha_contains_noalloc(self._h, _ptr(codes), codes.shape[0], _ptr(found)))
         return found
 

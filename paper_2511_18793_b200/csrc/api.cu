@@ -93,6 +93,7 @@ struct nezha_ctx {
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
   int chains_now;           // GemmArgs::chains of the products being queued: 2 inside a decode call, 0 otherwise
   int rounds_seen[3];       // rounds the last decode call of each mode needed: that many are launched without waiting
+  int device;               // the GPU that was current at nezha_create
   int state;                // 0 created, 1 hash set built, 2 prefilled
   int batch;                // prefilled batch
   std::string err;
@@ -667,6 +668,8 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   nezha_ctx* c = new nezha_ctx();
   c->cfg = *cfg; c->n_items = n_items; c->load_factor = load_factor; c->catalog = catalog_codes;
   c->st = (cudaStream_t)cuda_stream; c->arena = nullptr; c->state = 0; c->batch = 0;
+  c->device = 0;
+  if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return NEZHA_ERR_CUDA; }
   // the legacy default stream cannot be captured; NEZHA_NO_GRAPHS=1 keeps every launch eager
   c->use_graphs = cuda_stream != nullptr && !getenv("NEZHA_NO_GRAPHS");
   c->m_expected = 0;
@@ -1014,6 +1017,10 @@ nezha_status nezha_contains_noalloc(nezha_ctx* c, const int32_t* codes, size_t n
                                   "key buffer); split the request or use nezha_pack + nezha_probe");
   if (c->state < 1) return fail(c, NEZHA_ERR_STATE, "nezha_contains_noalloc before nezha_build_hashset");
   if (!n) return NEZHA_OK;
+  int dev = -1;
+  NZ_CUDA(c, cudaGetDevice(&dev));
+  if (dev != c->device)          // the built-in buffer is per device: the address looked up must be the context's GPU's
+    return fail(c, NEZHA_ERR_ARG, "nezha_contains_noalloc: the context's GPU must be the current device");
   unsigned long long* keys = nullptr;
   NZ_CUDA(c, noalloc_keys_address(&keys));
   launch_hs_pack(c->es.li, codes, n, keys, c->es.status, c->st);

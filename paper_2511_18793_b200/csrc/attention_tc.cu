@@ -352,23 +352,23 @@ __global__ void __launch_bounds__(AttnCfg<HD, RW, KW>::kThreads) attn_tc_kernel(
 template <int HD, int RW, int KW>
 void launch(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cudaStream_t st) {
   using C = AttnCfg<HD, RW, KW>;
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce configured;
+  configured.run([] {
     cudaFuncSetAttribute(attn_tc_kernel<HD, RW, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    configured = true;
-  }
+  });
   const int G = a.Hq / a.Hkv;
   dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + 16 * RW - 1) / (16 * RW));
   // the layer's draft-token caches as [positions of all requests, kv heads * hd] (a prefill has none: any valid map)
-  const CUtensorMap* tkx = tk;
-  const CUtensorMap* tvx = tv;
+  CUtensorMap tkx = *tk, tvx = *tv;
   if (a.n_ext_max > 0) {
     const long long rows = a.ext_rows_total, cols = (long long)a.Hkv * HD;
-    tkx = tma_map_bf16(a.k_ext, rows, cols, cols, kPos);
-    tvx = tma_map_bf16(a.v_ext, rows, cols, cols, kPos);
-    if (!tkx || !tvx) { static const int flag = kStInternal; cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st); return; }
+    if (!tma_map_bf16(a.k_ext, rows, cols, cols, kPos, &tkx) || !tma_map_bf16(a.v_ext, rows, cols, cols, kPos, &tvx)) {
+      static const int flag = kStInternal;
+      cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st);
+      return;
+    }
   }
-  launch_pdl(attn_tc_kernel<HD, RW, KW>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *tk, *tv, *tkx, *tvx, a, a.status);
+  launch_pdl(attn_tc_kernel<HD, RW, KW>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *tk, *tv, tkx, tvx, a, a.status);
 }
 
 }  // namespace
@@ -386,9 +386,12 @@ bool attention_tc_supported(const AttnArgs& a) {
 void launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   // the whole context cache of the layer as one [requests * kv_heads * positions, hd] matrix
   const long long rows = (long long)a.ctx_rows_total;
-  const CUtensorMap* tk = tma_map_bf16(a.k_ctx, rows, a.hd, a.hd, kPos);
-  const CUtensorMap* tv = tma_map_bf16(a.v_ctx, rows, a.hd, a.hd, kPos);
-  if (!tk || !tv) { launch_attention_simt(a, true, st); return; }
+  CUtensorMap tk_map, tv_map;
+  if (!tma_map_bf16(a.k_ctx, rows, a.hd, a.hd, kPos, &tk_map) || !tma_map_bf16(a.v_ctx, rows, a.hd, a.hd, kPos, &tv_map)) {
+    launch_attention_simt(a, true, st);
+    return;
+  }
+  const CUtensorMap *tk = &tk_map, *tv = &tv_map;
   LaunchScope ls(kcAttention, st);
   // Query rows per (request, KV head): the bound the grid must cover, and what the caller expects (shapes the tile only).
   const int G = a.Hq / a.Hkv;

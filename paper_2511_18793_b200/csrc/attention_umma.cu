@@ -354,23 +354,23 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
 template <int HD>
 void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cudaStream_t st) {
   using C = UmmaCfg<HD>;
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce configured;
+  configured.run([] {
     cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    configured = true;
-  }
+  });
   const int G = a.Hq / a.Hkv;
   dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + kRowsU - 1) / kRowsU);
   // the layer's draft-token caches as [positions of all requests, kv heads * hd] (a prefill has none: any valid map)
-  const CUtensorMap* tkx = tk;
-  const CUtensorMap* tvx = tv;
+  CUtensorMap tkx = *tk, tvx = *tv;
   if (a.n_ext_max > 0) {
     const long long rows = a.ext_rows_total, cols = (long long)a.Hkv * HD;
-    tkx = tma_map_bf16(a.k_ext, rows, cols, cols, kPosU);
-    tvx = tma_map_bf16(a.v_ext, rows, cols, cols, kPosU);
-    if (!tkx || !tvx) { static const int flag = kStInternal; cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st); return; }
+    if (!tma_map_bf16(a.k_ext, rows, cols, cols, kPosU, &tkx) || !tma_map_bf16(a.v_ext, rows, cols, cols, kPosU, &tvx)) {
+      static const int flag = kStInternal;
+      cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st);
+      return;
+    }
   }
-  launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, *tkx, *tvx, a, a.status);
+  launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, tkx, tvx, a, a.status);
 }
 
 }  // namespace

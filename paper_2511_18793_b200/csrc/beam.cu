@@ -309,8 +309,14 @@ size_t select_smem_bytes(int in_stride, int K) {
          (size_t)K * (sizeof(float) + 2 * sizeof(int)) + sizeof(int);
 }
 
+// The attribute belongs to the device, and several contexts may share one: it is only ever raised.
 cudaError_t select_configure(int max_beam) {
-  const int bytes = (int)select_smem_bytes(max_beam, max_beam);
+  static int configured_bytes[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  int bytes = (int)select_smem_bytes(max_beam, max_beam);
+  if (bytes <= configured_bytes[dev]) return cudaSuccess;
+  configured_bytes[dev] = bytes;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(select_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;
   if ((e = cudaFuncSetAttribute(select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return e;

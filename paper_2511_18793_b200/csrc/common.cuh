@@ -94,8 +94,10 @@ __device__ __forceinline__ unsigned long long hs_bucket(unsigned long long key, 
   return __umul64hi(hs_mix(key), n_buckets);
 }
 
-// One thread walks the probe sequence alone, a whole bucket (one sector) per step.
+// One thread walks the probe sequence alone, a whole bucket (one sector) per step.  The empty-slot sentinel is not a
+// packed key (Eq. 4 maps onto [0, prod T) and prod T < 2^64 - 1): it is never a member, although it equals every free slot.
 __device__ __forceinline__ bool hs_contains_thread(const HashSetView& hs, unsigned long long key) {
+  if (key == kEmptyKey) return false;
   unsigned long long b = hs_bucket(key, hs.n_buckets);
   for (int step = 0; step < kMaxProbeBuckets; ++step) {
     const ulonglong2* p = reinterpret_cast<const ulonglong2*>(hs.slots + b * kBucketSlots);
@@ -125,6 +127,7 @@ __device__ __forceinline__ void hs_contains_many(const HashSetView& hs, const un
     found[j] = false;
     if (!want[j]) continue;
     const unsigned long long k = keys[j];
+    if (k == kEmptyKey) continue;                      // the sentinel matches every free slot and is no key
     if (lo[j].x == k || lo[j].y == k || hi[j].x == k || hi[j].y == k) found[j] = true;
     else if (lo[j].x == kEmptyKey || lo[j].y == kEmptyKey || hi[j].x == kEmptyKey || hi[j].y == kEmptyKey) found[j] = false;
     else found[j] = hs_contains_thread(hs, k);        // home bucket full: rare at the load factors in use

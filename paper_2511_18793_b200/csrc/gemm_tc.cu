@@ -185,33 +185,35 @@ __global__ void __launch_bounds__(kThreads + 32 * (ISS - 1)) gemm_tc_kernel(cons
 // ---------------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------------
-int sm_count() {
-  static int n = [] {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
-      v = 148;
-    return v;
-  }();
-  return n;
+int sm_count() {                                  // of the current device
+  static std::mutex mu;
+  static int n[kMaxDevices] = {};
+  std::lock_guard<std::mutex> g(mu);
+  const int dev = current_device();
+  if (n[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    cudaGetLastError();
+    n[dev] = v;
+  }
+  return n[dev];
 }
 
 template <int BN, int EPI, int ISS>
 void launch(const GemmArgs& a, cudaStream_t st) {
-  const CUtensorMap* ta = tma_map_bf16(a.A, a.M, a.K, a.lda, BM);
-  const CUtensorMap* tb = tma_map_bf16(a.W, a.N, a.K, a.ldw, BN);
-  if (!ta || !tb) {                            // cannot happen for shapes gemm_tc_supported accepted; report, do not guess
-    static const int flag = kStInternal;
+  CUtensorMap ta, tb;
+  if (!tma_map_bf16(a.A, a.M, a.K, a.lda, BM, &ta) || !tma_map_bf16(a.W, a.N, a.K, a.ldw, BN, &tb)) {
+    static const int flag = kStInternal;       // cannot happen for shapes gemm_tc_supported accepted; report, do not guess
     cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st);
     return;
   }
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce configured;
+  configured.run([] {
     cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI, ISS>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
-    configured = true;
-  }
+  });
   const long long tiles = (long long)((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  launch_pdl(gemm_tc_kernel<BN, EPI, ISS>, dim3(grid), dim3(kThreads + 32 * (ISS - 1)), Cfg<BN>::kSmemBytes, st, *ta, *tb, a, a.status);
+  launch_pdl(gemm_tc_kernel<BN, EPI, ISS>, dim3(grid), dim3(kThreads + 32 * (ISS - 1)), Cfg<BN>::kSmemBytes, st, ta, tb, a, a.status);
 }
 
 template <int BN, int ISS>
@@ -275,7 +277,9 @@ void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
   // looks at N and K only, never at M or at the tiling, so such a product keeps its summation order (and its bits)
   // whatever the number of rows of a launch -- what lets two decode modes whose passes differ in size agree exactly.
   static const bool one_issuer = getenv("NEZHA_ONE_MMA_ISSUER") != nullptr;
-  if (a.chains == 2 && a.N <= 1024 && a.K >= 2 * BK && !one_issuer) {
+  // (An even number of k-steps: then every tile starts on ring slot parity 0 for issuer 0 and a slot keeps its issuer
+  // from tile to tile, which is what the kernel's one-waiter-per-slot rule needs.)
+  if (a.chains == 2 && a.N <= 1024 && a.K >= 2 * BK && (a.K / BK) % 2 == 0 && !one_issuer) {
     const long long tiles_m = (m_plan + BM - 1) / BM;
     static const int widths[3] = {128, 64, 32}, wave_cost[3] = {400, 300, 250};
     long long best = -1; int plan = 32;

@@ -189,18 +189,16 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_pair_kernel(const __grid_con
 
 template <int EPI>
 void launch_pair(const GemmArgs& a, int n_sm, cudaStream_t st) {
-  const CUtensorMap* ta = tma_map_bf16(a.A, a.M, a.K, a.lda, BM);
-  const CUtensorMap* tb = tma_map_bf16(a.W, a.N, a.K, a.ldw, kBN2 / 2);
-  if (!ta || !tb) {
+  CUtensorMap ta, tb;
+  if (!tma_map_bf16(a.A, a.M, a.K, a.lda, BM, &ta) || !tma_map_bf16(a.W, a.N, a.K, a.ldw, kBN2 / 2, &tb)) {
     static const int flag = kStInternal;
     cudaMemcpyAsync(a.status, &flag, sizeof(int), cudaMemcpyHostToDevice, st);
     return;
   }
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce configured;
+  configured.run([] {
     cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-    configured = true;
-  }
+  });
   const long long tiles = (long long)((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + kBN2 - 1) / kBN2);
   const int pairs = (int)(tiles < n_sm / 2 ? tiles : n_sm / 2);
   cudaLaunchConfig_t cfg{};
@@ -209,7 +207,7 @@ void launch_pair(const GemmArgs& a, int n_sm, cudaStream_t st) {
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<EPI>, *ta, *tb, a, a.status);
+  cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<EPI>, ta, tb, a, a.status);
 }
 
 }  // namespace

@@ -5,6 +5,7 @@
 #include <cuda.h>
 
 #include <map>
+#include <mutex>
 #include <tuple>
 
 #include "common.cuh"
@@ -89,14 +90,40 @@ inline EncodeTiledFn tma_encode_fn() {
   return fn;
 }
 
+// Index of the current device, clamped to the tables below.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+  int d = 0;
+  if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) d = 0;
+  cudaGetLastError();
+  return d;
+}
+
+// One-time set-up per device (a function attribute belongs to the device's context, not to the process): run(f) calls f
+// the first time it is reached with a given device current, under a lock, so that no other host thread launches before
+// the set-up has been made.
+struct PerDeviceOnce {
+  std::mutex mu;
+  bool done[kMaxDevices] = {};
+  template <typename F> void run(F&& f) {
+    std::lock_guard<std::mutex> g(mu);
+    const int d = current_device();
+    if (!done[d]) { f(); done[d] = true; }
+  }
+};
+
 // 2-D bf16 row-major [rows, cols] with row pitch ld (elements); box = 64 columns x box_rows rows, 128-byte swizzle.
-inline const CUtensorMap* tma_map_bf16(const void* ptr, long long rows, long long cols, long long ld, int box_rows) {
+// The map is returned by value (it is a kernel parameter anyway); encoded maps are kept in a process-wide table behind a
+// lock, keyed by everything that goes into them, and the table is emptied when it has grown past a few thousand entries.
+inline bool tma_map_bf16(const void* ptr, long long rows, long long cols, long long ld, int box_rows, CUtensorMap* out) {
   using Key = std::tuple<const void*, long long, long long, long long, int>;
   static std::map<Key, CUtensorMap> cache;
-  Key key{ptr, rows, cols, ld, box_rows};
+  static std::mutex mu;
+  if (!tma_encode_fn()) return false;
+  const Key key{ptr, rows, cols, ld, box_rows};
+  std::lock_guard<std::mutex> g(mu);
   auto it = cache.find(key);
-  if (it != cache.end()) return &it->second;
-  if (!tma_encode_fn()) return nullptr;
+  if (it != cache.end()) { *out = it->second; return true; }
   CUtensorMap tm;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
@@ -105,9 +132,11 @@ inline const CUtensorMap* tma_map_bf16(const void* ptr, long long rows, long lon
   if (tma_encode_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return nullptr;
+    return false;
   if (cache.size() > 8192) cache.clear();
-  return &cache.emplace(key, tm).first->second;
+  cache.emplace(key, tm);
+  *out = tm;
+  return true;
 }
 
 }  // namespace nz

@@ -73,3 +73,23 @@ def test_gemm_rows_do_not_depend_on_the_number_of_rows(ctx, N, K, path):
         ctx.eng.gemm(A[:M].contiguous(), W, part, epilogue=1, path=path)
         assert torch.equal(part, full[:M]), (N, K, path, M)
     ctx.eng.sync()
+
+
+@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("N,K", [(512, 192), (896, 320), (1024, 576), (256, 960), (64, 192)])
+def test_gemm_odd_number_of_k_steps_many_tiles_per_cta(ctx, N, K, path):
+    """K / 64 odd and far more output tiles than SMs: every CTA walks several tiles, so the operand ring's slots change
+    hands between tiles unless the kernel keeps one waiter per slot.  Against the fp64 product, and twice (bit-equal)."""
+    M = 128 * 148 * 3 + 77
+    g = torch.Generator(device="cuda"); g.manual_seed(N * 5 + K)
+    A = (torch.randn(M, K, generator=g, device="cuda") * 0.5).bfloat16()
+    W = (torch.randn(N, K, generator=g, device="cuda") * 0.05).bfloat16()
+    ref = _ref(A, W)
+    scale = np.abs(ref).max()
+    out = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    ctx.eng.gemm(A, W, out, epilogue=1, path=path)
+    assert np.abs(out.cpu().numpy() - ref).max() < 2e-5 * scale * np.sqrt(K / 64) + 1e-6
+    again = torch.empty_like(out)
+    ctx.eng.gemm(A, W, again, epilogue=1, path=path)
+    assert torch.equal(out, again)
+    ctx.eng.sync()

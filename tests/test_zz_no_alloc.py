@@ -59,3 +59,36 @@ def test_contains_noalloc_rejects_oversized_and_early_calls():
     eng.sync()
     exp = bool(O.ValidSet(catalog, w.T).contains(np.zeros((1, w.L), dtype=np.int64))[0])
     assert bool(got.all().item()) == exp and bool(got.any().item()) == exp
+
+
+def test_out_of_range_codes_are_never_found():
+    """A tuple with a code outside [0, T_l) is no semantic ID: both paths must answer 0 for it (its packed key is the
+    table's empty-slot value, which equals every free slot) and the next synchronising call reports NEZHA_ERR_CATALOG.
+    The same holds for a raw key of all ones handed to nezha_probe."""
+    from paper_2511_18793_b200 import binding
+    w = synth.scaled(synth.WORKLOADS["small"], n_items=50_000, n_layers=1, batch=2, n_hist=4)
+    catalog = synth.make_catalog(w)
+    eng = binding.Engine(binding.make_config(w), synth.make_weights(w, device="cuda"),
+                         torch.from_numpy(catalog).cuda(), w.load_factor)
+    assert eng.build_hashset() == w.n_items
+    good = catalog[:64].copy()
+    bad = np.repeat(catalog[:1], 64, axis=0)
+    for i in range(64):
+        bad[i, i % w.L] = -1 if i % 2 else w.T[i % w.L]
+    codes_np = np.concatenate([good, bad]).astype(np.int32)
+    codes = torch.from_numpy(codes_np).cuda()
+    want = np.concatenate([np.ones(64, bool), np.zeros(64, bool)])
+    for path in ("noalloc", "pack_probe"):
+        found = torch.full((128,), 7, dtype=torch.uint8, device="cuda")
+        if path == "noalloc":
+            eng.contains_noalloc(codes, found)
+        else:
+            eng.probe(eng.pack(codes), out=found)
+        with pytest.raises(binding.NezhaError) as e:
+            eng.sync()
+        assert e.value.status == 6                                          # NEZHA_ERR_CATALOG
+        assert np.array_equal(found.cpu().numpy().astype(bool), want), path
+        eng.sync()                                                          # the error was reported once and cleared
+    ones = torch.full((33,), -1, dtype=torch.int64, device="cuda")          # bit pattern of 2^64 - 1
+    assert not eng.probe(ones).any().item()
+    eng.sync()
