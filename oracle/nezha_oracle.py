@@ -25,14 +25,19 @@ Readings where the paper is silent (the same readings bind the CUDA path):
     as a sum of log-probabilities, stored in fp32; order: higher score first, ties to the smaller
     (parent rank, token).
   * plain autoregressive decoding sees no placeholders: the level-j code sits at position P + j - 1.
+  * Algorithm 2's "verify in parallel" takes the draft head's whole level-wise beam tree (the beam sets of every level
+    of Algorithm 3, one node per distinct prefix), not only the prefixes of its K final tuples.
 
 Pinned by tests/test_oracle_*.py:  Eq. 4 by the paper's worked example and bijectivity; ValidSet by python
 sets; PrimaryModel by an independent library implementation of the same architecture, closed forms and
 cached-vs-recomputed equality; nezha_draft and ar_beam_search by brute-force enumeration, independently
 recomputed joint log-probabilities and closed forms under zero heads; speculative_decode by equality with
-ar_beam_search for any drafts.  The per-tuple accepted lengths of speculative_decode are defined by this
-file's reading of Algorithm 2 and have no external pin beyond the two extreme cases (all drafts right, all
-drafts wrong): parity unpinned for accepted lengths in general.
+ar_beam_search for any drafts, and its walk (rounds, rejection levels, accepted lengths, tokens in the pass) by
+hand-worked cases on heads of all zeros, where the tie rule fixes every beam set in closed form.  How Algorithm 2's
+parallel verification is combined with NEZHA's head (which nodes the pass holds) is this file's reading: the paper
+never runs the two together.  DraftHead.logits / .transition follow readings of Section 4.1's one-line description
+(sum then one matmul; one shared Elman cell): pinned by hand-computed numbers and the ablation identities of
+Section 4.3, with no external implementation to compare against.
 """
 from __future__ import annotations
 
@@ -416,24 +421,43 @@ def ar_beam_search(model: PrimaryModel, req: Request, K: int, valid: Optional[Va
 class SpecStats:
     rounds: int = 0
     primary_tokens: int = 0                              # code tokens M_p processed, over all rounds
-    accepted_len: List[List[int]] = field(default_factory=list)   # per round, per draft tuple
+    accepted_len: List[List[int]] = field(default_factory=list)   # per round, per drafted tuple (the tree's level-L nodes)
     reject_level: List[int] = field(default_factory=list)         # per round: level m the round ended at
+    tree_nodes: List[List[int]] = field(default_factory=list)     # per round: nodes of levels m+1..L-1 that were in the pass
+
+
+def tree_from_tuples(tuples: Sequence[Tuple[int, ...]], L: int) -> List[List[Tuple[int, ...]]]:
+    """The prefix tree of a list of drafted L-tuples: level j (1-based) holds their distinct j-prefixes, in order of
+    first appearance.  Tuples that share a prefix share its node (one M_p token, not one per tuple)."""
+    tree: List[List[Tuple[int, ...]]] = []
+    for j in range(1, L + 1):
+        seen: List[Tuple[int, ...]] = []
+        for t in tuples:
+            p = tuple(int(c) for c in t[:j])
+            if p not in seen:
+                seen.append(p)
+        tree.append(seen)
+    return tree
 
 
 def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: int, valid: Optional[ValidSet],
                        drafts_round1: Optional[List[Tuple[int, ...]]] = None,
+                       draft_tree_round1: Optional[List[List[Tuple[int, ...]]]] = None,
                        use_drafts: bool = True) -> Tuple[List[List[Beam]], SpecStats]:
     """Algorithm 2 with the readings listed in the module header.
 
     B_1 comes from the prefill hidden state h_0.  Each round, with m levels settled (true beams B_m):
-      * drafts D: round 1 = NEZHA's drafts from the empty beam (all L codes; `drafts_round1` overrides them);
-        later rounds = drafting continued from B_m.  A draft is *alive* if its first m codes are a beam of B_m.
-      * the M_p pass processes the level-m code of every beam of B_m and the codes of levels m+1..L-1 of every
-        alive draft (each token attends to the context and to its own tuple's earlier codes).
-      * selection walks forward: B_{j+1} from the logits at the beams of B_j, while every beam of B_j is the
-        j-prefix of some alive draft (so its logits are in the pass); the first level where that fails is the
-        rejection level of Algorithm 2; the round ends there and m <- that level.
-      * accepted length of draft k = the largest i <= (level reached) with D[k][:i] in B_i.
+      * draft tree: what the draft model proposes is the whole level-wise beam tree of Algorithm 3, one node per distinct
+        drafted prefix: round 1 = the beam sets D_1..D_L of NEZHA's search from the empty beam; later rounds = the sets
+        D_{m+1}..D_L of the search continued from B_m.  `draft_tree_round1` overrides round 1's tree (level j = a list
+        of j-tuples); `drafts_round1` gives final tuples only, whose prefixes form the tree.
+      * a node of level m is *alive* if it is a beam of B_m; a node of a higher level if its parent is an alive node.
+      * the M_p pass ("verify in parallel", Section 2.2) processes the level-m code of every beam of B_m and the last code
+        of every alive node of levels m+1..L-1 (each token attends to the context and to its own prefix's earlier codes).
+      * selection walks forward: B_{j+1} from the logits at the beams of B_j, while every beam of B_j is an alive node
+        (so its logits are in the pass); the first level where that fails is the rejection level of Algorithm 2; the
+        round ends there and m <- that level.
+      * accepted length of a drafted tuple = the largest i <= (level reached) whose i-prefix is a beam of B_i.
     Every B_j is computed from M_p's logits only, so the result equals ar_beam_search whatever the drafts.
     use_drafts=False gives L-1 rounds of plain autoregressive steps.
     """
@@ -447,40 +471,44 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
     m = 1
     while m < L:
         stats.rounds += 1
-        # ---- draft (Algorithm 2, drafting step)
+        # ---- draft (Algorithm 2, drafting step): tree[j - 1] = drafted nodes of level j
+        tree: List[List[Tuple[int, ...]]] = [[] for _ in range(L)]
         if not use_drafts:
-            D: List[Tuple[int, ...]] = []
+            pass
+        elif stats.rounds == 1 and draft_tree_round1 is not None:
+            tree = [[tuple(int(c) for c in t) for t in lv] for lv in draft_tree_round1]
+        elif stats.rounds == 1 and drafts_round1 is not None:
+            tree = tree_from_tuples(drafts_round1, L)
         elif stats.rounds == 1:
-            if drafts_round1 is not None:
-                D = [tuple(int(c) for c in t) for t in drafts_round1]
-            else:
-                D = [b.codes for b in nezha_draft(head, req, K, valid)[-1]]
+            tree = [[b.codes for b in lv] for lv in nezha_draft(head, req, K, valid)]
         else:
-            lv = nezha_draft(head, req, K, valid, start=B)
-            D = [b.codes for b in lv[-1]] if lv else []
+            lv = nezha_draft(head, req, K, valid, start=B)                  # levels m+1 .. L
+            tree[m - 1] = [b.codes for b in B]
+            for i, beams in enumerate(lv):
+                tree[m + i] = [b.codes for b in beams]
         beam_set = {b.codes for b in B}
-        alive = [k for k, t in enumerate(D) if t[:m] in beam_set]
+        alive = {m: [t for t in tree[m - 1] if t in beam_set]}
+        for j in range(m + 1, L):
+            parents = set(alive[j - 1])
+            alive[j] = [t for t in tree[j - 1] if t[:-1] in parents]
         # ---- the parallel verification pass: count its tokens; logits are looked up per prefix below
-        stats.primary_tokens += len(B) + len(alive) * (L - 1 - m)
-        in_pass = {b.codes for b in B}
-        for k in alive:
-            for j in range(m + 1, L):
-                in_pass.add(D[k][:j])
+        nodes = [len(alive[j]) for j in range(m + 1, L)]
+        stats.tree_nodes.append(nodes)
+        stats.primary_tokens += len(B) + sum(nodes)
         # ---- progressive selection / rejection (Algorithm 2, rejection and update steps)
         j = m
         while True:
-            assert all(b.codes in in_pass for b in B)
             logits = model.next_level_logits_many(req, [b.codes for b in B])
             B = expand_level(B, logits, K, s.T[j], valid if j + 1 == L else None)
             j += 1
             true_sets.append(B)                          # true_sets[i - 1] is B_i
             if j == L:
                 break
-            alive_prefixes = {D[k][:j] for k in alive}
-            if not all(b.codes in alive_prefixes for b in B):
+            in_pass = set(alive[j])
+            if not all(b.codes in in_pass for b in B):
                 break
         acc = []
-        for k, t in enumerate(D):
+        for t in tree[L - 1]:
             a = 0
             for i in range(1, j + 1):
                 if t[:i] in {b.codes for b in true_sets[i - 1]}:

@@ -352,12 +352,17 @@ def test_speculative_decode_equals_autoregressive_beam_search():
             assert all(t in valid for t in codes_of(sp[-1]))
         _, st = O.speculative_decode(model, head, req, w.beam, V, use_drafts=False)
         assert st.rounds == w.L - 1 and st.primary_tokens == sum(len(x) for x in ar[:-1])
-        # perfect drafts: one round, every tuple accepted in full
+        # perfect draft tree (the true beam sets themselves): one round, every tuple accepted in full, and the pass costs
+        # exactly the tokens plain autoregressive decoding needs over its L-1 calls
+        sp, st = O.speculative_decode(model, head, req, w.beam, V, draft_tree_round1=[codes_of(x) for x in ar])
+        assert codes_of(sp[-1]) == codes_of(ar[-1])
+        assert st.rounds == 1 and st.accepted_len == [[w.L] * len(ar[-1])] and st.reject_level == [w.L]
+        assert st.primary_tokens == sum(len(x) for x in ar[:-1])
+        # the true final tuples alone: every prefix of a tuple of B_L is a beam of its level, so each tuple is accepted up
+        # to the level the round reached, whatever that level is
         sp, st = O.speculative_decode(model, head, req, w.beam, V, drafts_round1=codes_of(ar[-1]))
         assert codes_of(sp[-1]) == codes_of(ar[-1])
-        if {t[:2] for t in codes_of(ar[-1])} >= set(codes_of(ar[1])) and \
-           {t[:1] for t in codes_of(ar[-1])} >= set(codes_of(ar[0])):
-            assert st.rounds == 1 and st.accepted_len == [[w.L] * len(ar[-1])]
+        assert st.accepted_len[0] == [st.reject_level[0]] * len(ar[-1])
         # drafts whose first code is not in B_1: nothing accepted, L-1 rounds
         b1 = {t[0] for t in codes_of(ar[0])}
         bad = [c for c in range(w.T[0]) if c not in b1][: w.beam]
@@ -381,6 +386,145 @@ def test_speculative_round_two_drafts_extend_true_beams():
         st = O.teacher_forced_state(head, req, bm.codes[:2])
         lp = float(O.log_softmax(head.logits(2, req.h[3], st))[bm.codes[2]])
         assert abs(float(bm.score) - (float(parent.score) + lp)) < 1e-5
+
+
+def _zero_head_case(catalog):
+    """MICRO with every logit head zero: all probabilities are uniform, so the tie rule (smaller parent rank, then
+    smaller code) fixes every beam set by hand.  With K = 2: B_1 = {(0), (1)}, B_2 = {(0,0), (0,1)}, B_3 = the first two
+    valid tuples among (0,0,c), (0,1,c) in that order; the draft head's sets are the same before its filter."""
+    w = MICRO
+    W = synth.weights_to_numpy(synth.make_weights(w, std=0.5))
+    W = dict(W)
+    W["draft_logit"] = [np.zeros_like(a) for a in W["draft_logit"]]
+    W["lm_head"] = np.zeros_like(W["lm_head"])
+    model, head, V = oracle_bundle(w, W, np.asarray(catalog, dtype=np.int32))
+    req = model.prefill(synth.make_histories(w, None)[0])
+    return model, head, V, req
+
+
+def test_speculative_walk_hand_worked_cases():
+    """Accept-until-first-rejection (Section 2.2), worked by hand on the zero-head case.  Expected values below are
+    derived in the comments from the rule, not from the oracle."""
+    cat = [(0, 0, 2), (0, 1, 1), (0, 1, 3), (1, 0, 0), (3, 3, 3)]
+    model, head, V, req = _zero_head_case(cat)
+    K = 2
+    ar = O.ar_beam_search(model, req, K, V)
+    assert [codes_of(x) for x in ar] == [[(0,), (1,)], [(0, 0), (0, 1)], [(0, 0, 2), (0, 1, 1)]]
+    # (a) partly right.  Tree of the tuples: level 1 {(0),(1)}, level 2 {(0,0),(1,0)}.  Round 1 (m = 1): the pass holds
+    #     B_1's 2 tokens + the 2 level-2 nodes (both have an alive parent) = 4.  B_2 = {(0,0),(0,1)}; (0,1) is no node:
+    #     rejection at level 2.  (0,0,2): prefixes (0) in B_1, (0,0) in B_2 -> 2.  (1,0,0): (1) in B_1, (1,0) not in B_2 -> 1.
+    #     Round 2 (m = 2 = L-1): only B_2's 2 tokens; the zero draft head proposes codes 0,1 of each beam, of which only
+    #     (0,1,1) is valid -> one drafted tuple, which is in B_3 -> 3.
+    sp, st = O.speculative_decode(model, head, req, K, V, drafts_round1=[(0, 0, 2), (1, 0, 0)])
+    assert codes_of(sp[-1]) == [(0, 0, 2), (0, 1, 1)]
+    assert (st.rounds, st.reject_level, st.accepted_len, st.primary_tokens) == (2, [2, 3], [[2, 1], [3]], 6)
+    assert st.tree_nodes == [[2], []]
+    # (b) first codes wrong: no node of level 1 is a beam, nothing beyond B_1 is in the pass (2 tokens), rejection at
+    #     level 2, accepted lengths 0; round 2 as above.  Total = the 4 tokens of plain autoregressive decoding.
+    sp, st = O.speculative_decode(model, head, req, K, V, drafts_round1=[(2, 0, 0), (3, 3, 3)])
+    assert (st.rounds, st.reject_level, st.accepted_len, st.primary_tokens) == (2, [2, 3], [[0, 0], [3]], 4)
+    # (c) the true tuples: level 1 of their tree is {(0)} only, but B_1's own tokens are always in the pass; level 2 is
+    #     {(0,0),(0,1)} = B_2 -> the walk reaches level 3 in one round; 2 + 2 tokens.
+    sp, st = O.speculative_decode(model, head, req, K, V, drafts_round1=[(0, 0, 2), (0, 1, 1)])
+    assert (st.rounds, st.reject_level, st.accepted_len, st.primary_tokens) == (1, [3], [[3, 3]], 4)
+    # (d) shared prefixes are one node: four tuples under (0,0) and (0,1) still cost 2 level-2 tokens; (0,0,0) is not
+    #     in B_3 but its first two codes are beams -> 2.
+    sp, st = O.speculative_decode(model, head, req, K, V, drafts_round1=[(0, 0, 0), (0, 0, 2), (0, 1, 1), (0, 1, 3)])
+    assert (st.rounds, st.primary_tokens, st.tree_nodes) == (1, 4, [[2]])
+    assert st.accepted_len == [[2, 3, 3, 2]]
+    # (e) a level-2 node whose parent is no beam is dead: (2,0) costs no token; (0,0) alone does not cover B_2
+    sp, st = O.speculative_decode(model, head, req, K, V, draft_tree_round1=[[(0,), (2,)], [(0, 0), (2, 0)], [(0, 0, 2), (2, 0, 0)]])
+    assert (st.rounds, st.reject_level, st.tree_nodes[0], st.accepted_len[0]) == (2, [2, 3], [1], [2, 0])
+    # (f) the natural path (zero draft head): its level sets are D_1 = {(0),(1)}, D_2 = {(0,0),(0,1)} = the true ones,
+    #     D_3 = valid among (0,0,0),(0,0,1),(0,1,0),(0,1,1) = {(0,1,1)} -> one round, that tuple accepted in full
+    sp, st = O.speculative_decode(model, head, req, K, V)
+    assert (st.rounds, st.reject_level, st.accepted_len, st.primary_tokens) == (1, [3], [[3]], 4)
+    assert codes_of(sp[-1]) == [(0, 0, 2), (0, 1, 1)]
+
+
+def test_tree_from_tuples_shares_prefixes():
+    tree = O.tree_from_tuples([(1, 2, 3), (1, 2, 0), (1, 0, 3), (2, 2, 3), (1, 2, 3)], 3)
+    assert tree == [[(1,), (2,)], [(1, 2), (1, 0), (2, 2)], [(1, 2, 3), (1, 2, 0), (1, 0, 3), (2, 2, 3)]]
+
+
+def test_speculative_random_trees_keep_the_result_and_the_token_bound():
+    """Whatever tree is drafted: the result is Algorithm 1's, a round's pass never exceeds |B_m| + K per further level,
+    the rounds never exceed L - 1, and accepted lengths obey the prefix rule recomputed here from the true sets."""
+    w, W, cat, model, head, V, hist = _micro()
+    rng = np.random.default_rng(5)
+    req = model.prefill(hist[1])
+    K = 3
+    ar = O.ar_beam_search(model, req, K, V)
+    true_sets = [set(codes_of(x)) for x in ar]
+    for trial in range(30):
+        tuples = [tuple(int(rng.integers(0, t)) for t in w.T) for _ in range(K)]
+        for i in range(K):                                 # splice in true prefixes so that every regime occurs
+            cut = int(rng.integers(0, w.L + 1))
+            src = codes_of(ar[-1])[int(rng.integers(0, len(ar[-1])))]
+            tuples[i] = src[:cut] + tuples[i][cut:]
+        sp, st = O.speculative_decode(model, head, req, K, V, drafts_round1=tuples)
+        assert [codes_of(x) for x in sp] == [codes_of(x) for x in ar]
+        assert 1 <= st.rounds <= w.L - 1 and st.reject_level[-1] == w.L
+        assert all(n <= K for nodes in st.tree_nodes for n in nodes)
+        reached = st.reject_level[0]
+        uniq = []
+        for t in tuples:
+            if t not in uniq:
+                uniq.append(t)
+        want = []
+        for t in uniq:
+            a = 0
+            while a < reached and t[: a + 1] in true_sets[a]:
+                a += 1
+            want.append(a)
+        assert st.accepted_len[0] == want
+
+
+def test_draft_head_hand_computed_numbers():
+    """Eq. 2 and Eq. 3 on a two-dimensional head with numbers small enough to work by hand (a swapped W_s / W_e, a
+    dropped bias or a wrong sign changes them)."""
+    shape = O.ModelShape(1, 2, 1, 1, 2, 2, (2, 2))
+    W = {"draft_logit": [np.array([[1.0, 0.0], [0.0, 1.0]]), np.array([[2.0, -1.0], [0.0, 3.0]])],
+         "draft_ws": np.array([[0.5, 0.0], [0.0, 0.25]]), "draft_we": np.array([[1.0, 1.0], [0.0, -1.0]]),
+         "draft_b": np.array([0.1, -0.1]),
+         # rows: level-1 codes 0, 1; level-2 codes 0, 1; placeholders and BOS
+         "embed": np.array([[9.0, 9.0], [0.2, 0.4], [7.0, 7.0], [-1.0, 0.5], [0, 0], [0, 0], [0, 0]])}
+    head = O.DraftHead(shape, W)
+    h1, s1 = np.array([0.5, -0.25]), np.array([1.0, 2.0])
+    assert np.allclose(head.logits(0, h1, s1), [1.5, 1.75], atol=1e-15)            # identity head: z = h + s
+    assert np.allclose(head.logits(1, h1, s1), [2 * 1.5 - 1.75, 3 * 1.75], atol=1e-15)
+    # Eq. 3 with the level-1 code 1 (embedding (0.2, 0.4)):
+    #   W_s s = (0.5, 0.5);  W_e e = (0.6, -0.4);  + b = (1.2, 0.0)  ->  s_2 = (tanh 1.2, 0)
+    s2 = head.transition(0, s1, 1)
+    assert np.allclose(s2, [0.8336546070121553, 0.0], atol=1e-15)
+    # level-2 code 1 sits at embedding row T_1 + 1 = 3: e = (-1, 0.5); W_s s_2 = (0.41682730350607766, 0);
+    #   W_e e = (-0.5, -0.5); + b = (0.01682730350607766, -0.6)
+    s3 = head.transition(1, s2, 1)
+    assert np.allclose(s3, [np.tanh(0.01682730350607766), np.tanh(-0.6)], atol=1e-15)
+    assert abs(s3[1] + 0.5370495669980353) < 1e-15                                  # tanh(0.6), a table value
+
+
+def test_draft_head_ablation_identities():
+    """Section 4.3: NEZHA-1 removes the context state, so its distribution ignores the prefix; NEZHA-2 removes the hidden
+    state, so it ignores h_l; the full head uses both and, being one linear layer over their sum, treats them alike."""
+    w, W, cat, model, head, V, hist = _micro()
+    shape = oracle_shape(w)
+    req = model.prefill(hist[0])
+    rng = np.random.default_rng(1)
+    s_a, s_b = rng.standard_normal(w.d_model), rng.standard_normal(w.d_model)
+    h1 = O.DraftHead(shape, W, use_state=False)
+    h2 = O.DraftHead(shape, W, use_hidden=False)
+    for l in range(w.L):
+        assert np.array_equal(h1.logits(l, req.h[l + 1], s_a), h1.logits(l, req.h[l + 1], s_b))
+        assert np.array_equal(h2.logits(l, s_a, req.h[0]), h2.logits(l, s_b, req.h[0]))
+        assert not np.allclose(head.logits(l, req.h[l + 1], s_a), head.logits(l, req.h[l + 1], s_b))
+        assert not np.allclose(head.logits(l, s_a, req.h[0]), head.logits(l, s_b, req.h[0]))
+        assert np.allclose(head.logits(l, s_a, s_b), head.logits(l, s_b, s_a), atol=1e-12)
+        assert np.allclose(head.logits(l, s_a, s_b), h1.logits(l, s_a, s_b) + h2.logits(l, s_a, s_b), atol=1e-12)
+    # NEZHA-1's drafts do not depend on which codes were chosen before: the per-level distributions of two different
+    # prefixes are the same
+    assert np.array_equal(h1.logits(1, req.h[2], O.teacher_forced_state(h1, req, (0,))),
+                          h1.logits(1, req.h[2], O.teacher_forced_state(h1, req, (3,))))
 
 
 # ---------------------------------------------------------------------------------------- ablation variants (Section 4.3)
