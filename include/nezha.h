@@ -91,12 +91,16 @@ typedef struct {
 /* Optional per-round device outputs of nezha_decode (any pointer may be NULL).  R = L - 1 round slots;
  * slots of rounds that did not run are filled with -1. */
 typedef struct {
-  int32_t* drafts;               /* device [R, batch, beam, L]  drafted tuples of the round, -1 padded      */
+  int32_t* drafts;               /* device [R, batch, beam, L]  drafted tuples of the round (the draft tree's  */
+                                 /*                             level-L nodes, distinct), -1 padded           */
   int32_t* n_draft;              /* device [R, batch]                                                       */
   int32_t* accepted_len;         /* device [R, batch, beam]     largest i with D[k][1..i] in B_i            */
   int32_t* level_reached;        /* device [R, batch]           level m the row had settled after the round */
   int32_t* beams;                /* device [L, batch, beam, L]  the true beam sets B_1..B_L, -1 padded      */
   float*   beam_scores;          /* device [L, batch, beam]                                                 */
+  int32_t* tree_codes;           /* device [R, L, batch, beam, L]  the round's draft tree: nodes of level j  */
+                                 /*                             (j codes each) at index j - 1, -1 padded      */
+  int32_t* tree_count;           /* device [R, L, batch]        nodes per level (-1: the row took no part)  */
 } nezha_trace;
 
 /* Decode modes. */
@@ -156,11 +160,25 @@ nezha_status nezha_decode(nezha_ctx* ctx, int32_t batch, int32_t beam_width, int
                           nezha_decode_stats* stats, const nezha_trace* trace);
 
 /* Mode 1 with the first round's drafts supplied by the caller instead of the draft head.
- *   drafts   device int32 [batch, beam_width, L];  n_draft device int32 [batch] (tuples used per row). */
+ *   drafts   device int32 [batch, beam_width, L];  n_draft device int32 [batch] (tuples used per row).
+ * The draft tree of the round is the prefix tree of the tuples: tuples that share their first j codes share one node of
+ * level j (one primary-model token); repeated tuples count once, and accepted_len / drafts of the trace index the distinct
+ * tuples in order of first appearance.  A tuple with a code outside [0, T_l) is dropped (NEZHA_ERR_CATALOG). */
 nezha_status nezha_decode_with_drafts(nezha_ctx* ctx, int32_t batch, int32_t beam_width,
                                       const int32_t* drafts, const int32_t* n_draft,
                                       int32_t* out_codes, float* out_scores, int32_t* out_count,
                                       nezha_decode_stats* stats, const nezha_trace* trace);
+
+/* Mode 1 with the first round's whole draft tree supplied by the caller (Algorithm 2's drafting step replaced; what the
+ * draft head itself proposes is such a tree: the beam sets of every level of Algorithm 3).
+ *   tree_codes  device int32 [L, batch, beam_width, L]: at index j - 1 the nodes of level j, j codes each (the rest ignored)
+ *   tree_count  device int32 [L, batch]: nodes per level and row, each <= beam_width
+ * A node whose first j - 1 codes are no node of level j - 1 is dead (never verified).  The layout is that of
+ * nezha_trace.beams, so the true beam sets of an earlier call can be passed back as a perfect draft. */
+nezha_status nezha_decode_with_draft_tree(nezha_ctx* ctx, int32_t batch, int32_t beam_width,
+                                          const int32_t* tree_codes, const int32_t* tree_count,
+                                          int32_t* out_codes, float* out_scores, int32_t* out_count,
+                                          nezha_decode_stats* stats, const nezha_trace* trace);
 
 /* Variants of the draft head: the ablations of Section 4.3 ("Ablation Study").  Defaults give Eq. 1-3 and Eq. 5 as
  * printed.  Takes effect from the next nezha_decode / nezha_draft_logits call; never touches the primary model, so

@@ -440,6 +440,52 @@ def tree_from_tuples(tuples: Sequence[Tuple[int, ...]], L: int) -> List[List[Tup
     return tree
 
 
+def alive_nodes(tree: List[List[Tuple[int, ...]]], B: List[Beam], m: int, L: int) -> Dict[int, List[Tuple[int, ...]]]:
+    """Nodes of the draft tree that the pass holds, per level m..L-1: a level-m node is alive if it is a beam of B_m, a
+    higher node if its parent is alive (its own prefix's earlier codes must be in the pass for it to attend to)."""
+    beam_set = {b.codes for b in B}
+    alive = {m: [t for t in tree[m - 1] if t in beam_set]}
+    for j in range(m + 1, L):
+        parents = set(alive[j - 1])
+        alive[j] = [t for t in tree[j - 1] if t[:-1] in parents]
+    return alive
+
+
+def verification_walk(tree: List[List[Tuple[int, ...]]], B: List[Beam], m: int, L: int, next_beams):
+    """One round of Algorithm 2 after drafting: the pass holds B_m and the alive nodes of levels m+1..L-1; B_{j+1} is
+    selected from the logits at B_j (`next_beams(B_j, j)`), level after level, while every beam of B_j is an alive node
+    (so its logits are in the pass).  The first level where that fails is the rejection level.  Returns the new true beam
+    sets [B_{m+1}, ..., B_j] and the number of tree nodes of each level m+1..L-1 that were in the pass."""
+    alive = alive_nodes(tree, B, m, L)
+    new_sets: List[List[Beam]] = []
+    j = m
+    while True:
+        B = next_beams(B, j)
+        j += 1
+        new_sets.append(B)
+        if j == L:
+            break
+        in_pass = set(alive[j])
+        if not all(b.codes in in_pass for b in B):
+            break
+    return new_sets, [len(alive[i]) for i in range(m + 1, L)]
+
+
+def accepted_lengths(tuples: Sequence[Tuple[int, ...]], true_sets: List[List[Beam]], reached: int) -> List[int]:
+    """Accepted length of every drafted tuple: the largest i <= `reached` such that each of its prefixes of 1..i codes is
+    a beam of the true set of that level (accept until the first rejection, Section 2.2)."""
+    acc = []
+    for t in tuples:
+        a = 0
+        for i in range(1, reached + 1):
+            if t[:i] in {b.codes for b in true_sets[i - 1]}:
+                a = i
+            else:
+                break
+        acc.append(a)
+    return acc
+
+
 def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: int, valid: Optional[ValidSet],
                        drafts_round1: Optional[List[Tuple[int, ...]]] = None,
                        draft_tree_round1: Optional[List[List[Tuple[int, ...]]]] = None,
@@ -486,37 +532,17 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
             tree[m - 1] = [b.codes for b in B]
             for i, beams in enumerate(lv):
                 tree[m + i] = [b.codes for b in beams]
-        beam_set = {b.codes for b in B}
-        alive = {m: [t for t in tree[m - 1] if t in beam_set]}
-        for j in range(m + 1, L):
-            parents = set(alive[j - 1])
-            alive[j] = [t for t in tree[j - 1] if t[:-1] in parents]
-        # ---- the parallel verification pass: count its tokens; logits are looked up per prefix below
-        nodes = [len(alive[j]) for j in range(m + 1, L)]
+        # ---- the parallel verification pass, progressive selection / rejection (Algorithm 2, rejection and update steps)
+        def next_beams(beams: List[Beam], j: int) -> List[Beam]:
+            logits = model.next_level_logits_many(req, [b.codes for b in beams])
+            return expand_level(beams, logits, K, s.T[j], valid if j + 1 == L else None)
+        new_sets, nodes = verification_walk(tree, B, m, L, next_beams)
+        true_sets.extend(new_sets)                       # true_sets[i - 1] is B_i
+        B = true_sets[-1]
+        j = len(true_sets)
         stats.tree_nodes.append(nodes)
-        stats.primary_tokens += len(B) + sum(nodes)
-        # ---- progressive selection / rejection (Algorithm 2, rejection and update steps)
-        j = m
-        while True:
-            logits = model.next_level_logits_many(req, [b.codes for b in B])
-            B = expand_level(B, logits, K, s.T[j], valid if j + 1 == L else None)
-            j += 1
-            true_sets.append(B)                          # true_sets[i - 1] is B_i
-            if j == L:
-                break
-            in_pass = set(alive[j])
-            if not all(b.codes in in_pass for b in B):
-                break
-        acc = []
-        for t in tree[L - 1]:
-            a = 0
-            for i in range(1, j + 1):
-                if t[:i] in {b.codes for b in true_sets[i - 1]}:
-                    a = i
-                else:
-                    break
-            acc.append(a)
-        stats.accepted_len.append(acc)
+        stats.primary_tokens += len(true_sets[m - 1]) + sum(nodes)
+        stats.accepted_len.append(accepted_lengths(tree[L - 1], true_sets, j))
         stats.reject_level.append(j)
         m = j
     return true_sets, stats

@@ -49,7 +49,8 @@ class NezhaDecodeStats(C.Structure):
 
 class NezhaTrace(C.Structure):
     _fields_ = [("drafts", C.c_void_p), ("n_draft", C.c_void_p), ("accepted_len", C.c_void_p),
-                ("level_reached", C.c_void_p), ("beams", C.c_void_p), ("beam_scores", C.c_void_p)]
+                ("level_reached", C.c_void_p), ("beams", C.c_void_p), ("beam_scores", C.c_void_p),
+                ("tree_codes", C.c_void_p), ("tree_count", C.c_void_p)]
 
 
 _vp, _i32, _sz = C.c_void_p, C.c_int32, C.c_size_t
@@ -73,6 +74,9 @@ lib.nezha_decode.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, C.POINTER(Nez
 lib.nezha_decode_with_drafts.restype = C.c_int
 lib.nezha_decode_with_drafts.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, C.POINTER(NezhaDecodeStats),
                                          C.POINTER(NezhaTrace)]
+lib.nezha_decode_with_draft_tree.restype = C.c_int
+lib.nezha_decode_with_draft_tree.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, C.POINTER(NezhaDecodeStats),
+                                             C.POINTER(NezhaTrace)]
 lib.nezha_set_option.restype = C.c_int
 lib.nezha_set_option.argtypes = [_vp, _i32, _i32]
 lib.nezha_get_hidden.restype = C.c_int
@@ -107,7 +111,7 @@ lib.nezha_destroy.argtypes = [_vp]
 NOALLOC_MAX_TUPLES = 1 << 20
 EXPORTS = ["nezha_arena_bytes", "nezha_create", "nezha_build_hashset", "nezha_pack", "nezha_probe",
            "nezha_contains_noalloc", "nezha_prefill",
-           "nezha_decode", "nezha_decode_with_drafts", "nezha_set_option", "nezha_get_hidden", "nezha_primary_logits",
+           "nezha_decode", "nezha_decode_with_drafts", "nezha_decode_with_draft_tree", "nezha_set_option", "nezha_get_hidden", "nezha_primary_logits",
            "nezha_draft_logits", "nezha_select", "nezha_gemm", "nezha_launch_count", "nezha_profile_enable",
            "nezha_profile_read", "nezha_sync", "nezha_last_error", "nezha_destroy"]
 
@@ -246,7 +250,9 @@ class Engine:
                             "accepted_len": torch.empty(R, batch, beam, dtype=torch.int32, device=dev),
                             "level_reached": torch.empty(R, batch, dtype=torch.int32, device=dev),
                             "beams": torch.empty(self.L, batch, beam, self.L, dtype=torch.int32, device=dev),
-                            "beam_scores": torch.empty(self.L, batch, beam, dtype=torch.float32, device=dev)}
+                            "beam_scores": torch.empty(self.L, batch, beam, dtype=torch.float32, device=dev),
+                            "tree_codes": torch.empty(R, self.L, batch, beam, self.L, dtype=torch.int32, device=dev),
+                            "tree_count": torch.empty(R, self.L, batch, dtype=torch.int32, device=dev)}
         return out
 
     @staticmethod
@@ -255,7 +261,7 @@ class Engine:
             return None
         t = out["trace"]
         return NezhaTrace(_ptr(t["drafts"]), _ptr(t["n_draft"]), _ptr(t["accepted_len"]), _ptr(t["level_reached"]),
-                          _ptr(t["beams"]), _ptr(t["beam_scores"]))
+                          _ptr(t["beams"]), _ptr(t["beam_scores"]), _ptr(t.get("tree_codes")), _ptr(t.get("tree_count")))
 
     def decode(self, beam: int, mode: int = MODE_VERIFIED, out=None, trace: bool = False, want_stats: bool = True):
         out = out if out is not None else self.alloc_outputs(self.batch, beam, trace)
@@ -275,6 +281,21 @@ class Engine:
         self._check(lib.nezha_decode_with_drafts(self._h, self.batch, beam, _ptr(drafts), _ptr(n_draft),
                                                  _ptr(out["codes"]), _ptr(out["scores"]), _ptr(out["count"]),
                                                  C.byref(stats), C.byref(tr) if tr is not None else None))
+        out["stats"] = stats
+        return out
+
+    def decode_with_draft_tree(self, beam: int, tree_codes: torch.Tensor, tree_count: torch.Tensor, out=None,
+                               trace: bool = False):
+        """tree_codes int32 [L, batch, beam, L], tree_count int32 [L, batch] (the layout of the trace's `beams`)."""
+        out = out if out is not None else self.alloc_outputs(self.batch, beam, trace)
+        stats = NezhaDecodeStats()
+        tr = self._trace_struct(out)
+        assert tuple(tree_codes.shape) == (self.L, self.batch, beam, self.L) and tree_codes.dtype == torch.int32
+        assert tuple(tree_count.shape) == (self.L, self.batch) and tree_count.dtype == torch.int32
+        tree_codes, tree_count = tree_codes.contiguous(), tree_count.contiguous()
+        self._check(lib.nezha_decode_with_draft_tree(self._h, self.batch, beam, _ptr(tree_codes), _ptr(tree_count),
+                                                     _ptr(out["codes"]), _ptr(out["scores"]), _ptr(out["count"]),
+                                                     C.byref(stats), C.byref(tr) if tr is not None else None))
         out["stats"] = stats
         return out
 

@@ -250,8 +250,8 @@ size_t carve(nezha_ctx* c) {
   e.row_m = cv.take<int>(c->Bmax); e.row_cur = cv.take<int>(c->Bmax); e.row_P = cv.take<int>(c->Bmax);
   e.dw_codes = cv.take<int>(lbk * c->L); e.dw_score = cv.take<float>(lbk); e.dw_parent = cv.take<int>(lbk);
   e.dw_count = cv.take<int>((size_t)(c->L + 1) * c->Bmax);
-  e.d_m = cv.take<int>(c->Bmax); e.d_alive = cv.take<int>((size_t)c->Bmax * c->Kmax);
-  e.d_beam = cv.take<int>((size_t)c->Bmax * c->Kmax);
+  e.d_m = cv.take<int>(c->Bmax);
+  e.d_beam = cv.take<int>(lbk);
   e.state_lv = cv.take<float>(lbk * c->d);
   e.node_index = cv.take<int>((size_t)c->Bmax * c->L * c->Kmax);
   e.tok_row = cv.take<int>(c->Ms); e.tok_pos = cv.take<int>(c->Ms); e.tok_id = cv.take<int>(c->Ms);
@@ -524,7 +524,8 @@ nezha_status run_segment(nezha_ctx* c, const std::array<uintptr_t, 16>& key, F&&
   return NEZHA_OK;
 }
 
-nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* drafts, const int* n_draft,
+// drafts / n_draft: round 1's drafted tuples, or (is_tree) round 1's whole draft tree and its per-level counts
+nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* drafts, const int* n_draft, bool is_tree,
                          int* out_codes, float* out_scores, int* out_count, nezha_decode_stats* stats,
                          const nezha_trace* trace) {
   if (!c) return NEZHA_ERR_ARG;
@@ -547,10 +548,11 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
   const int R = L - 1;
   auto key_of = [&](int segment) {
     std::array<uintptr_t, 16> k{};
-    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20);
+    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20 | (is_tree ? 1 : 0) << 24);
     k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
     k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
-    k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams; k[14] = (uintptr_t)tr.beam_scores;
+    k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams ^ ((uintptr_t)tr.tree_codes << 1);
+    k[14] = (uintptr_t)tr.beam_scores ^ ((uintptr_t)tr.tree_count << 1);
     k[15] = (uintptr_t)c->m_seen[segment];           // the expected token count shapes the tiling of the round's GEMMs
     return k;
   };
@@ -559,6 +561,8 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     if (tr.n_draft) launch_fill_i32(tr.n_draft, (long long)R * batch, -1, c->st);
     if (tr.accepted_len) launch_fill_i32(tr.accepted_len, (long long)R * batch * K, -1, c->st);
     if (tr.level_reached) launch_fill_i32(tr.level_reached, (long long)R * batch, -1, c->st);
+    if (tr.tree_codes) launch_fill_i32(tr.tree_codes, (long long)R * L * batch * K * L, -1, c->st);
+    if (tr.tree_count) launch_fill_i32(tr.tree_count, (long long)R * L * batch, -1, c->st);
     launch_fill_i32(out_codes, (long long)batch * K * L, -1, c->st);
     launch_fill_f32(out_scores, (long long)batch * K, -INFINITY, c->st);
     launch_fill_i32(out_count, batch, 0, c->st);
@@ -596,6 +600,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     c->m_expected = c->m_seen[round];
     rs = run_segment(c, key_of(round), [&] {
       if (mode == NEZHA_MODE_AR) launch_draft_set(e, batch, K, nullptr, nullptr, c->st);
+      else if (round == 1 && drafts && is_tree) launch_draft_tree_set(e, batch, K, drafts, n_draft, c->st);
       else if (round == 1 && drafts) launch_draft_set(e, batch, K, drafts, n_draft, c->st);
       else draft_phase(c, batch, K, round == 1, round == 1 ? 1 : round + 1, c->opt_filter != 0);
       launch_build_nodes(e, batch, c->st);
@@ -824,7 +829,7 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
 
 nezha_status nezha_decode(nezha_ctx* c, int32_t batch, int32_t beam_width, int32_t mode, int32_t* out_codes,
                           float* out_scores, int32_t* out_count, nezha_decode_stats* stats, const nezha_trace* trace) {
-  return decode_impl(c, batch, beam_width, mode, nullptr, nullptr, out_codes, out_scores, out_count, stats, trace);
+  return decode_impl(c, batch, beam_width, mode, nullptr, nullptr, false, out_codes, out_scores, out_count, stats, trace);
 }
 
 nezha_status nezha_decode_with_drafts(nezha_ctx* c, int32_t batch, int32_t beam_width, const int32_t* drafts,
@@ -832,8 +837,17 @@ nezha_status nezha_decode_with_drafts(nezha_ctx* c, int32_t batch, int32_t beam_
                                       nezha_decode_stats* stats, const nezha_trace* trace) {
   if (!c) return NEZHA_ERR_ARG;
   if (!drafts || !n_draft) return fail(c, NEZHA_ERR_ARG, "nezha_decode_with_drafts: null drafts");
-  return decode_impl(c, batch, beam_width, NEZHA_MODE_VERIFIED, drafts, n_draft, out_codes, out_scores, out_count, stats,
-                     trace);
+  return decode_impl(c, batch, beam_width, NEZHA_MODE_VERIFIED, drafts, n_draft, false, out_codes, out_scores, out_count,
+                     stats, trace);
+}
+
+nezha_status nezha_decode_with_draft_tree(nezha_ctx* c, int32_t batch, int32_t beam_width, const int32_t* tree_codes,
+                                          const int32_t* tree_count, int32_t* out_codes, float* out_scores,
+                                          int32_t* out_count, nezha_decode_stats* stats, const nezha_trace* trace) {
+  if (!c) return NEZHA_ERR_ARG;
+  if (!tree_codes || !tree_count) return fail(c, NEZHA_ERR_ARG, "nezha_decode_with_draft_tree: null tree");
+  return decode_impl(c, batch, beam_width, NEZHA_MODE_VERIFIED, tree_codes, tree_count, true, out_codes, out_scores,
+                     out_count, stats, trace);
 }
 
 nezha_status nezha_set_option(nezha_ctx* c, int32_t option, int32_t value) {

@@ -370,7 +370,7 @@ __global__ void init_decode_kernel(EngineState e, int batch) {
   e.row_m[b] = 0;
   e.row_cur[b] = -1;
   e.d_m[b] = e.L;
-  e.dw_count[(long long)e.L * e.Bmax + b] = 0;
+  for (int l = 0; l <= e.L; ++l) e.dw_count[(long long)l * e.Bmax + b] = 0;     // no draft tree yet
 }
 
 // Start of a round's drafting (Algorithm 2's drafting step): the draft head continues from the true beams B_m, or from
@@ -405,26 +405,100 @@ __global__ void draft_init_kernel(EngineState e, int batch, int from_scratch, __
   if (threadIdx.x == 0) { e.dw_count[mm * e.Bmax + b] = cnt; e.d_m[b] = mm; }
 }
 
-// Caller-supplied drafts for the round (or none: n_draft == nullptr and drafts == nullptr -> zero drafts).
+// Caller-supplied drafted tuples for the round (or none: n_draft == nullptr and drafts == nullptr -> an empty tree).
+// The tree of the tuples is built level by level: level j holds their distinct j-prefixes in order of first appearance
+// (tuples that share a prefix share its node), each with the slot of its parent.  One block of >= Kmax threads per request.
 __global__ void draft_set_kernel(EngineState e, int batch, int K, const int* drafts, const int* n_draft) {
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x;
   if (b == 0 && threadIdx.x < 8) e.counters[threadIdx.x] = 0;      // first kernel of the round: clear its counters
   if (b >= batch) return;
-  const int cnt = (drafts && e.row_m[b] < e.L) ? max(0, min(n_draft[b], K)) : 0;
-  for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
-    const long long s = lvl_bk(e, e.L, b, k);
-    bool ok = k < cnt;
-    for (int l = 0; l < e.L; ++l) {
-      int c = ok ? drafts[((long long)b * K + k) * e.L + l] : -1;
-      if (ok && (c < 0 || c >= e.li.T[l])) { atomicOr(e.status, kStBadCode); c = 0; }
-      e.dw_codes[s * e.L + l] = c;
-    }
-    e.dw_score[s] = ok ? 0.f : -INFINITY;
-    e.dw_parent[s] = -1;
+  const int L = e.L, k = threadIdx.x;
+  __shared__ int s_slot[2][128];                 // slot of tuple k's prefix in the previous / the current level
+  __shared__ int s_new[128], s_ok[128], s_cnt;
+  const int cnt = (drafts && e.row_m[b] < L) ? max(0, min(n_draft[b], K)) : 0;
+  int code[kMaxLevels];
+  bool ok = k < cnt;
+  for (int l = 0; l < L; ++l) {
+    code[l] = ok ? drafts[((long long)b * K + k) * L + l] : -1;
+    if (k < cnt && (code[l] < 0 || code[l] >= e.li.T[l])) { atomicOr(e.status, kStBadCode); ok = false; }
   }
-  if (threadIdx.x == 0) { e.dw_count[(long long)e.L * e.Bmax + b] = cnt; e.d_m[b] = e.L; }
+  s_slot[0][k] = 0;                              // level 0: the empty prefix, slot 0
+  s_ok[k] = ok ? 1 : 0;                          // a tuple with an out-of-range code is dropped as a whole
+  __syncthreads();
+  for (int j = 1; j <= L; ++j) {
+    const int cur = j & 1, prev = cur ^ 1;
+    int first = -1;                              // the first tuple with the same j-prefix
+    if (ok) {
+      for (int k2 = 0; k2 <= k && first < 0; ++k2) {
+        if (!s_ok[k2]) continue;
+        bool eq = true;
+        for (int l = 0; l < j; ++l) eq &= (drafts[((long long)b * K + k2) * L + l] == code[l]);
+        if (eq) first = k2;
+      }
+    }
+    s_new[k] = (ok && first == k) ? 1 : 0;
+    __syncthreads();
+    if (k == 0) {                                // exclusive scan of the "new node" flags -> slots
+      int c = 0;
+      for (int i = 0; i < cnt; ++i) { const int f = s_new[i]; s_new[i] = c; c += f; }
+      s_cnt = c;
+    }
+    __syncthreads();
+    if (ok) {
+      const int slot = s_new[first];
+      s_slot[cur][k] = slot;
+      if (first == k) {
+        const long long s = lvl_bk(e, j, b, slot);
+        for (int l = 0; l < L; ++l) e.dw_codes[s * L + l] = l < j ? code[l] : -1;
+        e.dw_score[s] = 0.f;
+        e.dw_parent[s] = s_slot[prev][k];
+      }
+    }
+    if (k == 0) e.dw_count[(long long)j * e.Bmax + b] = s_cnt;
+    __syncthreads();
+  }
+  if (k == 0) e.d_m[b] = L;
+}
+
+// Caller-supplied draft tree (test hook): level j's nodes are taken as listed; a node's parent is the node of level j - 1
+// that equals its first j - 1 codes (-1 if there is none: the node is then dead).  One block of >= Kmax threads per request.
+__global__ void draft_tree_set_kernel(EngineState e, int batch, int K, const int* tree_codes, const int* tree_count) {
+  pdl_wait();
+  pdl_launch();
+  const int b = blockIdx.x;
+  if (b == 0 && threadIdx.x < 8) e.counters[threadIdx.x] = 0;
+  if (b >= batch) return;
+  const int L = e.L, k = threadIdx.x;
+  const bool row_live = e.row_m[b] < L;
+  for (int j = 1; j <= L; ++j) {
+    const int cnt = row_live ? max(0, min(tree_count[(long long)(j - 1) * batch + b], K)) : 0;
+    const int cnt_prev = j > 1 && row_live ? max(0, min(tree_count[(long long)(j - 2) * batch + b], K)) : 0;
+    if (k < cnt) {
+      const int* src = tree_codes + (((long long)(j - 1) * batch + b) * K + k) * L;
+      const long long s = lvl_bk(e, j, b, k);
+      bool ok = true;
+      for (int l = 0; l < L; ++l) {
+        int c = l < j ? src[l] : -1;
+        if (l < j && (c < 0 || c >= e.li.T[l])) { atomicOr(e.status, kStBadCode); ok = false; c = 0; }
+        e.dw_codes[s * L + l] = c;
+      }
+      int parent = j == 1 ? 0 : -1;
+      if (ok && j > 1) {
+        const int* prv = tree_codes + (((long long)(j - 2) * batch + b) * K) * L;
+        for (int k2 = 0; k2 < cnt_prev && parent < 0; ++k2) {
+          bool eq = true;
+          for (int l = 0; l < j - 1; ++l) eq &= (prv[(long long)k2 * L + l] == src[l]);
+          if (eq) parent = k2;
+        }
+      }
+      e.dw_score[s] = 0.f;
+      e.dw_parent[s] = ok ? parent : -1;
+    }
+    if (k == 0) e.dw_count[(long long)j * e.Bmax + b] = cnt;
+  }
+  if (k == 0) e.d_m[b] = L;
 }
 
 // Eq. 2 input: x = h_l + s_l for every (request, beam); s_1 = h_0 (Eq. 1).
@@ -551,9 +625,11 @@ __global__ void copy_logits_bias_kernel(const float* src, long long row_stride, 
 // ----------------------------------------------------------------------------------------------------
 // verify-pass token list (the nodes M_p runs on this round)
 // ----------------------------------------------------------------------------------------------------
-// Request with m levels settled: nodes = the level-m code of every beam of B_m (slot = beam rank) and the codes
-// of levels m+1..L-1 of every alive draft (slot = draft index).  Tokens of a request are contiguous; requests
-// are laid out in order (each block sums the counts of the requests before it).
+// Request with m levels settled: nodes = the level-m code of every beam of B_m (slot = beam rank) and, for the levels
+// m+1..L-1, the last code of every alive node of the round's draft tree (slot = the node's slot in its level): one token
+// per distinct drafted prefix.  A level-m node of the tree is alive if its codes are a beam of B_m; a higher node if its
+// parent is alive.  Tokens of a request are contiguous; requests are laid out in order (each block sums the counts of the
+// requests before it).
 __global__ void nodes_count_kernel(EngineState e, int batch) {
   pdl_wait();
   pdl_launch();
@@ -565,39 +641,46 @@ __global__ void nodes_count_kernel(EngineState e, int batch) {
   __syncthreads();
   if (m >= L) {
     if (threadIdx.x == 0) { e.row_tok_count[b] = 0; e.row_cur[b] = -1; e.req_info[b] = make_int4(0, 0, b, 0); }
-    for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) e.d_alive[b * e.Kmax + k] = 0;
     return;
   }
   const int nb = e.tb_count[m * e.Bmax + b];
-  const int nd = e.dw_count[(long long)L * e.Bmax + b];
-  for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
-    int beta = -1;
-    if (k < nd) {
-      const int* dc = e.dw_codes + lvl_bk(e, L, b, k) * L;
-      for (int r = 0; r < nb && beta < 0; ++r) {
-        const int* bc = e.tb_codes + lvl_bk(e, m, b, r) * L;
-        bool eq = true;
-        for (int l = 0; l < m; ++l) eq &= (dc[l] == bc[l]);
-        if (eq) beta = r;
+  for (int j = m; j < L; ++j) {
+    const int cnt = min(e.dw_count[(long long)j * e.Bmax + b], e.Kmax);
+    for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
+      int beta = -1;
+      if (k < cnt) {
+        if (j == m) {
+          const int* dc = e.dw_codes + lvl_bk(e, m, b, k) * L;
+          for (int r = 0; r < nb && beta < 0; ++r) {
+            const int* bc = e.tb_codes + lvl_bk(e, m, b, r) * L;
+            bool eq = true;
+            for (int l = 0; l < m; ++l) eq &= (dc[l] == bc[l]);
+            if (eq) beta = r;
+          }
+        } else {
+          const int p = e.dw_parent[lvl_bk(e, j, b, k)];
+          if (p >= 0 && p < e.Kmax) beta = e.d_beam[lvl_bk(e, j - 1, b, p)];
+          if (beta >= 0) atomicAdd(&n_alive, 1);
+        }
       }
+      e.d_beam[lvl_bk(e, j, b, k)] = beta;
     }
-    e.d_alive[b * e.Kmax + k] = beta >= 0;
-    e.d_beam[b * e.Kmax + k] = beta;
-    if (beta >= 0) atomicAdd(&n_alive, 1);
+    __syncthreads();                               // level j's answers (global, this block's own) before level j + 1 reads them
   }
-  __syncthreads();
   if (threadIdx.x == 0) {
-    e.row_tok_count[b] = nb + n_alive * (L - 1 - m);
+    e.row_tok_count[b] = nb + n_alive;
     e.row_cur[b] = m;
   }
 }
 
-__global__ void nodes_fill_kernel(EngineState e, int batch) {
+__global__ void __launch_bounds__(128) nodes_fill_kernel(EngineState e, int batch) {
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x;
   const int L = e.L, Kmax = e.Kmax;
-  __shared__ int s_off, s_alive_rank[128], s_n_alive;
+  __shared__ int s_off, s_rank[kMaxLevels][128], s_level_start[kMaxLevels + 1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  const int m = e.row_m[b];
   if (threadIdx.x == 0) {
     int off = 0;
     for (int i = 0; i < b; ++i) off += e.row_tok_count[i];
@@ -605,15 +688,28 @@ __global__ void nodes_fill_kernel(EngineState e, int batch) {
     e.row_tok_start[b] = off;
     if (e.row_tok_count[b] > 0) e.req_info[b] = make_int4(off, e.row_tok_count[b], b, e.row_P[b]);
     if (b == batch - 1) *e.n_tokens = off + e.row_tok_count[b];
-    int c = 0;
-    for (int k = 0; k < Kmax; ++k) { s_alive_rank[k] = c; c += e.d_alive[b * Kmax + k]; }
-    s_n_alive = c;
   }
   for (int i = threadIdx.x; i < L * Kmax; i += blockDim.x) e.node_index[(long long)b * L * Kmax + i] = -1;
+  // rank of every alive node within its level (a warp per level: ballots over its <= 128 slots)
+  for (int j = m + 1 + warp; j < L; j += n_warps) {
+    int base = 0;
+    for (int k0 = 0; k0 < Kmax; k0 += 32) {
+      const int k = k0 + lane;
+      const bool alive = k < Kmax && k < e.dw_count[(long long)j * e.Bmax + b] && e.d_beam[lvl_bk(e, j, b, k)] >= 0;
+      const unsigned mask = __ballot_sync(0xffffffffu, alive);
+      if (k < 128) s_rank[j][k] = alive ? base + __popc(mask & ((1u << lane) - 1u)) : -1;
+      base += __popc(mask);
+    }
+    if (lane == 0) s_level_start[j] = base;        // the level's count for now; turned into a start below
+  }
   __syncthreads();
-  const int m = e.row_m[b];
   if (m >= L) return;
   const int nb = e.tb_count[m * e.Bmax + b];
+  if (threadIdx.x == 0) {
+    int start = nb;
+    for (int j = m + 1; j < L; ++j) { const int c = s_level_start[j]; s_level_start[j] = start; start += c; }
+  }
+  __syncthreads();
   const int P = e.row_P[b];
   const long long slab_elems = (long long)Kmax * e.Hkv * e.hd;       // one level slab of one request
   const long long row_elems = (long long)(L - 1) * slab_elems;
@@ -637,23 +733,27 @@ __global__ void nodes_fill_kernel(EngineState e, int batch) {
     e.tb_self[bi] = r;
     e.node_index[((long long)b * L + m) * Kmax + r] = t;
   }
-  // levels m+1 .. L-1 of alive drafts
+  // levels m+1 .. L-1: the alive nodes of the draft tree
   const int n_lv = L - 1 - m;
   for (int idx = threadIdx.x; idx < n_lv * Kmax; idx += blockDim.x) {
     const int j = m + 1 + idx / Kmax, k = idx % Kmax;
-    if (!e.d_alive[b * Kmax + k]) continue;
-    const int t = s_off + nb + (j - m - 1) * s_n_alive + s_alive_rank[k];
-    const int beta = e.d_beam[b * Kmax + k];
+    const int rank = s_rank[j][k];
+    if (rank < 0) continue;
+    const int t = s_off + s_level_start[j] + rank;
+    const int beta = e.d_beam[lvl_bk(e, j, b, k)];
     const long long bi = lvl_bk(e, m, b, beta);
-    const long long di = lvl_bk(e, L, b, k);
+    const long long di = lvl_bk(e, j, b, k);
     e.tok_row[t] = b; e.tok_pos[t] = P + j - 1; e.tok_ctx_len[t] = P;
     e.tok_id[t] = e.li.off[j - 1] + e.dw_codes[di * L + (j - 1)];
     e.tok_kv_dst[t] = kv_off(j, k);
+    int anc[kMaxLevels + 1];                       // anc[i] = slot of the node's ancestor of level i in the tree
+    anc[j] = k;
+    for (int i = j; i > m + 1; --i) anc[i - 1] = e.dw_parent[lvl_bk(e, i, b, anc[i])];
     for (int i = 1; i <= L; ++i) {
       long long o = -1;
       if (i < m) o = kv_off(i, e.tb_anc[bi * L + (i - 1)]);
       else if (i == m) o = kv_off(m, beta);
-      else if (i <= j) o = kv_off(i, k);
+      else if (i <= j) o = kv_off(i, anc[i]);
       e.tok_ext[(long long)t * L + (i - 1)] = o;
     }
     e.node_index[((long long)b * L + j) * Kmax + k] = t;
@@ -699,8 +799,8 @@ __global__ void nodes_from_prefixes_kernel(EngineState e, int batch, int n_beams
 // After B_{n+1} has been selected for a request whose beams B_n had logits in this pass:
 //   n + 1 == L : the request is finished; B_L is the result.
 //   otherwise  : every beam of B_{n+1} inherits its parent's KV slots (a slot-table rewrite: rejected drafts'
-//                KV rows simply become unreachable) and is matched against the alive drafts.  If every beam is
-//                the (n+1)-prefix of a draft, its hidden state is already in the pass and selection goes on;
+//                KV rows simply become unreachable) and is matched against the alive nodes of level n+1 of the draft
+//                tree.  If every beam is such a node, its hidden state is already in the pass and selection goes on;
 //                else level n+1 is the rejection level and the request waits for the next round.
 __device__ __forceinline__ void advance_body(const EngineState& e, int n, int K, int* out_codes, float* out_score, int* out_count) {
   const int b = blockIdx.x;
@@ -720,7 +820,7 @@ __device__ __forceinline__ void advance_body(const EngineState& e, int n, int K,
   __shared__ int all_matched;
   if (threadIdx.x == 0) all_matched = 1;
   __syncthreads();
-  const int nd = e.dw_count[(long long)L * e.Bmax + b];
+  const int nd = min(e.dw_count[(long long)n1 * e.Bmax + b], Kmax);
   for (int r = threadIdx.x; r < cnt; r += blockDim.x) {
     const long long bi = lvl_bk(e, n1, b, r);
     const int parent = e.tb_parent[bi];
@@ -730,8 +830,8 @@ __device__ __forceinline__ void advance_body(const EngineState& e, int n, int K,
     const int* bc = e.tb_codes + bi * L;
     int match = -1;
     for (int k = 0; k < nd && match < 0; ++k) {
-      if (!e.d_alive[b * Kmax + k]) continue;
-      const int* dc = e.dw_codes + lvl_bk(e, L, b, k) * L;
+      if (e.d_beam[lvl_bk(e, n1, b, k)] < 0) continue;
+      const int* dc = e.dw_codes + lvl_bk(e, n1, b, k) * L;
       bool eq = true;
       for (int l = 0; l < n1; ++l) eq &= (dc[l] == bc[l]);
       if (eq) match = k;
@@ -807,7 +907,16 @@ __global__ void round_end_kernel(EngineState e, int batch, int K, int round, nez
     if (tr.drafts)
       for (int l = 0; l < L; ++l)
         tr.drafts[(tro * K + k) * L + l] = (k < nd) ? e.dw_codes[lvl_bk(e, L, b, k) * L + l] : -1;
+    if (tr.tree_codes)
+      for (int j = 1; j <= L; ++j) {
+        const int nj = took_part ? min(e.dw_count[(long long)j * e.Bmax + b], Kmax) : 0;
+        const long long o = ((((long long)(round - 1) * L + (j - 1)) * batch + b) * K + k) * L;
+        for (int l = 0; l < L; ++l) tr.tree_codes[o + l] = (k < nj && l < j) ? e.dw_codes[lvl_bk(e, j, b, k) * L + l] : -1;
+      }
   }
+  if (tr.tree_count && threadIdx.x < L)
+    tr.tree_count[((long long)(round - 1) * L + threadIdx.x) * batch + b] =
+        took_part ? min(min(e.dw_count[(long long)(threadIdx.x + 1) * e.Bmax + b], Kmax), K) : -1;
   __syncthreads();
   if (threadIdx.x == 0) {
     if (tr.n_draft) tr.n_draft[tro] = took_part ? nd : -1;
@@ -885,7 +994,11 @@ void launch_draft_init(const EngineState& e, int batch, int from_scratch, void* 
 }
 void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);
-  launch_pdl(draft_set_kernel, dim3(batch), dim3(64), 0, st, e, batch, K, drafts, n_draft);
+  launch_pdl(draft_set_kernel, dim3(batch), dim3(128), 0, st, e, batch, K, drafts, n_draft);
+}
+void launch_draft_tree_set(const EngineState& e, int batch, int K, const int* tree_codes, const int* tree_count, cudaStream_t st) {
+  LaunchScope ls(kcDraftGlue, st);
+  launch_pdl(draft_tree_set_kernel, dim3(batch), dim3(128), 0, st, e, batch, K, tree_codes, tree_count);
 }
 void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st) {
   LaunchScope ls(kcDraftGlue, st);

@@ -27,11 +27,13 @@ struct EngineState {
   int* row_cur;     // [Bmax] level whose beams have logits in the current pass, -1 = row stopped this round
   int* row_P;       // [Bmax] context length of the row (BOS + history tokens)
 
-  // draft working sets, [L+1][Bmax][Kmax]([L]); the drafts of the round are level L
+  // The round's draft tree, [L+1][Bmax][Kmax]([L]): level l holds the drafted nodes with l codes (the draft head's beam
+  // set of that level, or the distinct l-prefixes of caller-supplied tuples); dw_parent = slot of the node's parent in
+  // level l - 1.  The drafted tuples of the round are level L.
   int* dw_codes; float* dw_score; int* dw_parent; int* dw_count;
-  int* d_m;         // [Bmax] level the row's drafting started from this round (L = row takes no part)
-  int* d_alive;     // [Bmax][Kmax] 1 if the draft's first row_m codes are a true beam
-  int* d_beam;      // [Bmax][Kmax] rank of that beam
+  int* d_m;         // [Bmax] level the row's drafting started from this round (L = the draft head takes no part)
+  int* d_beam;      // [L+1][Bmax][Kmax] for a node in this round's pass: rank of the true beam of B_m it descends from
+                    //                   (-1: the node is dead -- its first m codes are no beam, or it has no parent)
   float* state_lv;  // [L+1][Bmax][Kmax][d] draft-head context states s_l (l = 2..L used; s_1 = h_0)
 
   // verify-pass token list
@@ -79,6 +81,8 @@ cudaError_t select_configure(int max_beam);
 void launch_init_decode(const EngineState& e, int batch, cudaStream_t st);
 void launch_draft_init(const EngineState& e, int batch, int from_scratch, void* s_act, cudaStream_t st);   // s_act may be null
 void launch_draft_set(const EngineState& e, int batch, int K, const int* drafts, const int* n_draft, cudaStream_t st);
+// the whole tree given by the caller: tree_codes [L][batch][K][L], tree_count [L][batch]
+void launch_draft_tree_set(const EngineState& e, int batch, int K, const int* tree_codes, const int* tree_count, cudaStream_t st);
 void launch_draft_x(const EngineState& e, int batch, int l, void* x, bool bf16, cudaStream_t st);
 void launch_trans_gather(const EngineState& e, int batch, int l, const void* embed, void* A, bool bf16,
                          cudaStream_t st);

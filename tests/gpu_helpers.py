@@ -135,3 +135,48 @@ def check_levels(case, b, beams, beam_scores, K, per_beam_all=True, tol=None):
         cnt = int((beams[n, :, 0] >= 0).sum())
         assert_topk_matches(beams[n][:, : n + 1], beam_scores[n], cnt, ref, K, tol)
         prev = [O.Beam(tuple(int(c) for c in beams[n, k, : n + 1]), np.float32(beam_scores[n, k])) for k in range(cnt)]
+
+
+def replay_walk_from_trace(tr, b, L):
+    """Algorithm 2's walk of one request replayed from the GPU's own trace -- the draft tree of every round and the true
+    beam sets -- with the oracle's integer rules (which nodes are alive, where the walk stops, accepted lengths).  No
+    logits are involved, so the comparison is bit exact on any workload.
+    Returns (rounds, level reached per round, accepted lengths per round, primary-model tokens)."""
+    sets = []
+    for n in range(L):
+        cnt = int((tr["beams"][n, b, :, 0] >= 0).sum())
+        sets.append([O.Beam(tuple(int(c) for c in tr["beams"][n, b, k, : n + 1]), np.float32(tr["beam_scores"][n, b, k]))
+                     for k in range(cnt)])
+    m, r, tokens, reached, acc = 1, 0, 0, [], []
+    while m < L:
+        tree = [[tuple(int(c) for c in tr["tree_codes"][r, j, b, k, : j + 1]) for k in range(max(int(tr["tree_count"][r, j, b]), 0))]
+                for j in range(L)]
+        new_sets, nodes = O.verification_walk(tree, sets[m - 1], m, L, lambda beams, j: sets[j])
+        j = m + len(new_sets)
+        tokens += len(sets[m - 1]) + sum(nodes)
+        reached.append(j)
+        acc.append(O.accepted_lengths(tree[L - 1], sets, j))
+        m, r = j, r + 1
+    return r, reached, acc, tokens
+
+
+def check_walk_against_trace(out, batch, L, rows=None):
+    """accepted_len, level_reached, rounds and token counts of a traced decode call against the replay above."""
+    tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+    tot_tokens, max_rounds = 0, 0
+    for b in range(batch):
+        rounds, reached, acc, tokens = replay_walk_from_trace(tr, b, L)
+        tot_tokens += tokens
+        max_rounds = max(max_rounds, rounds)
+        if rows is not None and b not in rows:
+            continue
+        for r in range(rounds):
+            n = int(tr["n_draft"][r, b])
+            assert n == len(acc[r]), (b, r, n, len(acc[r]))
+            assert list(tr["accepted_len"][r, b, :n]) == acc[r], (b, r)
+            assert np.all(tr["accepted_len"][r, b, n:] == -1)
+            assert int(tr["level_reached"][r, b]) == reached[r], (b, r)
+        assert np.all(tr["level_reached"][rounds:, b] == -1)
+    assert out["stats"].primary_tokens == tot_tokens, (out["stats"].primary_tokens, tot_tokens)
+    assert out["stats"].rounds == max_rounds
+    return tot_tokens, max_rounds

@@ -11,7 +11,7 @@ import torch
 
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
-from gpu_helpers import Case, check_levels, e2e_tolerance, hidden_rms_bound, hidden_tolerance, stage_tolerance
+from gpu_helpers import Case, check_levels, check_walk_against_trace, e2e_tolerance, hidden_rms_bound, hidden_tolerance, stage_tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -48,6 +48,14 @@ def test_full_size_workload(name):
     live = np.arange(w.beam)[None, :] < count[:, None]
     assert V.contains(codes[live]).all() and np.all(codes[~live] == -1)
     assert 1 <= out["stats"].rounds <= w.L - 1
+    # accept / roll-back bookkeeping of every request, replayed from the GPU's own beams and draft trees (integers only)
+    check_walk_against_trace(out, w.batch, w.L)
+    beams_dev = out["trace"]["beams"]
+    counts = (beams_dev[:, :, :, 0] >= 0).sum(dim=2).to(torch.int32)
+    perfect = case.eng.decode_with_draft_tree(w.beam, beams_dev.clone(), counts, trace=True)
+    assert torch.equal(perfect["codes"], ar["codes"]) and torch.allclose(perfect["scores"], ar["scores"], atol=1e-4)
+    assert perfect["stats"].rounds == 1 and perfect["stats"].primary_tokens == int(counts[: w.L - 1].sum())
+    check_walk_against_trace(perfect, w.batch, w.L)
     dr = case.eng.decode(w.beam, mode=0)
     dcodes, dcount = dr["codes"].cpu().numpy(), dr["count"].cpu().numpy()
     dlive = np.arange(w.beam)[None, :] < dcount[:, None]

@@ -6,7 +6,7 @@ import torch
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
 from helpers import codes_of
-from gpu_helpers import Case, assert_topk_matches, check_levels, tolerance
+from gpu_helpers import Case, assert_topk_matches, check_levels, check_walk_against_trace, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -208,10 +208,14 @@ def test_mode_verified_equals_ar_and_matches_oracle_trace(tiny):
             nd = tr["n_draft"][r, b]
             assert list(tr["accepted_len"][r, b, :nd]) == st.accepted_len[r]
             assert tr["level_reached"][r, b] == st.reject_level[r]
+            want_tree = [len(x) for x in O.nezha_draft(head, tiny.req(b), w.beam, V)] if r == 0 else None
+            if want_tree is not None:
+                assert list(tr["tree_count"][0, :, b]) == want_tree
         assert np.all(tr["level_reached"][st.rounds:, b] == -1)
         tot_tokens += st.primary_tokens
         max_rounds = max(max_rounds, st.rounds)
     assert out["stats"].primary_tokens == tot_tokens and out["stats"].rounds == max_rounds
+    assert check_walk_against_trace(out, w.batch, w.L) == (tot_tokens, max_rounds)
 
 
 def test_decode_with_drafts_acceptance_regimes(tiny):
@@ -232,14 +236,47 @@ def test_decode_with_drafts_acceptance_regimes(tiny):
         out = tiny.eng.decode_with_drafts(K, torch.from_numpy(drafts).cuda(), torch.from_numpy(n_draft).cuda(), trace=True)
         assert torch.equal(out["codes"], ar["codes"])                        # result never depends on the drafts
         tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+        tot = 0
         for b in range(w.batch):
             D = [tuple(int(c) for c in drafts[b, k]) for k in range(n_draft[b])]
             sets, st = O.speculative_decode(model, head, tiny.req(b), K, V, drafts_round1=D)
             assert codes_of(sets[-1]) == [tuple(int(c) for c in ar_codes[b, k]) for k in range(len(sets[-1]))]
-            assert list(tr["accepted_len"][0, b, : n_draft[b]]) == st.accepted_len[0]
+            n = len(st.accepted_len[0])                                      # distinct tuples
+            assert tr["n_draft"][0, b] == n
+            assert list(tr["accepted_len"][0, b, :n]) == st.accepted_len[0]
             assert tr["level_reached"][0, b] == st.reject_level[0]
-            if rho == 0.0 and st.rounds == 1:
-                assert st.accepted_len[0] == [w.L] * n_draft[b]
+            assert list(tr["tree_count"][0, :, b]) == [len(x) for x in O.tree_from_tuples(D, w.L)]
+            if rho == 0.0:                                                   # true tuples: accepted as far as the round got
+                assert st.accepted_len[0] == [st.reject_level[0]] * n
+            tot += st.primary_tokens
+        assert out["stats"].primary_tokens == tot
+        check_walk_against_trace(out, w.batch, w.L)
+    # the true beam sets of every level as the draft tree: one round, everything accepted, no token beyond plain decoding's
+    art = tiny.eng.decode(K, mode=2, trace=True)
+    beams = art["trace"]["beams"]
+    counts = (beams[:, :, :, 0] >= 0).sum(dim=2).to(torch.int32)
+    out = tiny.eng.decode_with_draft_tree(K, beams, counts, trace=True)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.allclose(out["scores"], art["scores"], atol=1e-5)
+    assert out["stats"].rounds == 1
+    assert out["stats"].primary_tokens == int(counts[: w.L - 1].sum())
+    tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+    for b in range(w.batch):
+        n = int(counts[w.L - 1, b])
+        assert list(tr["accepted_len"][0, b, :n]) == [w.L] * n and tr["level_reached"][0, b] == w.L
+    check_walk_against_trace(out, w.batch, w.L)
+    # repeated tuples and tuples with shared prefixes: one node per distinct prefix
+    dup = ar_codes.copy()
+    dup[:, 1] = dup[:, 0]
+    nd = torch.full((w.batch,), K, dtype=torch.int32, device="cuda")
+    out = tiny.eng.decode_with_drafts(K, torch.from_numpy(dup).cuda(), nd, trace=True)
+    assert torch.equal(out["codes"], ar["codes"])
+    tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+    for b in range(w.batch):
+        D = [tuple(int(c) for c in dup[b, k]) for k in range(K)]
+        assert list(tr["tree_count"][0, :, b]) == [len(x) for x in O.tree_from_tuples(D, w.L)]
+        got = [tuple(int(c) for c in tr["drafts"][0, b, k]) for k in range(tr["n_draft"][0, b])]
+        assert got == O.tree_from_tuples(D, w.L)[-1]
+    check_walk_against_trace(out, w.batch, w.L)
     # decode is repeatable from the same prefilled state
     again = tiny.eng.decode(K, mode=1)
     assert torch.equal(again["codes"], ar["codes"])

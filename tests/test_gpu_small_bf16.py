@@ -9,7 +9,7 @@ import torch
 
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
-from gpu_helpers import Case, assert_topk_matches, check_levels, tolerance
+from gpu_helpers import Case, assert_topk_matches, check_levels, check_walk_against_trace, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -72,6 +72,46 @@ def test_small_verified_decode_all_rows(small):
     for b in range(w.batch):
         check_levels(small, b, beams[:, b], scores[:, b], w.beam)
         assert np.array_equal(beams[w.L - 1, b], codes[b])
+    check_walk_against_trace(out, w.batch, w.L)
+
+
+def test_small_accept_and_roll_back_bookkeeping(small):
+    """Accepted lengths, rejection levels, rounds and token counts at beam 10, four levels, 64 requests: replayed with the
+    oracle's integer rules from the GPU's own beam sets and draft trees -- for the head's own drafts, for seeded
+    corruptions of the true tuples, and for the true beam sets themselves (one round, nothing beyond plain decoding's
+    tokens)."""
+    w = small.w
+    K, L = w.beam, w.L
+    art = small.eng.decode(K, mode=2, trace=True)
+    ar_codes = art["codes"].cpu().numpy()
+    rng = np.random.default_rng(17)
+    for rho in (0.0, 0.3, 1.0):
+        drafts = np.maximum(ar_codes, 0)
+        n_draft = art["count"].cpu().numpy().copy()
+        for b in range(w.batch):
+            for k in range(n_draft[b]):
+                if rng.random() < rho:
+                    lvl = int(rng.integers(0, L))
+                    drafts[b, k, lvl] = (drafts[b, k, lvl] + 1 + rng.integers(0, w.T[lvl] - 1)) % w.T[lvl]
+        out = small.eng.decode_with_drafts(K, torch.from_numpy(drafts).cuda(), torch.from_numpy(n_draft).cuda(), trace=True)
+        assert torch.equal(out["codes"], art["codes"]) and torch.allclose(out["scores"], art["scores"], atol=1e-4)
+        check_walk_against_trace(out, w.batch, L)
+        tr_tree = out["trace"]["tree_count"].cpu().numpy()
+        for b in range(w.batch):
+            D = [tuple(int(c) for c in drafts[b, k]) for k in range(n_draft[b])]
+            assert list(tr_tree[0, :, b]) == [len(x) for x in O.tree_from_tuples(D, L)]
+    beams = art["trace"]["beams"]
+    counts = (beams[:, :, :, 0] >= 0).sum(dim=2).to(torch.int32)
+    out = small.eng.decode_with_draft_tree(K, beams, counts, trace=True)
+    assert torch.equal(out["codes"], art["codes"]) and torch.allclose(out["scores"], art["scores"], atol=1e-4)
+    assert out["stats"].rounds == 1 and out["stats"].primary_tokens == int(counts[: L - 1].sum())
+    acc = out["trace"]["accepted_len"].cpu().numpy()
+    for b in range(w.batch):
+        n = int(counts[L - 1, b])
+        assert np.all(acc[0, b, :n] == L)
+    check_walk_against_trace(out, w.batch, L)
+    check_walk_against_trace(art, w.batch, L)                      # plain decoding: empty trees, L - 1 rounds
+    assert art["stats"].rounds == L - 1
 
 
 def test_small_draft_mode(small):
@@ -127,6 +167,7 @@ def test_bf16_shapes_ragged_histories(shape):
     scores = out["trace"]["beam_scores"].cpu().numpy()
     for b in range(w.batch):
         check_levels(case, b, beams[:, b], scores[:, b], w.beam)
+    check_walk_against_trace(out, w.batch, w.L)
 
 
 def test_paper_setting_three_levels_of_512_codes():
@@ -149,6 +190,7 @@ def test_paper_setting_three_levels_of_512_codes():
     codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
     live = np.arange(w.beam)[None, :] < count[:, None]
     assert V.contains(codes[live]).all()
+    check_walk_against_trace(out, w.batch, w.L)
 
 
 @pytest.mark.parametrize("name", ["tiny", "small"])
