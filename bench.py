@@ -1,14 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the speculative semantic-ID decode step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload small] [--mode 1] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--mode 1] [--impl ours|reference]
 
 One step = one nezha_decode call (draft head -> hash-set filter -> primary verify pass -> masked log-softmax /
 beam top-k -> accept / roll back, all rounds) over the whole batch, always from the same prefilled state.
 Prints ONE JSON line.  `value` = items (batch x beam) decoded per second with all inputs resident in HBM;
 `e2e` = the same through the C ABI starting from pinned HOST histories (H2D copy + prefill + decode + D2H of
-the results inside the timed region).  With N > 1 (torchrun) every rank runs an independent replica on its own
-GPU -- requests are independent, so there is no collective on the data path -- and `value` sums the replicas.
+the results inside the timed region).  With N > 1 every rank runs an independent replica on its own GPU -- requests are
+independent, so there is no collective on the data path -- and `value` sums the replicas (under torchrun, or started
+by this script itself when it is called with --gpus N and no launcher).  The default workload is the largest
+single-GPU configuration (the 7B shape); the default one-GPU run also times the other four configurations briefly and
+reports them under `per_workload`.
 """
 from __future__ import annotations
 
@@ -102,34 +105,6 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_sample(w, weights_np, catalog, hist, mode, budget_s=20.0, max_rows=None):
-    """The CPU oracle, as it stands, on the first rows of the workload until ~budget_s of work is done."""
-    import numpy as np
-    from oracle import nezha_oracle as O
-    shape = O.ModelShape(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.d_ffn, w.L, tuple(w.T), w.rope_theta, w.rms_eps)
-    big = w.d_model * w.d_ffn * w.n_layers > 2e8
-    model = O.PrimaryModel(shape, weights_np, cache_f64=not big)
-    head, valid = O.DraftHead(shape, weights_np), O.ValidSet(catalog, w.T)
-    rows, t_decode, t_prefill = 0, 0.0, 0.0
-    limit = hist.shape[0] if max_rows is None else min(max_rows, hist.shape[0])
-    while rows < limit and (t_decode + t_prefill) < budget_s:
-        t0 = time.perf_counter()
-        req = model.prefill(hist[rows])
-        t1 = time.perf_counter()
-        if mode == 0:
-            O.nezha_draft(head, req, w.beam, valid)
-        elif mode == 2:
-            O.ar_beam_search(model, req, w.beam, valid)
-        else:
-            O.speculative_decode(model, head, req, w.beam, valid)
-        t2 = time.perf_counter()
-        t_prefill += t1 - t0
-        t_decode += t2 - t1
-        rows += 1
-    return {"rows": rows, "decode_s": t_decode, "prefill_s": t_prefill,
-            "items_per_s": rows * w.beam / t_decode if t_decode > 0 else 0.0}
-
-
 def algorithmic_work(w, stats_tokens_per_step, rounds):
     """Algorithmic flops / bytes of one decode step, per kernel class.
 
@@ -196,131 +171,51 @@ def probe_bench(args, w, eng, cat_dev, config, dev):
                                    "algorithmic_bytes_per_key": 41}}))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="small")
-    ap.add_argument("--mode", type=int, default=1, help="0 draft-only, 1 verified (default), 2 plain autoregressive")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--drafts", default="natural", choices=["natural", "perfect"],
-                    help="mode 1 only: 'natural' = the (random-init) draft head's own drafts; 'perfect' = the true top-k "
-                         "tuples injected as round-1 drafts (best case: one round, everything accepted)")
-    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (requests per decode call)")
-    ap.add_argument("--final-mask", default="prefix", choices=["hash", "prefix"],
-                    help="how the primary model's last-level validity mask (Eq. 5) is answered: the prefix map (the "
-                         "library's default) or one hash-set probe per candidate code")
-    ap.add_argument("--probe-keys", type=int, default=0,
-                    help="instead of the decode step, time the stand-alone hash-set probe (Eq. 5) on this many keys, "
-                         "half of them catalogue items, and print its own JSON line")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-budget-s", type=float, default=20.0)
-    args = ap.parse_args()
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-
-    import numpy as np
+def build_engine(w, dev, final_mask: str):
+    """Weights, catalogue, histories and a prefilled engine for one workload; everything resident on the device."""
     import torch
-    from paper_2511_18793_b200 import synth
-
-    w = synth.WORKLOADS[args.workload]
-    if args.batch > 0:
-        w = synth.scaled(w, batch=args.batch)
-    config = {"workload": f"{w.name}: {w.n_layers}L d{w.d_model} {w.n_q_heads}q/{w.n_kv_heads}kv ffn{w.d_ffn}, "
-                          f"L={w.L} T={w.T[0]}, catalogue {w.n_items} ({w.catalog}), history {w.n_hist} items, "
-                          f"batch {w.batch} x beam {w.beam}, seed {w.seed}",
-              "mode": {0: "draft-only (Algorithm 3)", 1: "verified (Algorithm 2)", 2: "autoregressive (Algorithm 1)"}[args.mode],
-              "batch": w.batch, "beam": w.beam, "l2": "flushed between steps (256 MB write, outside the timed events)",
-              "drafts": "natural (random-init draft head)" if args.drafts == "natural" or args.mode != 1 else
-                        "perfect (the true top-k tuples injected as round-1 drafts)"}
-
-    # ------------------------------------------------------------------ reference arm: the oracle on host cores
-    if args.impl == "reference":
-        if rank != 0:
-            return
-        weights = synth.make_weights(w, device="cpu")
-        catalog = synth.make_catalog(w)
-        hist = synth.make_histories(w, catalog)
-        Wn = synth.weights_to_numpy(weights)
-        per_step = max(2.0, min(args.cpu_budget_s, 120.0 / max(1, args.steps + args.warmup)))
-        vals, rows = [], 0
-        for i in range(args.warmup + args.steps):
-            r = oracle_sample(w, Wn, catalog, hist, args.mode, budget_s=per_step, max_rows=4)
-            if i >= args.warmup:
-                vals.append(r["items_per_s"]); rows = r["rows"]
-        v = statistics.mean(vals)
-        cores = os.cpu_count()
-        print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
-                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * rows * w.beam / v if v else None,
-                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-                          "data": "synthetic", "config": config,
-                          "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                           "sample": f"decode of the first {rows} request(s) of the batch per step, prefill excluded"},
-                          "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
-        return
-
-    # ------------------------------------------------------------------ our arm
-    from paper_2511_18793_b200 import binding
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
-    torch.cuda.set_device(local_rank)
-    dev = f"cuda:{local_rank}"
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_
-        dist = dist_
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-
+    from paper_2511_18793_b200 import binding, synth
     weights = synth.make_weights(w, device=dev)
     catalog = synth.make_catalog(w)
     hist = synth.make_histories(w, catalog)
     cat_dev = torch.from_numpy(catalog).to(dev)
-    # a stream of its own (not the legacy default stream), so that the library may capture its rounds into CUDA graphs;
-    # made current, so that the flushes, copies and timing events below are ordered on it too
-    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
     eng = binding.Engine(binding.make_config(w), weights, cat_dev, w.load_factor, stream=torch.cuda.current_stream())
     n_unique = eng.build_hashset()
     assert n_unique == w.n_items
-    if args.probe_keys > 0:
-        probe_bench(args, w, eng, cat_dev, config, dev)
-        return
-    eng.set_option(binding.OPT_FINAL_MASK, 1 if args.final_mask == "prefix" else 0)
-    config["final_mask"] = "prefix map (one look-up per beam)" if args.final_mask == "prefix" else "hash-set probes"
-    hist_pinned = torch.from_numpy(hist).pin_memory()
+    eng.set_option(binding.OPT_FINAL_MASK, 1 if final_mask == "prefix" else 0)
+    return {"w": w, "weights": weights, "catalog": catalog, "hist": hist, "cat_dev": cat_dev, "eng": eng}
+
+
+def time_decode(ctx, mode, drafts, steps, warmup, flush, dist, world, dev, barrier):
+    """W warm-up steps, then K timed steps (one CUDA-event pair per step, L2 flushed before each, outside the events);
+    then the per-class pass.  Returns the numbers of one workload."""
+    import torch
+    from paper_2511_18793_b200 import binding
+    w, eng = ctx["w"], ctx["eng"]
+    hist_pinned = torch.from_numpy(ctx["hist"]).pin_memory()
     nh_pinned = torch.full((w.batch,), w.n_hist, dtype=torch.int32).pin_memory()
     hist_dev = hist_pinned.to(dev, non_blocking=True)
     nh_dev = nh_pinned.to(dev, non_blocking=True)
     eng.prefill(hist_dev, nh_dev)
     out = eng.alloc_outputs(w.batch, w.beam)
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
     items = w.batch * w.beam
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
     inject = None
-    if args.drafts == "perfect" and args.mode == 1:
-        ar = eng.decode(w.beam, mode=2)
-        inject = (ar["codes"].clone().clamp_(min=0), ar["count"].clone())
+    if drafts == "perfect" and mode == 1:
+        art = eng.decode(w.beam, mode=2, trace=True)
+        beams = art["trace"]["beams"].clone()
+        inject = (beams, (beams[:, :, :, 0] >= 0).sum(dim=2).to(torch.int32).contiguous())
 
     def step():
         if inject is not None:
-            return eng.decode_with_drafts(w.beam, inject[0], inject[1], out=out)
-        return eng.decode(w.beam, mode=args.mode, out=out)
+            return eng.decode_with_draft_tree(w.beam, inject[0], inject[1], out=out)
+        return eng.decode(w.beam, mode=mode, out=out)
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         flush.fill_(1)
         step()
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     launches0 = binding.lib.nezha_launch_count()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     tokens = rounds = 0
     for a, b in evs:
         flush.fill_(1)
@@ -331,46 +226,13 @@ def main():
         rounds += r["stats"].rounds
     barrier()
     launches = binding.lib.nezha_launch_count() - launches0
-    clocks = sampler.stop()
     per_step_ms = [a.elapsed_time(b) for a, b in evs]
-    total_ms = sum(per_step_ms)
-    value, total_ms_max = whole_job_throughput(dist, total_ms, items, args.steps, world, dev)
-
-    # ---- end to end from pinned host memory: H2D histories, prefill, decode, D2H results
-    host_codes = torch.empty(w.batch, w.beam, w.L, dtype=torch.int32).pin_memory()
-    host_scores = torch.empty(w.batch, w.beam, dtype=torch.float32).pin_memory()
-    host_count = torch.empty(w.batch, dtype=torch.int32).pin_memory()
-    e2e_steps = max(3, min(args.steps, 10))
-
-    def e2e_step():
-        hd = hist_pinned.to(dev, non_blocking=True)
-        nd = nh_pinned.to(dev, non_blocking=True)
-        eng.prefill(hd, nd)
-        step()
-        host_codes.copy_(out["codes"], non_blocking=True)
-        host_scores.copy_(out["scores"], non_blocking=True)
-        host_count.copy_(out["count"], non_blocking=True)
-        torch.cuda.synchronize()
-
-    e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ea.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    eb.record()
-    barrier()
-    e2e_ms = max(ea.elapsed_time(eb), 0.0)
-    e2e_value, e2e_ms_max = whole_job_throughput(dist, e2e_ms, items, e2e_steps, world, dev)
-    h2d = hist_pinned.numel() * 4 + nh_pinned.numel() * 4
-    d2h = host_codes.numel() * 4 + host_scores.numel() * 4 + host_count.numel() * 4
+    value, total_ms_max = whole_job_throughput(dist, sum(per_step_ms), items, steps, world, dev)
 
     # ---- per-kernel-class CUDA-event timing (separate pass: two event records per launch perturb throughput)
-    eng.prefill(hist_dev, nh_dev)
     eng.profile_enable(True)
     eng.profile_read()
-    prof_steps = max(3, min(args.steps, 10))
+    prof_steps = max(3, min(steps, 10))
     ptok = prd = 0
     for _ in range(prof_steps):
         flush.fill_(1)
@@ -390,7 +252,8 @@ def main():
     dom_s = shares[dom]["ms_per_step"] / 1e3
     if dom == "gemm":
         ach = work["gemm_flops"] / dom_s / 1e12
-        peak = peaks["bf16_tflops_sustained"] if w.dtype == "bf16" else 75.0
+        # fp32 workload: CUDA-core FMA peak = 148 SMs x 128 FMA lanes x 2 flops x 1.965 GHz = 74.4 TFLOP/s
+        peak = peaks["bf16_tflops_sustained"] if w.dtype == "bf16" else 148 * 128 * 2 * 1.965e9 / 1e12
         roof.update(bound="tensor" if w.dtype == "bf16" else "alu", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
     elif dom == "attention":
         ach = work["attention_bytes"] / dom_s / 1e9
@@ -405,37 +268,279 @@ def main():
         roof["traffic_source"] = rec["source"]
     # the whole step against its floor: per class the larger of (bytes / copy bandwidth) and (flops / tensor peak),
     # summed over the GEMM and attention classes (the rest moves kilobytes), divided by the measured step time
-    if w.dtype == "bf16" and args.mode != 0:
+    if w.dtype == "bf16" and mode != 0:
         tf, bw = peaks["bf16_tflops_sustained"] * 1e12, peaks["hbm_gbs"] * 1e9
         floor_s = max(work["gemm_flops"] / tf, work["gemm_weight_bytes"] / bw) + \
             max(work["attention_flops"] / tf, work["attention_bytes"] / bw)
         roof["step_floor_ms"] = floor_s * 1e3
-        roof["step_frac"] = floor_s * 1e3 / (total_ms_max / args.steps)
+        roof["step_frac"] = floor_s * 1e3 / (total_ms_max / steps)
     roof["classes"] = shares
     roof["attention_gbs"] = work["attention_bytes"] / (shares["attention"]["ms_per_step"] / 1e3) / 1e9 if "attention" in shares else None
+    roof["attention_tflops"] = work["attention_flops"] / (shares["attention"]["ms_per_step"] / 1e3) / 1e12 if "attention" in shares else None
     roof["gemm_tflops"] = work["gemm_flops"] / (shares["gemm"]["ms_per_step"] / 1e3) / 1e12 if "gemm" in shares else None
+    return {"value": value, "ms_per_step": total_ms_max / steps, "p50_ms": statistics.median(per_step_ms),
+            "launches": int(launches), "rounds_per_step": rounds / steps, "primary_tokens_per_step": tokens / steps,
+            "roofline": roof, "step": step, "out": out, "hist_pinned": hist_pinned, "nh_pinned": nh_pinned}
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": total_ms_max / args.steps, "p50_ms": statistics.median(per_step_ms),
+
+def workload_label(w):
+    return (f"{w.name}: {w.n_layers}L d{w.d_model} {w.n_q_heads}q/{w.n_kv_heads}kv ffn{w.d_ffn}, "
+            f"L={w.L} T={w.T[0]}, catalogue {w.n_items} ({w.catalog}), history {w.n_hist} items, "
+            f"batch {w.batch} x beam {w.beam}, seed {w.seed}")
+
+
+def reference_arm(args, w, config):
+    """The CPU oracle as it stands on the host cores.  One step = the decode of ONE request of the workload (the first of
+    the batch), from its prefilled state; the prefill is computed once before the loop and excluded, as in our arm."""
+    import numpy as np
+    from oracle import nezha_oracle as O
+    from paper_2511_18793_b200 import synth
+    weights = synth.make_weights(w, device="cpu")
+    catalog = synth.make_catalog(w)
+    hist = synth.make_histories(w, catalog, batch=1)
+    Wn = synth.weights_to_numpy(weights)
+    del weights
+    shape = O.ModelShape(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.d_ffn, w.L, tuple(w.T), w.rope_theta, w.rms_eps)
+    big = w.d_model * w.d_ffn * w.n_layers > 2e8
+    # multi-billion-parameter shapes: the oracle's fp32 arithmetic option (its fp64 default would convert 20 GB of weights
+    # on every call); everything else as it stands
+    odt = np.float32 if big else np.float64
+    model = O.PrimaryModel(shape, Wn, cache_f64=not big, dtype=odt)
+    head, valid = O.DraftHead(shape, Wn), O.ValidSet(catalog, w.T)
+    req = model.prefill(hist[0])
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        if args.mode == 0:
+            O.nezha_draft(head, req, w.beam, valid)
+        elif args.mode == 2:
+            O.ar_beam_search(model, req, w.beam, valid)
+        else:
+            O.speculative_decode(model, head, req, w.beam, valid)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    ms = 1e3 * sum(times) / len(times)
+    v = w.beam / (ms / 1e3)
+    try:
+        import torch
+        threads = torch.get_num_threads()
+    except Exception:
+        threads = os.cpu_count()
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                      "dtype": "f32" if big else "f64", "data": "synthetic", "config": config,
+                      "cpu_baseline": {"value": v, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                       "sample": "decode of one request (the first of the batch, beam as configured) per "
+                                                 "step; its prefill computed once before the loop and excluded",
+                                       "blas_threads": threads},
+                      "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def relaunch_replicas(args):
+    """`--gpus N` without a launcher: start N replica processes, one per GPU, the way the launcher would."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.exit(subprocess.call(cmd))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="7b",
+                    help="7b (default: the largest single-GPU configuration), 1.5b, 0.5b, small, tiny, paper")
+    ap.add_argument("--mode", type=int, default=1, help="0 draft-only, 1 verified (default), 2 plain autoregressive")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--drafts", default="natural", choices=["natural", "perfect"],
+                    help="mode 1 only: 'natural' = the (random-init) draft head's own draft tree; 'perfect' = the true beam "
+                         "sets of every level injected as round 1's draft tree (best case: one round, everything accepted)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (requests per decode call)")
+    ap.add_argument("--final-mask", default="prefix", choices=["hash", "prefix"],
+                    help="how the primary model's last-level validity mask (Eq. 5) is answered: the prefix map (the "
+                         "library's default) or one hash-set probe per candidate code")
+    ap.add_argument("--probe-keys", type=int, default=0,
+                    help="instead of the decode step, time the stand-alone hash-set probe (Eq. 5) on this many keys, "
+                         "half of them catalogue items, and print its own JSON line")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the short runs of the other configurations that the default run adds under `per_workload`")
+    ap.add_argument("--cpu-budget-s", type=float, default=20.0)
+    args = ap.parse_args()
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        relaunch_replicas(args)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import numpy as np
+    import torch
+    from paper_2511_18793_b200 import synth
+
+    w = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = synth.scaled(w, batch=args.batch)
+    config = {"workload": workload_label(w),
+              "mode": {0: "draft-only (Algorithm 3)", 1: "verified (Algorithm 2)", 2: "autoregressive (Algorithm 1)"}[args.mode],
+              "batch": w.batch, "beam": w.beam, "l2": "flushed between steps (256 MB write, outside the timed events)",
+              "drafts": "natural (random-init draft head)" if args.drafts == "natural" or args.mode != 1 else
+                        "perfect (the true beam sets injected as round 1's draft tree)"}
+
+    # ------------------------------------------------------------------ reference arm: the oracle on host cores
+    if args.impl == "reference":
+        if rank == 0:
+            reference_arm(args, w, config)
+        return
+
+    # ------------------------------------------------------------------ our arm
+    from paper_2511_18793_b200 import binding
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    # a stream of its own (not the legacy default stream), so that the library may capture its rounds into CUDA graphs;
+    # made current, so that the flushes, copies and timing events below are ordered on it too
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
+    ctx = build_engine(w, dev, args.final_mask)
+    eng = ctx["eng"]
+    if args.probe_keys > 0:
+        probe_bench(args, w, eng, ctx["cat_dev"], config, dev)
+        return
+    config["final_mask"] = "prefix map (one look-up per beam)" if args.final_mask == "prefix" else "hash-set probes"
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    items = w.batch * w.beam
+    warmup = max(args.warmup, 3)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    res = time_decode(ctx, args.mode, args.drafts, args.steps, warmup, flush, dist, world, dev, barrier)
+    clocks = sampler.stop()
+    step, out, hist_pinned, nh_pinned = res["step"], res["out"], res["hist_pinned"], res["nh_pinned"]
+
+    # ---- end to end from pinned host memory: H2D histories, prefill, decode, D2H results
+    host_codes = torch.empty(w.batch, w.beam, w.L, dtype=torch.int32).pin_memory()
+    host_scores = torch.empty(w.batch, w.beam, dtype=torch.float32).pin_memory()
+    host_count = torch.empty(w.batch, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        hd = hist_pinned.to(dev, non_blocking=True)
+        nd = nh_pinned.to(dev, non_blocking=True)
+        eng.prefill(hd, nd)
+        step()
+        host_codes.copy_(out["codes"], non_blocking=True)
+        host_scores.copy_(out["scores"], non_blocking=True)
+        host_count.copy_(out["count"], non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record()
+    barrier()
+    e2e_ms = max(ea.elapsed_time(eb), 0.0)
+    e2e_value, e2e_ms_max = whole_job_throughput(dist, e2e_ms, items, e2e_steps, world, dev)
+    h2d = hist_pinned.numel() * 4 + nh_pinned.numel() * 4
+    d2h = host_codes.numel() * 4 + host_scores.numel() * 4 + host_count.numel() * 4
+
+    line = {"metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": res["ms_per_step"], "p50_ms": res["p50_ms"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
-            "clocks": clocks, "gpu_launches": int(launches),
-            "rounds_per_step": rounds / args.steps, "primary_tokens_per_step": tokens / args.steps,
+            "clocks": clocks, "gpu_launches": res["launches"],
+            "rounds_per_step": res["rounds_per_step"], "primary_tokens_per_step": res["primary_tokens_per_step"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "includes": "H2D histories + prefill + decode + D2H results", "steps": e2e_steps,
                     "ms_per_step": e2e_ms_max / e2e_steps},
-            "roofline": roof}
+            "roofline": res["roofline"]}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        Wn = synth.weights_to_numpy(weights)
-        r = oracle_sample(w, Wn, catalog, hist, args.mode, budget_s=args.cpu_budget_s)
-        line["cpu_baseline"] = {"value": r["items_per_s"], "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                                "sample": f"decode of the first {r['rows']} request(s) of the batch "
-                                          f"({r['decode_s']:.1f} s; their prefill, {r['prefill_s']:.1f} s, excluded)"}
+        line["cpu_baseline"] = cpu_baseline(ctx, args)
+
+    # ---- the other configurations, briefly (one GPU, default run only): same step, fewer repetitions
+    if world == 1 and not args.no_per_workload and args.workload == "7b" and args.batch == 0:
+        per = {}
+        del res, step, out
+        ctx.clear(); eng.close(); del eng
+        torch.cuda.empty_cache()
+        for name in ("tiny", "small", "0.5b", "1.5b"):
+            wn = synth.WORKLOADS[name]
+            c2 = build_engine(wn, dev, args.final_mask)
+            entry = {"workload": workload_label(wn)}
+            for label, mode, drafts in (("verified", 1, "natural"), ("verified_perfect_tree", 1, "perfect"),
+                                        ("autoregressive", 2, "natural"), ("draft_only", 0, "natural")):
+                r2 = time_decode(c2, mode, drafts, 10, 3, flush, None, 1, dev, barrier)
+                rf = r2["roofline"]
+                entry[label] = {"value": r2["value"], "ms_per_step": r2["ms_per_step"], "p50_ms": r2["p50_ms"],
+                                "rounds_per_step": r2["rounds_per_step"],
+                                "primary_tokens_per_step": r2["primary_tokens_per_step"], "launches_per_step": r2["launches"] / 10,
+                                "dominant": rf["kernel"], "bound": rf["bound"], "frac": rf["frac"],
+                                "step_frac": rf.get("step_frac"), "gemm_tflops": rf.get("gemm_tflops"),
+                                "attention_gbs": rf.get("attention_gbs")}
+                del r2
+            per[name] = entry
+            c2["eng"].close(); c2.clear()
+            torch.cuda.empty_cache()
+        line["per_workload"] = per
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def cpu_baseline(ctx, args):
+    """The oracle as it stands on the host cores, on a bounded sample of the same workload: the decode of its first
+    request(s) until about `--cpu-budget-s` seconds of decode work are done (at least one request); prefill excluded."""
+    import numpy as np
+    import torch
+    from oracle import nezha_oracle as O
+    from paper_2511_18793_b200 import synth
+    w = ctx["w"]
+    Wn = synth.weights_to_numpy(ctx["weights"])
+    shape = O.ModelShape(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.d_ffn, w.L, tuple(w.T), w.rope_theta, w.rms_eps)
+    big = w.d_model * w.d_ffn * w.n_layers > 2e8
+    model = O.PrimaryModel(shape, Wn, cache_f64=not big, dtype=np.float32 if big else np.float64)
+    head, valid = O.DraftHead(shape, Wn), O.ValidSet(ctx["catalog"], w.T)
+    rows, t_decode, t_prefill = 0, 0.0, 0.0
+    while rows < w.batch and t_decode < args.cpu_budget_s:
+        t0 = time.perf_counter()
+        req = model.prefill(ctx["hist"][rows])
+        t1 = time.perf_counter()
+        if args.mode == 0:
+            O.nezha_draft(head, req, w.beam, valid)
+        elif args.mode == 2:
+            O.ar_beam_search(model, req, w.beam, valid)
+        else:
+            O.speculative_decode(model, head, req, w.beam, valid)
+        t2 = time.perf_counter()
+        t_prefill += t1 - t0
+        t_decode += t2 - t1
+        rows += 1
+    return {"value": rows * w.beam / t_decode if t_decode > 0 else 0.0, "unit": UNIT, "cores": os.cpu_count(),
+            "kind": "oracle", "blas_threads": torch.get_num_threads(),
+            "arithmetic": "fp32 option of the oracle (multi-billion-parameter shape)" if big else "fp64",
+            "sample": f"decode of the first {rows} request(s) of the batch ({t_decode:.1f} s; their prefill, "
+                      f"{t_prefill:.1f} s, excluded)"}
 
 
 if __name__ == "__main__":

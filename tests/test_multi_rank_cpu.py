@@ -48,3 +48,22 @@ def test_single_rank_needs_no_process_group():
     import bench
     value, worst = bench.whole_job_throughput(None, 50.0, 640, 5, 1)
     assert worst == 50.0 and abs(value - 640 * 5 / 0.05) < 1e-9
+
+
+def test_gpus_flag_without_a_launcher_starts_one_replica_per_gpu(monkeypatch):
+    """`python bench.py --gpus 4` with no WORLD_SIZE in the environment must start 4 ranks itself (one per GPU, rendezvous
+    on 127.0.0.1), not run one replica and call it four."""
+    sys.path.insert(0, ROOT)
+    import argparse
+    import bench
+    seen = {}
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(bench.sys, "argv", ["bench.py", "--gpus", "4", "--steps", "3"])
+    try:
+        bench.relaunch_replicas(argparse.Namespace(gpus=4))
+    except SystemExit as e:
+        assert e.code == 0
+    cmd = seen["cmd"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "3"] and cmd[-5].endswith("bench.py")
