@@ -195,11 +195,18 @@ nezha_status nezha_decode_with_draft_tree(nezha_ctx* ctx, int32_t batch, int32_t
  *                                  look-up per beam instead of T_L probes, the same answers bit for bit (the set V of
  *                                  Eq. 5 regrouped by prefix; the paper itself only describes the hash set)
  *                               The draft head's K chosen codes per beam (Algorithm 3) are always probed in the hash set.
+ *   NEZHA_OPT_LEVEL_FILTER      0 (default): the validity filter acts at the last level only, as Algorithm 3 prints it
+ *                               1: at every level (the per-step variant Section 3.4 mentions): a partial ID survives only
+ *                                  if some valid ID begins with it -- in the draft head's search (after its per-beam top-K,
+ *                                  unless NEZHA_OPT_DRAFT_FILTER is 0) and in the primary model's beam search of modes 1 and 2
+ *                                  (before the top-K).  Answered by the same table as NEZHA_OPT_FINAL_MASK 1, which holds the
+ *                                  prefixes of every length.  Modes 1 and 2 still agree item for item.
  * Errors: NEZHA_ERR_ARG (unknown option or value). */
 #define NEZHA_OPT_DRAFT_TRANSITION 0
 #define NEZHA_OPT_DRAFT_INPUTS 1
 #define NEZHA_OPT_DRAFT_FILTER 2
 #define NEZHA_OPT_FINAL_MASK 3
+#define NEZHA_OPT_LEVEL_FILTER 4
 nezha_status nezha_set_option(nezha_ctx* ctx, int32_t option, int32_t value);
 
 /* ---- stage-wise entry points (the same kernels as nezha_decode, one step at a time) ------------------- */
@@ -221,9 +228,9 @@ nezha_status nezha_draft_logits(nezha_ctx* ctx, int32_t batch, int32_t n_beams, 
                                 const int32_t* prefixes, float* logits);
 
 /* One beam-search level (the top-K, union and pruning steps of Algorithm 1 / Algorithm 3) on caller-supplied logits:
- * log-softmax over the codebook, per-beam top `per_beam` codes, optional hash-set filter of the resulting
- * tuples (only meaningful when level + 1 == L), top beam_width by cumulative log-probability; ties go to the
- * smaller (parent rank, code).
+ * log-softmax over the codebook, per-beam top `per_beam` codes, optional validity filter of the resulting tuples (at
+ * level + 1 == L: Eq. 5 in the hash set; at an earlier level: "some valid ID begins with it", from the prefix map), top
+ * beam_width by cumulative log-probability; ties go to the smaller (parent rank, code).
  *   logits [batch, n_beams, T[level]] float, beam_scores [batch, n_beams] float,
  *   beam_codes [batch, n_beams, level] int32, n_live [batch] int32 (beams in use per row)      -- device
  *   out_parent, out_code [batch, beam_width] int32 (-1 padded), out_score [batch, beam_width] float (-inf

@@ -81,6 +81,7 @@ class ValidSet:
     def __init__(self, catalog_codes: np.ndarray, T: Sequence[int]):
         self.T = tuple(int(t) for t in T)
         self.keys = np.unique(pack_keys(catalog_codes, self.T))
+        self._prefix: Dict[int, np.ndarray] = {}
 
     def __len__(self) -> int:
         return int(self.keys.size)
@@ -93,6 +94,24 @@ class ValidSet:
 
     def contains(self, codes: np.ndarray) -> np.ndarray:
         return self.contains_keys(pack_keys(codes, self.T))
+
+    def prefix_keys(self, n: int) -> np.ndarray:
+        """The sorted packed keys of the distinct n-code prefixes of the valid IDs.  Level 1 is the least significant digit
+        of Eq. 4, so the key of an ID's first n codes is its own key modulo prod_{j<=n} T_j."""
+        if n not in self._prefix:
+            self._prefix[n] = np.unique(self.keys % np.uint64(int(np.prod([int(t) for t in self.T[:n]], dtype=object))))
+        return self._prefix[n]
+
+    def contains_prefix(self, codes: np.ndarray) -> np.ndarray:
+        """Is each code tuple [..., n] (n <= L) the beginning of at least one valid ID?  (n = L: Eq. 5 itself.)"""
+        codes = np.asarray(codes)
+        n = codes.shape[-1]
+        if n == len(self.T):
+            return self.contains(codes)
+        table = self.prefix_keys(n)
+        keys = pack_keys(codes, self.T[:n])
+        pos = np.minimum(np.searchsorted(table, keys), table.size - 1)
+        return table[pos] == keys
 
 
 # ----------------------------------------------------------------------------------------------------
@@ -343,6 +362,8 @@ def expand_level(beams: List[Beam], logits: List[np.ndarray], K: int, per_beam: 
 
     per_beam = K is the draft-head setting of Algorithm 3 (K x K candidates before the filter); per_beam = T_l
     applies the filter to every extension before the top-K (top-k restricted to valid tuples).
+    The paper verifies at the last level only; the per-step variant it mentions (verification at every level, Section 3.4)
+    passes `valid` at the earlier levels too, where a partial ID counts as valid if some valid ID begins with it.
     """
     cands: List[Tuple[np.float32, int, int]] = []
     for r, beam in enumerate(beams):
@@ -352,7 +373,7 @@ def expand_level(beams: List[Beam], logits: List[np.ndarray], K: int, per_beam: 
             cands.append((_extend_score(beam.score, float(logp[t])), r, t))
     if valid is not None and cands:
         tuples = np.asarray([beams[r].codes + (t,) for _, r, t in cands], dtype=np.int64)
-        ok = valid.contains(tuples)
+        ok = valid.contains_prefix(tuples)               # full-length tuples: Eq. 5; shorter ones: prefix of a valid ID
         cands = [c for c, keep in zip(cands, ok) if keep]
     return [Beam(beams[r].codes + (t,), sc, r) for sc, r, t in _keep_best(cands, K)]
 
@@ -370,7 +391,7 @@ def teacher_forced_state(head: DraftHead, req: Request, codes: Sequence[int]) ->
 
 
 def nezha_draft(head: DraftHead, req: Request, K: int, valid: Optional[ValidSet],
-                start: Optional[List[Beam]] = None) -> List[List[Beam]]:
+                start: Optional[List[Beam]] = None, every_level: bool = False) -> List[List[Beam]]:
     """Algorithm 3, inference after the prefill.  Returns the beam sets of every level reached (last entry = final drafts).
 
     start = None is the paper's inference from the empty beam.  Otherwise drafting continues from the given
@@ -390,7 +411,7 @@ def nezha_draft(head: DraftHead, req: Request, K: int, valid: Optional[ValidSet]
             continue
         logits = [head.logits(l, req.h[l + 1], st) for st in states]
         per_beam = min(K, head.s.T[l])
-        nxt = expand_level(beams, logits, K, per_beam, valid if l == L - 1 else None)
+        nxt = expand_level(beams, logits, K, per_beam, valid if (l == L - 1 or every_level) else None)
         states = [head.transition(l, states[b.parent], b.codes[-1]) for b in nxt] if l < L - 1 else []
         beams = nxt
         levels.append(beams)
@@ -401,14 +422,15 @@ def nezha_draft(head: DraftHead, req: Request, K: int, valid: Optional[ValidSet]
 # Algorithm 1: plain autoregressive beam search of M_p under the same validity filter
 # ----------------------------------------------------------------------------------------------------
 
-def ar_beam_search(model: PrimaryModel, req: Request, K: int, valid: Optional[ValidSet]) -> List[List[Beam]]:
-    """Returns [B_1, ..., B_L]; B_L is the result."""
+def ar_beam_search(model: PrimaryModel, req: Request, K: int, valid: Optional[ValidSet],
+                   every_level: bool = False) -> List[List[Beam]]:
+    """Returns [B_1, ..., B_L]; B_L is the result.  every_level: the validity filter at every level (prefixes of valid IDs)."""
     s = model.s
     beams = [Beam((), np.float32(0.0))]
     out = []
     for l in range(s.L):
         logits = model.next_level_logits_many(req, [b.codes for b in beams])
-        beams = expand_level(beams, logits, K, s.T[l], valid if l == s.L - 1 else None)
+        beams = expand_level(beams, logits, K, s.T[l], valid if (l == s.L - 1 or every_level) else None)
         out.append(beams)
     return out
 
@@ -489,7 +511,7 @@ def accepted_lengths(tuples: Sequence[Tuple[int, ...]], true_sets: List[List[Bea
 def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: int, valid: Optional[ValidSet],
                        drafts_round1: Optional[List[Tuple[int, ...]]] = None,
                        draft_tree_round1: Optional[List[List[Tuple[int, ...]]]] = None,
-                       use_drafts: bool = True) -> Tuple[List[List[Beam]], SpecStats]:
+                       use_drafts: bool = True, every_level: bool = False) -> Tuple[List[List[Beam]], SpecStats]:
     """Algorithm 2 with the readings listed in the module header.
 
     B_1 comes from the prefill hidden state h_0.  Each round, with m levels settled (true beams B_m):
@@ -505,14 +527,15 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
         round ends there and m <- that level.
       * accepted length of a drafted tuple = the largest i <= (level reached) whose i-prefix is a beam of B_i.
     Every B_j is computed from M_p's logits only, so the result equals ar_beam_search whatever the drafts.
-    use_drafts=False gives L-1 rounds of plain autoregressive steps.
+    use_drafts=False gives L-1 rounds of plain autoregressive steps.  every_level: the validity filter at every level,
+    in the draft head's search and in the primary model's alike.
     """
     s = model.s
     L = s.L
     stats = SpecStats()
     true_sets: List[List[Beam]] = []
     B = expand_level([Beam((), np.float32(0.0))], [model.next_level_logits(req, ())], K, s.T[0],
-                     valid if L == 1 else None)
+                     valid if (L == 1 or every_level) else None)
     true_sets.append(B)
     m = 1
     while m < L:
@@ -526,16 +549,16 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
         elif stats.rounds == 1 and drafts_round1 is not None:
             tree = tree_from_tuples(drafts_round1, L)
         elif stats.rounds == 1:
-            tree = [[b.codes for b in lv] for lv in nezha_draft(head, req, K, valid)]
+            tree = [[b.codes for b in lv] for lv in nezha_draft(head, req, K, valid, every_level=every_level)]
         else:
-            lv = nezha_draft(head, req, K, valid, start=B)                  # levels m+1 .. L
+            lv = nezha_draft(head, req, K, valid, start=B, every_level=every_level)   # levels m+1 .. L
             tree[m - 1] = [b.codes for b in B]
             for i, beams in enumerate(lv):
                 tree[m + i] = [b.codes for b in beams]
         # ---- the parallel verification pass, progressive selection / rejection (Algorithm 2, rejection and update steps)
         def next_beams(beams: List[Beam], j: int) -> List[Beam]:
             logits = model.next_level_logits_many(req, [b.codes for b in beams])
-            return expand_level(beams, logits, K, s.T[j], valid if j + 1 == L else None)
+            return expand_level(beams, logits, K, s.T[j], valid if (j + 1 == L or every_level) else None)
         new_sets, nodes = verification_walk(tree, B, m, L, next_beams)
         true_sets.extend(new_sets)                       # true_sets[i - 1] is B_i
         B = true_sets[-1]

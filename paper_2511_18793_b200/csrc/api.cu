@@ -89,6 +89,7 @@ struct nezha_ctx {
   bool use_graphs;
   int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
   int opt_mask;             // nezha_set_option: 0 = the primary model's last-level mask probes the hash set, 1 (default) = it reads the prefix map
+  int opt_level_filter;     // nezha_set_option: 1 = validity filter at every level (prefixes of valid IDs), 0 (default) = last level only
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
   int chains_now;           // GemmArgs::chains of the products being queued: 2 inside a decode call, 0 otherwise
@@ -176,12 +177,21 @@ size_t carve(nezha_ctx* c) {
   c->n_unique_dev = cv.take<unsigned long long>(1);
   e.hs.n_buckets = bucket_count(c->n_items, c->load_factor);
   e.hs.slots = cv.take<unsigned long long>(e.hs.n_buckets * kBucketSlots);
-  {  // prefix map: at most one slot per item and per possible prefix, at the hash set's load factor
+  {  // prefix map: for every prefix length n < L at most one slot per item and per possible prefix, at the hash set's
+     // load factor; slots hold the bit set of the widest codebook
+    const double items = (double)(c->n_items ? c->n_items : 1);
     double prefixes = 1.0;
-    for (int l = 0; l + 1 < g.L; ++l) prefixes *= (double)g.T[l];
-    const double n_pref = prefixes < (double)(c->n_items ? c->n_items : 1) ? prefixes : (double)(c->n_items ? c->n_items : 1);
-    e.pm.n_slots = (unsigned long long)ceil(n_pref / c->load_factor) + 1;
-    int words = 1 + (g.T[g.L - 1] + 63) / 64, stride = 2;
+    unsigned long long total = 0;
+    for (int n = 0; n < g.L; ++n) {
+      if (n > 0) prefixes *= (double)g.T[n - 1];
+      const double n_pref = prefixes < items ? prefixes : items;
+      e.pm.level_off[n] = total;
+      e.pm.level_slots[n] = (unsigned long long)ceil(n_pref / c->load_factor) + 1;
+      total += e.pm.level_slots[n];
+    }
+    for (int n = g.L; n < kMaxLevels; ++n) { e.pm.level_off[n] = 0; e.pm.level_slots[n] = 0; }
+    e.pm.n_slots = total;
+    int words = 1 + (c->Tmax + 63) / 64, stride = 2;
     while (stride < words) stride *= 2;
     e.pm.stride = stride;
     e.pm.slots = cv.take<unsigned long long>(e.pm.n_slots * (unsigned long long)stride);
@@ -424,7 +434,7 @@ SelectArgs select_base(nezha_ctx* c, int batch, int K) {
   SelectArgs s{};
   s.in_stride = c->Kmax; s.out_stride = c->Kmax; s.K = K; s.tuple_len = c->L; s.batch = batch;
   s.li = c->es.li; s.hs = c->es.hs;
-  if (c->opt_mask == 1) s.pm = c->es.pm;
+  s.pm = c->es.pm; s.final_mask_from_map = c->opt_mask;
   return s;
 }
 
@@ -464,6 +474,7 @@ void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_le
       }
       s.in_codes = e.dw_codes + lv_in * c->L; s.in_score = e.dw_score + lv_in; s.in_count = e.dw_count + (size_t)(l - 1) * c->Bmax;
       s.n = l - 1; s.T = c->cfg.T[l - 1]; s.per_beam = K < s.T ? K : s.T; s.filter = (filter && l == c->L) ? 1 : 0;
+      s.prefix_filter = (filter && c->opt_level_filter && l < c->L) ? 1 : 0;
       s.gate = e.d_m; s.gate_mode = 2; s.gate_value = l;
       s.out_codes = e.dw_codes + lv_out * c->L; s.out_score = e.dw_score + lv_out; s.out_parent = e.dw_parent + lv_out;
       s.out_token = nullptr; s.out_count = e.dw_count + (size_t)l * c->Bmax;
@@ -548,7 +559,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
   const int R = L - 1;
   auto key_of = [&](int segment) {
     std::array<uintptr_t, 16> k{};
-    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20 | (is_tree ? 1 : 0) << 24);
+    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20 | (is_tree ? 1 : 0) << 24 | c->opt_level_filter << 25);
     k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
     k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
     k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams ^ ((uintptr_t)tr.tree_codes << 1);
@@ -582,6 +593,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     s.logits = c->logits0; s.row_stride = c->cfg.T[0]; s.col_off = 0; s.src_row = nullptr; s.src_mul = 1;
     s.in_codes = e.tb_codes; s.in_score = e.tb_score; s.in_count = e.tb_count; s.n = 0; s.T = c->cfg.T[0];
     s.per_beam = s.T; s.filter = (L == 1) ? 1 : 0; s.gate_mode = 0;
+    s.prefix_filter = (c->opt_level_filter && L > 1) ? 1 : 0;
     s.out_codes = e.tb_codes + lv_out * L; s.out_score = e.tb_score + lv_out; s.out_parent = e.tb_parent + lv_out;
     s.out_count = e.tb_count + (size_t)1 * c->Bmax;
     launch_select(s, c->st);
@@ -612,6 +624,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
         s.src_row = e.tb_src + lv_in; s.src_mul = 0;
         s.in_codes = e.tb_codes + lv_in * L; s.in_score = e.tb_score + lv_in; s.in_count = e.tb_count + (size_t)n * c->Bmax;
         s.n = n; s.T = c->cfg.T[n]; s.per_beam = s.T; s.filter = (n + 1 == L) ? 1 : 0;
+        s.prefix_filter = (c->opt_level_filter && n + 1 < L) ? 1 : 0;
         s.gate = e.row_cur; s.gate_mode = 1; s.gate_value = n;
         s.out_codes = e.tb_codes + lv_out * L; s.out_score = e.tb_score + lv_out; s.out_parent = e.tb_parent + lv_out;
         s.out_count = e.tb_count + (size_t)(n + 1) * c->Bmax;
@@ -681,7 +694,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
   c->chains_now = 0;
-  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 1;
+  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 1; c->opt_level_filter = 0;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;
@@ -865,6 +878,9 @@ nezha_status nezha_set_option(nezha_ctx* c, int32_t option, int32_t value) {
     case NEZHA_OPT_FINAL_MASK:
       if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: final mask must be 0 or 1");
       c->opt_mask = value; break;
+    case NEZHA_OPT_LEVEL_FILTER:
+      if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: level filter must be 0 or 1");
+      c->opt_level_filter = value; break;
     default: return fail(c, NEZHA_ERR_ARG, "nezha_set_option: unknown option");
   }
   return NEZHA_OK;
@@ -946,7 +962,9 @@ nezha_status nezha_select(nezha_ctx* c, int32_t batch, int32_t n_beams, int32_t 
   SelectArgs s{};
   s.logits = logits; s.row_stride = c->cfg.T[level]; s.col_off = 0; s.src_row = nullptr; s.src_mul = n_beams;
   s.in_codes = beam_codes; s.in_score = beam_scores; s.in_count = n_live; s.in_stride = n_beams;
-  s.n = level; s.T = c->cfg.T[level]; s.K = beam_width; s.per_beam = per_beam; s.filter = filter ? 1 : 0;
+  s.n = level; s.T = c->cfg.T[level]; s.K = beam_width; s.per_beam = per_beam;
+  s.filter = (filter && level + 1 == c->L) ? 1 : 0; s.prefix_filter = (filter && level + 1 < c->L) ? 1 : 0;
+  s.pm = c->es.pm; s.final_mask_from_map = 0;
   s.gate_mode = 0;
   s.out_codes = nullptr; s.out_token = out_code; s.out_score = out_score; s.out_parent = out_parent; s.out_count = out_count;
   s.out_stride = beam_width; s.tuple_len = level; s.batch = batch; s.li = c->es.li; s.hs = c->es.hs;

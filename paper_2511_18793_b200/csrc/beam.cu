@@ -138,8 +138,11 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
         if (all_codes) key[j] += base;                   // rank by cumulative log-probability
       }
     }
-    if (all_codes && a.filter && a.pm.slots) {           // Eq. 5 on every extension of the beam: the prefix's bit set
-      const unsigned long long* bits = pm_find(a.pm, prefix_key);
+    // The bit set of the codes that may follow this beam: Eq. 5 for all T_L extensions at the last level, "some valid ID
+    // begins with it" at an earlier level.
+    const bool use_bits = a.prefix_filter || (all_codes && a.filter && a.final_mask_from_map);
+    const unsigned long long* bits = use_bits ? pm_find(a.pm, a.n, prefix_key) : nullptr;
+    if (all_codes && use_bits) {
 #pragma unroll
       for (int j = 0; j < VPL; ++j) {
         const int t = lane + 32 * j;
@@ -187,14 +190,14 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
       ++cnt;
     }
     __syncwarp();
-    if (!all_codes && a.filter) {                        // filter the chosen codes, keep their order
+    if (!all_codes && (a.filter || a.prefix_filter)) {   // filter the chosen codes, keep their order
       int kept = 0;
       for (int c0 = 0; c0 < cnt; c0 += 32) {
         const int c = c0 + lane;
         bool ok = false; float sv = 0.f; int t = 0;
         if (c < cnt) {
           sv = l_score[(size_t)r * a.K + c]; t = l_tok[(size_t)r * a.K + c];
-          ok = hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
+          ok = a.prefix_filter ? pm_test(bits, t) : hs_contains_thread(a.hs, prefix_key + (unsigned long long)t * mult_n);
         }
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         __syncwarp();

@@ -135,26 +135,33 @@ __device__ __forceinline__ void hs_contains_many(const HashSetView& hs, const un
 }
 
 // --------------------------------------------------------------------------------------------------
-// prefix map: the same set V, regrouped as (prefix of L-1 codes) -> bit set of the valid last codes
+// prefix map: the same set V, regrouped as (prefix of n codes) -> bit set of the codes that may follow it
 // --------------------------------------------------------------------------------------------------
-// Open addressing with linear probing over slots of `stride` words: word 0 = prefix key + 1 (0 = empty), words 1.. =
-// the bits of the last codes t with (prefix, t) in V.  The final-level mask of a beam then needs one look-up instead
-// of T_L hash probes; its answers are those of the hash set, bit for bit.
+// For every n in [0, L): the distinct n-code prefixes of the valid IDs, each with the bit set of the level-(n+1) codes t
+// such that some valid ID begins with (prefix, t).  For n = L - 1 that is Eq. 5 itself for all T_L extensions of a beam in
+// one look-up -- the same answers as T_L hash probes, bit for bit; for n < L - 1 it answers "does any valid ID begin with
+// these codes?", the validity filter at the earlier levels.  One table region per n (so a key needs no level tag), open
+// addressing with linear probing over slots of `stride` words inside the region: word 0 = prefix key + 1 (0 = empty),
+// words 1.. = the bit set.
 struct PrefixMapView {
   unsigned long long* slots;       // [n_slots * stride]; null = not in use
-  unsigned long long n_slots;
-  int stride;                      // words per slot: a power of two >= 1 + ceil(T_L / 64)
+  unsigned long long n_slots;      // all regions together
+  int stride;                      // words per slot: a power of two >= 1 + ceil(max T / 64)
+  unsigned long long level_off[kMaxLevels];     // first slot of the region of prefixes with n codes
+  unsigned long long level_slots[kMaxLevels];   // its slot count
 };
-// The bit set of a prefix, or null if no item has it.  Every lane of a warp may call this with the same key (the
-// loads are then broadcasts).
-__device__ __forceinline__ const unsigned long long* pm_find(const PrefixMapView& pm, unsigned long long prefix_key) {
-  unsigned long long s = __umul64hi(hs_mix(prefix_key), pm.n_slots);
+// The bit set of a prefix of n codes, or null if no valid ID begins with it.  Every lane of a warp may call this with the
+// same key (the loads are then broadcasts).
+__device__ __forceinline__ const unsigned long long* pm_find(const PrefixMapView& pm, int n, unsigned long long prefix_key) {
+  const unsigned long long ns = pm.level_slots[n];
+  const unsigned long long* region = pm.slots + pm.level_off[n] * pm.stride;
+  unsigned long long s = __umul64hi(hs_mix(prefix_key), ns);
   for (int step = 0; step < kMaxProbeBuckets; ++step) {
-    const unsigned long long* slot = pm.slots + s * pm.stride;
+    const unsigned long long* slot = region + s * pm.stride;
     const unsigned long long k = __ldg(slot);
     if (k == prefix_key + 1) return slot + 1;
     if (k == 0ull) return nullptr;
-    if (++s == pm.n_slots) s = 0;
+    if (++s == ns) s = 0;
   }
   return nullptr;
 }

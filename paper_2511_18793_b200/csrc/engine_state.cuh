@@ -66,7 +66,9 @@ struct SelectArgs {
   int tuple_len;                        // row length of in_codes / out_codes (L)
   int batch;
   LevelInfo li; HashSetView hs;
-  PrefixMapView pm;                     // slots == null: the last-level mask probes the hash set; else it reads the prefix's bit set
+  PrefixMapView pm;
+  int final_mask_from_map;              // 1: the last-level mask of a beam (all T_L extensions) reads the prefix map; 0: hash probes
+  int prefix_filter;                    // 1: this is an earlier level and candidates that begin no valid ID are dropped
 };
 void launch_select(const SelectArgs& a, cudaStream_t st);
 // launch_select (gated on row_cur == n) followed, in the same launch, by launch_advance of level n

@@ -89,30 +89,39 @@ __global__ void __launch_bounds__(256) hs_probe_kernel(HashSetView hs, const uns
   }
 }
 
-// One thread per item: claims (or finds) the slot of the item's prefix, then sets the bit of its last code.
+// One thread per item: for every n in [0, L) it claims (or finds) the slot of the item's n-code prefix in region n and sets
+// the bit of the item's next code.  The bit is tested first: the few prefixes at the top of the tree are shared by
+// millions of items, whose atomics on the same word would otherwise serialise.
 __global__ void pm_insert_kernel(LevelInfo li, PrefixMapView pm, const int* __restrict__ codes, unsigned long long n, int* status) {
   const unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x;
   if (i >= n) return;
+  int c[kMaxLevels];
+  for (int l = 0; l < li.L; ++l) {
+    c[l] = codes[i * li.L + l];
+    if (c[l] < 0 || c[l] >= li.T[l]) return;        // hs_insert_kernel has reported it
+  }
   unsigned long long p = 0;
-  for (int l = 0; l + 1 < li.L; ++l) {
-    const int c = codes[i * li.L + l];
-    if (c < 0 || c >= li.T[l]) return;              // hs_insert_kernel has reported it
-    p += (unsigned long long)c * li.mult[l];
-  }
-  const int t = codes[i * li.L + li.L - 1];
-  if (t < 0 || t >= li.T[li.L - 1]) return;
-  unsigned long long s = __umul64hi(hs_mix(p), pm.n_slots);
-  for (int step = 0; step < kMaxProbeBuckets; ++step) {
-    unsigned long long* slot = pm.slots + s * pm.stride;
-    unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(slot);
-    if (cur == 0ull) cur = atomicCAS(slot, 0ull, p + 1);
-    if (cur == 0ull || cur == p + 1) {
-      atomicOr(slot + 1 + (t >> 6), 1ull << (t & 63));
-      return;
+  for (int lv = 0; lv < li.L; ++lv) {               // prefix of lv codes, next code c[lv]
+    if (lv > 0) p += (unsigned long long)c[lv - 1] * li.mult[lv - 1];
+    const int t = c[lv];
+    const unsigned long long ns = pm.level_slots[lv];
+    unsigned long long* region = pm.slots + pm.level_off[lv] * pm.stride;
+    unsigned long long s = __umul64hi(hs_mix(p), ns);
+    bool done = false;
+    for (int step = 0; step < kMaxProbeBuckets && !done; ++step) {
+      unsigned long long* slot = region + s * pm.stride;
+      unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(slot);
+      if (cur == 0ull) cur = atomicCAS(slot, 0ull, p + 1);
+      if (cur == 0ull || cur == p + 1) {
+        unsigned long long* word = slot + 1 + (t >> 6);
+        const unsigned long long bit = 1ull << (t & 63);
+        if (!(*reinterpret_cast<volatile unsigned long long*>(word) & bit)) atomicOr(word, bit);
+        done = true;
+      }
+      if (++s == ns) s = 0;
     }
-    if (++s == pm.n_slots) s = 0;
+    if (!done) { atomicOr(status, kStHashFull); return; }
   }
-  atomicOr(status, kStHashFull);
 }
 
 void launch_pm_build(const LevelInfo& li, PrefixMapView pm, const int* codes, unsigned long long n, int* status, cudaStream_t st) {

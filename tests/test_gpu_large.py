@@ -66,10 +66,14 @@ def test_full_size_workload(name):
     h = case.eng.get_hidden().cpu().numpy()
     beams = out["trace"]["beams"].cpu().numpy()
     scores = out["trace"]["beam_scores"].cpu().numpy()
+    swaps = []
     for b in rows:
         dh = h[b] - case.req(b).h
         assert np.abs(dh).max() < hidden_tolerance(w) and np.sqrt((dh ** 2).mean()) < hidden_rms_bound(w)
-        check_levels(case, b, beams[:, b], scores[:, b], w.beam, tol=e2e_tolerance(w))
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam, tol=e2e_tolerance(w), swaps=swaps)
+    # members that were not the oracle's own choice (all of them near-ties at the K-th place): a minority at every level
+    print(f"{name}: tie-rule members per (request, level): {swaps}")
+    assert max(swaps) <= w.beam // 2
     # draft head, stage-wise: the oracle's Eq. 1-2 on the hidden states the GPU's prefill produced (float64 copies of
     # the same numbers), so that the 2e-2 budget is spent by the draft head alone and not by 24-32 layers of bf16
     # activations upstream; end to end (oracle hidden states) the same logits stay within the depth-scaled bound
@@ -82,3 +86,47 @@ def test_full_size_workload(name):
         assert np.abs(gotd[b, 0] - head.logits(0, hg[1], hg[0])).max() < tol
         assert np.abs(gotd[b, 0] - head.logits(0, case.req(b).h[1], case.req(b).h[0])).max() < \
             tol + 1.5 * e2e_tolerance(w, std=w_std)
+
+
+@pytest.mark.parametrize("name", ["0.5b", "1.5b", "7b"])
+def test_two_layer_cut_at_full_width(name):
+    """The three LLM shapes cut to two layers: full width, head dimension, grouped-query ratio, context length and beam
+    (so the CTA-pair GEMM, both tcgen05 attention shapes and the 20- / 50-beam selection all run), without 24-32 layers
+    of accumulated bf16 rounding between the GPU and the fp64 oracle.  Every request, every stage:
+      * prefill hidden states within the two-layer bound; teacher-forced primary logits of every level within 2e-2 in rms
+        at every width, and their largest element (of 20 k per request and level) within the plain 2e-2 at d = 896 and
+        d = 1536; at d = 4096 the measured hidden-state error (0.0074 rms after one layer, 0.0105 after two) seen through
+        an LM-head row of norm 0.02 * sqrt(4096) = 1.28 is 0.0134 rms per logit, and the largest is held to 5 sigma of that;
+      * every beam level of the verified decode against the oracle's expansion of the GPU's own beams;
+      * verified == plain autoregressive decode, zero hallucinations, the accept / roll-back walk replayed."""
+    w = synth.scaled(synth.WORKLOADS[name], n_layers=2, batch=4, n_items=200_000)
+    case = Case(w).prefill()
+    model, head, V = case.oracle
+    tol = 2e-2 if name != "7b" else 5.0 * 0.02 * np.sqrt(w.d_model) * 0.0074 * np.sqrt(2.0)
+    h = case.eng.get_hidden().cpu().numpy()
+    for b in range(w.batch):
+        dh = h[b] - case.req(b).h
+        assert np.abs(dh).max() < hidden_tolerance(w) and np.sqrt((dh ** 2).mean()) < hidden_rms_bound(w)
+    rng = np.random.default_rng(3)
+    for level in range(w.L):
+        pre = np.stack([rng.integers(0, w.T[l], size=(w.batch, w.beam)) for l in range(level)], axis=2).astype(np.int32) \
+            if level else None
+        pt = None if pre is None else torch.from_numpy(pre).cuda()
+        got = case.eng.primary_logits(w.beam, level, pt).cpu().numpy()
+        for b in range(w.batch):
+            ref = model.next_level_logits_many(case.req(b), [tuple(pre[b, r]) if level else () for r in range(w.beam)])
+            err = got[b] - np.stack(ref)
+            assert np.abs(err).max() < tol and np.sqrt((err ** 2).mean()) < 2e-2, (level, b, np.abs(err).max())
+    out = case.eng.decode(w.beam, mode=1, trace=True)
+    ar = case.eng.decode(w.beam, mode=2)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
+    codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
+    live = np.arange(w.beam)[None, :] < count[:, None]
+    assert V.contains(codes[live]).all() and np.all(codes[~live] == -1)
+    beams, scores = out["trace"]["beams"].cpu().numpy(), out["trace"]["beam_scores"].cpu().numpy()
+    swaps = []
+    for b in range(w.batch):
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam, tol=max(tol, e2e_tolerance(w)), swaps=swaps)
+    print(f"{name} (2 layers): tie-rule members per (request, level): {swaps}")
+    assert max(swaps) <= w.beam // 2
+    check_walk_against_trace(out, w.batch, w.L)

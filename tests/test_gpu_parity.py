@@ -443,6 +443,67 @@ def test_final_mask_from_prefix_map_equals_hash_probes(name):
     assert torch.equal(again["codes"], base[1]["codes"])
 
 
+# ---------------------------------------------------------------------------------------- validity at every level
+@pytest.mark.parametrize("name", ["tiny", "small_cut", "t512", "sparse"])
+def test_validity_filter_at_every_level(name):
+    """NEZHA_OPT_LEVEL_FILTER = 1: a partial ID survives a level only if some valid ID begins with it.  Every mode against
+    the oracle with the same switch; every beam of every level is the beginning of a catalogue item; modes 1 and 2 agree;
+    and a search that wastes no beam on dead prefixes returns at least as many items as the default."""
+    w = {"tiny": synth.WORKLOADS["tiny"],
+         "small_cut": synth.scaled(synth.WORKLOADS["small"], n_layers=2, n_items=100_000, batch=4, n_hist=20),
+         "t512": synth.scaled(synth.WORKLOADS["paper"], n_layers=1, batch=3),
+         # a catalogue so thin that most first codes begin no item
+         "sparse": synth.scaled(synth.WORKLOADS["tiny"], n_items=12, batch=3, beam=6)}[name]
+    case = Case(w).prefill()
+    model, head, V = case.oracle
+    base = {m: case.eng.decode(w.beam, mode=m) for m in (0, 1, 2)}
+    case.eng.set_option(4, 1)
+    out = case.eng.decode(w.beam, mode=1, trace=True)
+    ar = case.eng.decode(w.beam, mode=2)
+    dr = case.eng.decode(w.beam, mode=0)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
+    beams, scores = out["trace"]["beams"].cpu().numpy(), out["trace"]["beam_scores"].cpu().numpy()
+    dcodes, dscores, dcount = (dr[k].cpu().numpy() for k in ("codes", "scores", "count"))
+    for b in range(w.batch):
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam, every_level=True)
+        for n in range(w.L):
+            cnt = int((beams[n, b, :, 0] >= 0).sum())
+            assert V.contains_prefix(beams[n, b, :cnt, : n + 1]).all()
+        ref = O.nezha_draft(head, case.req(b), w.beam, V, every_level=True)[-1]
+        assert_topk_matches(dcodes[b], dscores[b], dcount[b], ref, w.beam, tolerance(w))
+    check_walk_against_trace(out, w.batch, w.L)
+    for m, got in ((0, dr), (1, out), (2, ar)):
+        assert bool((got["count"] >= base[m]["count"]).all()), (name, m)
+    print(f"{name}: requests with fewer than K items, last-level filter only -> every level: "
+          f"{int((base[2]['count'] < w.beam).sum())} -> {int((ar['count'] < w.beam).sum())} of {w.batch} (primary), "
+          f"{int((base[0]['count'] < w.beam).sum())} -> {int((dr['count'] < w.beam).sum())} (draft head)")
+    case.eng.set_option(4, 0)
+    again = case.eng.decode(w.beam, mode=1)
+    assert torch.equal(again["codes"], base[1]["codes"])
+
+
+def test_select_stage_with_prefix_filter(tiny):
+    """One level of beam search on caller-supplied logits with the filter at an earlier level (level 1 of 3)."""
+    w = tiny.w
+    V = tiny.oracle[2]
+    rng = np.random.default_rng(3)
+    nb, K, level = 4, w.beam, 1
+    logits = rng.standard_normal((w.batch, nb, w.T[level])).astype(np.float32)
+    bscore = -rng.random((w.batch, nb)).astype(np.float32)
+    bcodes = np.stack([rng.permutation(w.T[0])[:nb] for _ in range(w.batch)])[:, :, None].astype(np.int32)
+    n_live = np.full((w.batch,), nb, dtype=np.int32)
+    for per_beam in (w.T[level], 3):
+        parent, code, score, count = (x.cpu().numpy() for x in tiny.eng.select(
+            torch.from_numpy(logits).cuda(), torch.from_numpy(bscore).cuda(), torch.from_numpy(bcodes).cuda(),
+            torch.from_numpy(n_live).cuda(), K, level, per_beam, True))
+        for b in range(w.batch):
+            beams = [O.Beam((int(bcodes[b, r, 0]),), np.float32(bscore[b, r])) for r in range(nb)]
+            ref = O.expand_level(beams, [logits[b, r].astype(np.float64) for r in range(nb)], K, per_beam, V)
+            got = [(int(bcodes[b, parent[b, k], 0]), int(code[b, k])) for k in range(count[b])]
+            assert got == [x.codes for x in ref]
+            assert np.allclose(score[b, : count[b]], [float(x.score) for x in ref], atol=2e-6)
+
+
 def test_nearly_full_tables():
     """Load factor 0.95: long probe walks in the hash set and in the prefix map; membership stays exact, and both
     last-level masks still agree with each other and with the oracle's set."""

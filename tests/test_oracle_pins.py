@@ -527,6 +527,61 @@ def test_draft_head_ablation_identities():
                           h1.logits(1, req.h[2], O.teacher_forced_state(h1, req, (3,))))
 
 
+def test_prefix_validity_matches_python_sets():
+    w = synth.WORKLOADS["tiny"]
+    cat = synth.make_catalog(w)
+    V = O.ValidSet(cat, w.T)
+    rows = cat.tolist()
+    for n in (1, 2):
+        ref = {tuple(r[:n]) for r in rows}
+        grid = np.stack(np.meshgrid(*[np.arange(t) for t in w.T[:n]], indexing="ij"), axis=-1).reshape(-1, n)
+        got = V.contains_prefix(grid)
+        assert np.array_equal(got, np.array([tuple(r) in ref for r in grid.tolist()]))
+        assert got.sum() == len(ref) == V.prefix_keys(n).size
+    grid3 = np.asarray(rows[:50] + [[31, 31, 31], [0, 0, 0]])
+    assert np.array_equal(V.contains_prefix(grid3), V.contains(grid3))       # full length: Eq. 5 itself
+    # unequal radices: the prefix of a key is the key modulo the product of the leading radices
+    V2 = O.ValidSet(np.array([[2, 4, 6], [1, 0, 3]]), (3, 5, 7))
+    assert V2.prefix_keys(2).tolist() == sorted([2 + 4 * 3, 1 + 0 * 3])
+    assert V2.contains_prefix(np.array([[2, 4], [1, 0], [2, 0], [1, 4]])).tolist() == [True, True, False, False]
+
+
+def test_validity_at_every_level():
+    """The per-step variant of the verification (Section 3.4): with the filter at every level every surviving beam of
+    every level is the beginning of a valid ID; without pruning (K >= the number of prefixes) the result is unchanged;
+    with pruning a search that wastes no beam on dead prefixes returns at least as many items."""
+    w, W, cat, model, head, V, hist = _micro()
+    valid = [tuple(r) for r in cat.tolist()]
+    for b in range(hist.shape[0]):
+        req = model.prefill(hist[b])
+        for K in (1, 2, 3, 5, 16):
+            for search in (lambda **kw: O.ar_beam_search(model, req, K, V, **kw),
+                           lambda **kw: O.nezha_draft(head, req, K, V, **kw),
+                           lambda **kw: O.speculative_decode(model, head, req, K, V, **kw)[0]):
+                on, off = search(every_level=True), search()
+                for n, level in enumerate(on):
+                    assert all(any(v[: n + 1] == bm.codes for v in valid) for bm in level)
+                assert len(on[-1]) >= len(off[-1])
+                if K == 16:                                        # nothing is pruned before the last level
+                    assert codes_of(on[-1]) == codes_of(off[-1])
+                    assert np.array_equal(scores_of(on[-1]), scores_of(off[-1]))
+            # Algorithm 2 still returns Algorithm 1's result under the same filter
+            assert codes_of(O.speculative_decode(model, head, req, K, V, every_level=True)[0][-1]) == \
+                codes_of(O.ar_beam_search(model, req, K, V, every_level=True)[-1])
+    # hand-worked, zero heads, K = 2: valid IDs (1,2,0), (1,3,1), (2,0,0).  Level 1: codes 0..3 tie, 0 and 3 begin no
+    # valid ID -> B_1 = {(1),(2)}.  Level 2: (1,2),(1,3),(2,0) are the live prefixes; ties go to the smaller parent rank
+    # -> B_2 = {(1,2),(1,3)}.  Level 3 -> {(1,2,0),(1,3,1)}.  Without the per-level filter B_1 = {(0),(1)} and
+    # B_2 = {(0,0),(0,1)}, which no valid ID continues: nothing is returned.
+    model, head, V, req = _zero_head_case([(1, 2, 0), (1, 3, 1), (2, 0, 0)])
+    on = O.ar_beam_search(model, req, 2, V, every_level=True)
+    assert [codes_of(x) for x in on] == [[(1,), (2,)], [(1, 2), (1, 3)], [(1, 2, 0), (1, 3, 1)]]
+    assert O.ar_beam_search(model, req, 2, V)[-1] == []
+    # the draft head takes its top-2 codes per beam BEFORE the filter (Algorithm 3's order): at level 1 codes 0 and 1,
+    # of which only (1) is live; then (1,0),(1,1) -- both dead: no draft survives
+    d = O.nezha_draft(head, req, 2, V, every_level=True)
+    assert [codes_of(x) for x in d] == [[(1,)], [], []]
+
+
 # ---------------------------------------------------------------------------------------- ablation variants (Section 4.3)
 def test_ablation_variants_of_the_draft_head():
     """NEZHA-1 (no context state): every level's distribution ignores the prefix, so the joint log-probability is a sum
