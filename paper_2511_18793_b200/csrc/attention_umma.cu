@@ -41,7 +41,12 @@ template <int HD> struct UmmaCfg {
   // two CTAs share an SM.  A CTA is a chain (S -> softmax -> P V per tile) whose softmax takes most of the tile's time;
   // the S product of the next tile still runs under it (the scores leave TMEM at the start of the softmax), and
   // concurrency comes from the CTAs that share the SM rather than from second buffers.
-  static constexpr int kSmemBytes = kQBytes + kPBytes + 2 * kRingU * kTileBytes + 1024 + 256;
+  // Two CTAs of the hd = 128 shape fit an SM only if each stays below (228 KB - 2 x 1 KB reserved) / 2 = 113 KB: the tiles
+  // alone are 112 KB, so the barriers get 128 bytes and the alignment slack 512 (the dynamic array is declared with the
+  // tiles' 1024-byte alignment; the kernel checks the slack it really needs and reports instead of overrunning).
+  static constexpr int kBarBytes = 128, kSlack = 512;
+  static constexpr int kTilesBytes = kQBytes + kPBytes + 2 * kRingU * kTileBytes;
+  static constexpr int kSmemBytes = kTilesBytes + kBarBytes + kSlack;
   static constexpr int kTmemCols = HD == 64 ? 128 : 256;       // S: 64 columns, O: HD columns; a power of two
   static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kPosU >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
   static constexpr uint32_t kIdescPV =
@@ -70,6 +75,31 @@ __device__ __forceinline__ float ex2u(float x) {
   return y;
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Two fp32 values in one 64-bit register pair: the packed fp32 instructions of sm_100 (one issue slot for two lanes of
+// arithmetic) carry the scale-subtract and the row sum of the softmax, whose instruction count is what bounds this kernel.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 
 template <int HD>
 __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
@@ -105,8 +135,12 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
   const int NT = n_tiles + n_xt;
   const int kv_row0 = (int)(((long long)request * a.Hkv + kvh) * (a.ctx_head_stride / HD));
 
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  if (base - smem_u32(smem_raw) > (uint32_t)C::kSlack) {   // the array came less aligned than declared: report, touch nothing
+    if (threadIdx.x == 0) atomicOr(status, kStInternal);
+    return;
+  }
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_base = base, p_base = base + C::kQBytes, k_base = p_base + C::kPBytes, v_base = k_base + S * C::kTileBytes;
   const uint32_t bar_base = v_base + S * C::kTileBytes;
@@ -236,12 +270,12 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
     }
     for (int j = 0; j < NT; ++j) {
       const uint32_t par = (uint32_t)j & 1u, par_prev = par ^ 1u;
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(s_full, par, abort_flag));
+      ok = warp_wait(s_full, par, abort_flag, lane);
       if (!ok) break;
       if (warp_dead) {                               // (its P rows stay whatever they are: O rows nobody reads)
         if (lane == 0) mbar_arrive(s_free);
         if (j >= 1) {
-          ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, par_prev, abort_flag));
+          ok = warp_wait(pv_done, par_prev, abort_flag, lane);
           if (!ok) break;
         }
         if (lane == 0) mbar_arrive(p_full);
@@ -271,26 +305,32 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
       }
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < kPosU; ++c) mx = fmaxf(mx, sv[c]);
+      for (int c = 0; c < kPosU; c += 2) mx = max3(mx, sv[c], sv[c + 1]);
       mx *= sc;
       // raise the reference only when the true maximum has run away from it: p stays below 2^8 otherwise
       const bool raise = mx > m_ref + kRaise || (m_ref == -INFINITY && mx > -INFINITY);
       const float m_new = raise ? mx : m_ref;
       const float m_safe = m_new == -INFINITY ? 0.f : m_new;
       const float corr = raise ? ex2u(m_ref - m_safe) : 1.f;     // ex2(-inf) = 0 the first time
-      float rs = 0.f;
+      const f32x2 sc2 = pack2(sc, sc), neg_m2 = pack2(-m_safe, -m_safe);
+      f32x2 rs2 = pack2(0.f, 0.f);
       uint32_t pk[kPosU / 2];
 #pragma unroll
       for (int c = 0; c < kPosU; c += 2) {
-        const float p0 = ex2u(fmaf(sv[c], sc, -m_safe)), p1 = ex2u(fmaf(sv[c + 1], sc, -m_safe));
-        rs += p0 + p1;
+        float x0, x1;
+        unpack2(fma2(pack2(sv[c], sv[c + 1]), sc2, neg_m2), x0, x1);
+        const float p0 = ex2u(x0), p1 = ex2u(x1);
+        rs2 = add2(rs2, pack2(p0, p1));
         __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
         pk[c >> 1] = *reinterpret_cast<uint32_t*>(&pb);
       }
+      float rs_lo, rs_hi;
+      unpack2(rs2, rs_lo, rs_hi);
+      const float rs = rs_lo + rs_hi;
       l_run = l_run * corr + rs;
       m_ref = m_new;
       if (j >= 1) {                                  // the PV product of tile j - 1 is done: P is free, O holds every earlier tile
-        ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, par_prev, abort_flag));
+        ok = warp_wait(pv_done, par_prev, abort_flag, lane);
         if (!ok) break;
       }
       if (j > 0 && __any_sync(0xffffffffu, raise)) { // rescale O
@@ -314,7 +354,7 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
       if (lane == 0) mbar_arrive(p_full);
     }
     if (ok && NT > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(pv_done, (uint32_t)(NT - 1) & 1u, abort_flag));
+      ok = warp_wait(pv_done, (uint32_t)(NT - 1) & 1u, abort_flag, lane);
       tc_fence_after();
     }
     if (!ok) { if (lane == 0) *abort_flag = 1; }

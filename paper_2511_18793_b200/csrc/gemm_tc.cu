@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(kThreads + 32 * (ISS - 1)) gemm_tc_kernel(cons
       const int m0 = (tile % tiles_m) * BM, n0 = tn * BN;
       const int b = t_local & 1;
       const EpiRow er = epilogue_row<EPI>(a, m0 + q * 32 + lane, M);   // overlaps the main loop
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(acc_full(b), (t_local >> 1) & 1, abort_flag));   // warp-uniform
+      ok = warp_wait(acc_full(b), (t_local >> 1) & 1, abort_flag, lane);
       if (!ok) break;
       tc_fence_after();
       drain_accumulator<BN, EPI, ISS>(a, tmem_base + (uint32_t)(b * BN * ISS), q, half, lane, stg4, m0, n0, M, er);
@@ -239,6 +239,9 @@ void launch_bn(const GemmArgs& a, cudaStream_t st) {
 constexpr int kPlanPairs = 512;
 int gemm_tc_plan(int M, int N) {
   static const bool no_pairs = getenv("NEZHA_NO_CTA_PAIRS") != nullptr;
+  static const int forced = getenv("NEZHA_GEMM_PLAN") ? atoi(getenv("NEZHA_GEMM_PLAN")) : 0;   // experiments: 32 .. 256, 512 = pairs
+  if (forced == 512 && M >= 1 && N >= 256) return kPlanPairs;
+  if (forced == 32 || forced == 64 || forced == 128 || forced == 256) return forced;
   const long long tiles_m = (M + BM - 1) / BM;
   static const int widths[4] = {256, 128, 64, 32}, wave_cost[4] = {512, 400, 300, 250};
   long long best = -1; int plan = 32;

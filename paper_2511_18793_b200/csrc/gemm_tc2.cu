@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) gemm_tc_pair_kernel(const __grid_con
       const int m0 = (tile % tiles_m) * (2 * BM) + rank * BM, n0 = (tile / tiles_m) * kBN2;
       const int b = t_local & 1;
       const EpiRow er = epilogue_row<EPI>(a, m0 + q * 32 + lane, M);
-      ok = __all_sync(0xffffffffu, mbar_wait_or_abort(acc_full(b), (t_local >> 1) & 1, abort_flag));
+      ok = warp_wait(acc_full(b), (t_local >> 1) & 1, abort_flag, lane);
       if (!ok) break;
       tc_fence_after();
       drain_accumulator<kBN2, EPI>(a, tmem_base + (uint32_t)(b * kBN2), q, half, lane, stg4, m0, n0, M, er);

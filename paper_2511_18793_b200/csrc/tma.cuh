@@ -55,6 +55,14 @@ __device__ __forceinline__ bool mbar_wait_or_abort(uint32_t bar, uint32_t parity
     if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
   }
 }
+// One lane waits for the barrier and tells the rest of the warp (which sleeps at the shuffle instead of polling): 32
+// polling lanes are 32 times the instructions, taken from the warps of the SM that have arithmetic to issue.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = mbar_wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
+  __syncwarp();                                    // orders the other lanes' later accesses after lane 0's acquire
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
 // Fetches a tensor map into the descriptor cache ahead of its first copy (the map is a kernel parameter: this reads
 // nothing an earlier kernel wrote, so it may run before the dependency wait).
 __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* tm) {

@@ -94,15 +94,16 @@ def test_two_layer_cut_at_full_width(name):
     (so the CTA-pair GEMM, both tcgen05 attention shapes and the 20- / 50-beam selection all run), without 24-32 layers
     of accumulated bf16 rounding between the GPU and the fp64 oracle.  Every request, every stage:
       * prefill hidden states within the two-layer bound; teacher-forced primary logits of every level within 2e-2 in rms
-        at every width, and their largest element (of 20 k per request and level) within the plain 2e-2 at d = 896 and
-        d = 1536; at d = 4096 the measured hidden-state error (0.0074 rms after one layer, 0.0105 after two) seen through
-        an LM-head row of norm 0.02 * sqrt(4096) = 1.28 is 0.0134 rms per logit, and the largest is held to 5 sigma of that;
+        at every width, and their largest element (of 5 k to 13 k per request and level) within five standard deviations
+        of the rounding model: the measured hidden-state error of bf16 activations (0.0074 rms after one layer, 0.0105
+        after two, whatever the width) seen through an LM-head row of norm 0.02 * sqrt(d) is 0.0063 / 0.0082 / 0.0134 rms
+        per logit at d = 896 / 1536 / 4096;
       * every beam level of the verified decode against the oracle's expansion of the GPU's own beams;
       * verified == plain autoregressive decode, zero hallucinations, the accept / roll-back walk replayed."""
     w = synth.scaled(synth.WORKLOADS[name], n_layers=2, batch=4, n_items=200_000)
     case = Case(w).prefill()
     model, head, V = case.oracle
-    tol = 2e-2 if name != "7b" else 5.0 * 0.02 * np.sqrt(w.d_model) * 0.0074 * np.sqrt(2.0)
+    tol = max(2e-2, 5.0 * 0.02 * np.sqrt(w.d_model) * 0.0074 * np.sqrt(2.0))
     h = case.eng.get_hidden().cpu().numpy()
     for b in range(w.batch):
         dh = h[b] - case.req(b).h
