@@ -27,7 +27,7 @@ template <int BN> struct Cfg {
   static constexpr int kStageBytes = kTileBytesA + kTileBytesB;
   // as many stages as fit beside the transpose tiles: short-M launches are bound by bytes in flight per CTA
   // (even, so that with two MMA issuers a ring slot always belongs to the same issuer: see the kernel)
-  static constexpr int kStages = BN == 256 ? 4 : BN == 128 ? 6 : 8;
+  static constexpr int kStages = BN >= 192 ? 4 : BN == 160 ? 5 : BN == 128 ? 6 : 8;
   static constexpr int kSmemBytes =
       kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTransposeBytes;
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;       // two accumulators; a power of two >= 32
@@ -47,8 +47,10 @@ __global__ void __launch_bounds__(kThreads + 32 * (ISS - 1)) gemm_tc_kernel(cons
                                                                             const __grid_constant__ CUtensorMap tmB,
                                                                             GemmArgs a, int* status) {
   using C = Cfg<BN>;
-  constexpr int kTmemCols = 2 * BN * ISS < 32 ? 32 : 2 * BN * ISS;   // two accumulators of ISS chains each
-  static_assert(2 * BN * ISS <= 512, "accumulator chains do not fit");
+  // two accumulators of ISS chains each, in a power-of-two number of TMEM columns
+  constexpr int kAccCols = 2 * BN * ISS;
+  constexpr int kTmemCols = kAccCols <= 32 ? 32 : kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;
+  static_assert(kAccCols <= 512, "accumulator chains do not fit");
   // A slot's `full` barrier must be waited for by ONE thread, phase after phase: a thread that asked for the phase after
   // the one still in flight would be told "complete" (the parity it names is also that of the phase before).  With the
   // k-steps dealt round-robin that holds exactly when the ring length is a multiple of the number of issuers.
@@ -232,27 +234,32 @@ void launch_bn(const GemmArgs& a, cudaStream_t st) {
 
 }  // namespace
 
-// Tiling of a launch: 32 / 64 / 128 / 256 = output-tile width of the single-CTA kernel, kPlanPairs = 256 x 256 tiles on
-// CTA pairs.  Cost model: waves of tiles over the SMs (over the SM pairs) times the measured relative cost of one wave
-// of that tile (a wider tile does more per wave but costs less than proportionally more: it moves fewer operand bytes
-// per flop).  Pairs need at least a thousand rows: below that every launch is a single short wave anyway.
+// Tiling of a launch: 32 ... 256 = output-tile width of the single-CTA kernel, kPlanPairs = 256 x 256 tiles on CTA pairs.
+// Cost model: waves of tiles over the SMs (over the SM pairs) times the relative cost of one wave of that tile.  The
+// tiling never changes the order in which a product's K range is summed, so it may depend on the row count.
 constexpr int kPlanPairs = 512;
-int gemm_tc_plan(int M, int N) {
+// Output-tile widths of the single-CTA kernel and the measured relative cost of one wave of each (a wider tile does more
+// per wave but costs less than proportionally more: it moves fewer operand bytes per flop; 256 / 128 / 64 / 32 measured,
+// the widths in between interpolated).  The in-between widths exist for passes of a few hundred rows over a wide model:
+// 640 rows x 4096 columns are 80 tiles of 256 columns on 148 SMs, but 130 tiles of 160 columns, each a third shorter.
+static const int kWidths[7] = {256, 224, 192, 160, 128, 64, 32}, kWaveCost[7] = {512, 484, 456, 428, 400, 300, 250};
+int gemm_tc_plan(int M, int N, int K) {
   static const bool no_pairs = getenv("NEZHA_NO_CTA_PAIRS") != nullptr;
-  static const int forced = getenv("NEZHA_GEMM_PLAN") ? atoi(getenv("NEZHA_GEMM_PLAN")) : 0;   // experiments: 32 .. 256, 512 = pairs
+  static const int forced = getenv("NEZHA_GEMM_PLAN") ? atoi(getenv("NEZHA_GEMM_PLAN")) : 0;   // experiments: a width, 512 = pairs
   if (forced == 512 && M >= 1 && N >= 256) return kPlanPairs;
-  if (forced == 32 || forced == 64 || forced == 128 || forced == 256) return forced;
+  for (int i = 0; i < 7; ++i)
+    if (forced == kWidths[i]) return forced;
   const long long tiles_m = (M + BM - 1) / BM;
-  static const int widths[4] = {256, 128, 64, 32}, wave_cost[4] = {512, 400, 300, 250};
   long long best = -1; int plan = 32;
-  for (int i = 0; i < 4; ++i) {
-    const int bn = widths[i];
+  for (int i = 0; i < 7; ++i) {
+    const int bn = kWidths[i];
     if (bn > 32 && N < bn) continue;
     const long long tiles = tiles_m * ((N + bn - 1) / bn);
-    const long long cost = ((tiles + sm_count() - 1) / sm_count()) * wave_cost[i];
+    const long long cost = ((tiles + sm_count() - 1) / sm_count()) * kWaveCost[i];
     if (best < 0 || cost < best) { best = cost; plan = bn; }
   }
-  if (!no_pairs && M >= 1024 && N >= 512) {
+  // pairs: a thousand rows or more, or half of that when the k-loop is long enough to outweigh a cluster launch
+  if (!no_pairs && (M >= 1024 || (M >= 512 && K >= 2048)) && N >= 512) {
     const long long pairs = sm_count() / 2;
     const long long tiles = ((M + 2 * BM - 1) / (2 * BM)) * (long long)((N + 255) / 256);
     const long long cost = ((tiles + pairs - 1) / pairs) * 480;
@@ -299,9 +306,12 @@ void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     }
     return;
   }
-  switch (gemm_tc_plan(m_plan, a.N)) {
+  switch (gemm_tc_plan(m_plan, a.N, a.K)) {
     case kPlanPairs: launch_gemm_tc_pair(a, sm_count(), st); break;
     case 256: launch_bn<256, 1>(a, st); break;
+    case 224: launch_bn<224, 1>(a, st); break;
+    case 192: launch_bn<192, 1>(a, st); break;
+    case 160: launch_bn<160, 1>(a, st); break;
     case 128: launch_bn<128, 1>(a, st); break;
     case 64: launch_bn<64, 1>(a, st); break;
     default: launch_bn<32, 1>(a, st); break;
