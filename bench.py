@@ -361,6 +361,10 @@ def main():
                     help="mode 1 only: 'natural' = the (random-init) draft head's own draft tree; 'perfect' = the true beam "
                          "sets of every level injected as round 1's draft tree (best case: one round, everything accepted)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (requests per decode call)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="cut the backbone down to this many layers (profiler captures on a small case: a kernel's launch "
+                         "is the same at any depth); the line then describes a cut-down workload, not the configuration")
+    ap.add_argument("--items", type=int, default=0, help="cut the catalogue down to this many items (same purpose)")
     ap.add_argument("--final-mask", default="prefix", choices=["hash", "prefix"],
                     help="how the primary model's last-level validity mask (Eq. 5) is answered: the prefix map (the "
                          "library's default) or one hash-set probe per candidate code")
@@ -386,7 +390,11 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.batch > 0:
         w = synth.scaled(w, batch=args.batch)
-    config = {"workload": workload_label(w),
+    if args.layers > 0:
+        w = synth.scaled(w, n_layers=args.layers)
+    if args.items > 0:
+        w = synth.scaled(w, n_items=args.items)
+    config = {"workload": workload_label(w) + (" [cut down for profiling]" if args.layers > 0 or args.items > 0 else ""),
               "mode": {0: "draft-only (Algorithm 3)", 1: "verified (Algorithm 2)", 2: "autoregressive (Algorithm 1)"}[args.mode],
               "batch": w.batch, "beam": w.beam, "l2": "flushed between steps (256 MB write, outside the timed events)",
               "drafts": "natural (random-init draft head)" if args.drafts == "natural" or args.mode != 1 else
@@ -478,7 +486,7 @@ def main():
         line["cpu_baseline"] = cpu_baseline(ctx, args)
 
     # ---- the other configurations, briefly (one GPU, default run only): same step, fewer repetitions
-    if world == 1 and not args.no_per_workload and args.workload == "7b" and args.batch == 0:
+    if world == 1 and not args.no_per_workload and args.workload == "7b" and args.batch == 0 and not args.layers and not args.items:
         per = {}
         del res, step, out
         ctx.clear(); eng.close(); del eng

@@ -114,11 +114,12 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
 
   pdl_wait();                                       // before the first global read and before any exit
   pdl_launch();
-  // the row tile is the slowest grid index: tiles beyond a request's rows (the grid covers the largest row count a
-  // call may have) are scheduled after every tile that has work, instead of holding its place in the first wave
-  // (a causal prefill has no such tiles to speak of, and its last tiles see the most context: those go first)
-  const int req_local = blockIdx.y, kvh = blockIdx.x;
-  const int tile = a.n_ext_max > 0 ? (int)blockIdx.z : (int)(gridDim.z - 1 - blockIdx.z);
+  // Grid = (KV head, row tile, request): the row tiles of a (request, KV head) are neighbours in launch order, so they run
+  // at the same time and the second one finds the K/V tiles the first one pulled in L2 (with the row tile as the slowest
+  // index a request of more than 128 rows streamed its context from HBM once per tile: twice the DRAM bytes).  A causal
+  // prefill's last tiles see the most context: those go first.
+  const int req_local = blockIdx.z, kvh = blockIdx.x;
+  const int tile = a.n_ext_max > 0 ? (int)blockIdx.y : (int)(gridDim.y - 1 - blockIdx.y);
   const int G = a.Hq / a.Hkv;
   const int4 info = a.req_info[req_local];          // {first token, token count, cache row, context length or -1}
   const int tok0 = info.x, n_tok = info.y, request = info.z;
@@ -399,7 +400,7 @@ void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a
     cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   });
   const int G = a.Hq / a.Hkv;
-  dim3 grid(a.Hkv, a.n_rows, (a.max_tokens_per_row * G + kRowsU - 1) / kRowsU);
+  dim3 grid(a.Hkv, (a.max_tokens_per_row * G + kRowsU - 1) / kRowsU, a.n_rows);
   // the layer's draft-token caches as [positions of all requests, kv heads * hd] (a prefill has none: any valid map)
   CUtensorMap tkx = *tk, tvx = *tv;
   if (a.n_ext_max > 0) {
