@@ -186,7 +186,7 @@ def build_engine(w, dev, final_mask: str):
     return {"w": w, "weights": weights, "catalog": catalog, "hist": hist, "cat_dev": cat_dev, "eng": eng}
 
 
-def time_decode(ctx, mode, drafts, steps, warmup, flush, dist, world, dev, barrier):
+def time_decode(ctx, mode, drafts, steps, warmup, flush, dist, world, dev, barrier, adaptive=False):
     """W warm-up steps, then K timed steps (one CUDA-event pair per step, L2 flushed before each, outside the events);
     then the per-class pass.  Returns the numbers of one workload."""
     import torch
@@ -197,6 +197,7 @@ def time_decode(ctx, mode, drafts, steps, warmup, flush, dist, world, dev, barri
     hist_dev = hist_pinned.to(dev, non_blocking=True)
     nh_dev = nh_pinned.to(dev, non_blocking=True)
     eng.prefill(hist_dev, nh_dev)
+    eng.set_option(binding.OPT_ADAPTIVE_DRAFT, 1 if adaptive else 0)
     out = eng.alloc_outputs(w.batch, w.beam)
     items = w.batch * w.beam
     inject = None
@@ -371,6 +372,9 @@ def main():
     ap.add_argument("--probe-keys", type=int, default=0,
                     help="instead of the decode step, time the stand-alone hash-set probe (Eq. 5) on this many keys, "
                          "half of them catalogue items, and print its own JSON line")
+    ap.add_argument("--adaptive", action="store_true",
+                    help="mode 1 with NEZHA_OPT_ADAPTIVE_DRAFT: a request stops drafting after a round that gained nothing "
+                         "from its drafts (an engine policy; off by default, as in the library)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-workload", action="store_true",
                     help="skip the short runs of the other configurations that the default run adds under `per_workload`")
@@ -438,7 +442,9 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    res = time_decode(ctx, args.mode, args.drafts, args.steps, warmup, flush, dist, world, dev, barrier)
+    res = time_decode(ctx, args.mode, args.drafts, args.steps, warmup, flush, dist, world, dev, barrier, adaptive=args.adaptive)
+    if args.adaptive:
+        config["drafts"] += ", drafting switched off per request after a round without gain"
     clocks = sampler.stop()
     step, out, hist_pinned, nh_pinned = res["step"], res["out"], res["hist_pinned"], res["nh_pinned"]
 
@@ -495,11 +501,12 @@ def main():
             wn = synth.WORKLOADS[name]
             c2 = build_engine(wn, dev, args.final_mask)
             entry = {"workload": workload_label(wn)}
-            for label, mode, drafts in (("verified", 1, "natural"), ("verified_perfect_tree", 1, "perfect"),
+            for label, mode, drafts in (("verified", 1, "natural"), ("verified_adaptive", 1, "natural"),
+                                        ("verified_perfect_tree", 1, "perfect"),
                                         ("autoregressive", 2, "natural"), ("draft_only", 0, "natural")):
-                if name == "7b" and label == "verified" and args.mode == 1 and args.drafts == "natural":
+                if name == "7b" and label == "verified" and args.mode == 1 and args.drafts == "natural" and not args.adaptive:
                     continue                                   # the headline of this line
-                r2 = time_decode(c2, mode, drafts, 10, 3, flush, None, 1, dev, barrier)
+                r2 = time_decode(c2, mode, drafts, 10, 3, flush, None, 1, dev, barrier, adaptive=label == "verified_adaptive")
                 rf = r2["roofline"]
                 entry[label] = {"value": r2["value"], "ms_per_step": r2["ms_per_step"], "p50_ms": r2["p50_ms"],
                                 "rounds_per_step": r2["rounds_per_step"],

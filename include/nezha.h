@@ -201,12 +201,18 @@ nezha_status nezha_decode_with_draft_tree(nezha_ctx* ctx, int32_t batch, int32_t
  *                                  unless NEZHA_OPT_DRAFT_FILTER is 0) and in the primary model's beam search of modes 1 and 2
  *                                  (before the top-K).  Answered by the same table as NEZHA_OPT_FINAL_MASK 1, which holds the
  *                                  prefixes of every length.  Modes 1 and 2 still agree item for item.
+ *   NEZHA_OPT_ADAPTIVE_DRAFT    0 (default): mode 1 drafts in every round, as Algorithm 2 prints it
+ *                               1: a request whose round settled only the one level that the verification pass settles
+ *                                  anyway -- its drafts gained nothing -- stops drafting and finishes with plain
+ *                                  autoregressive steps (an engine policy; the paper has no counterpart).  The result does
+ *                                  not change; rounds, primary_tokens and the trace do.
  * Errors: NEZHA_ERR_ARG (unknown option or value). */
 #define NEZHA_OPT_DRAFT_TRANSITION 0
 #define NEZHA_OPT_DRAFT_INPUTS 1
 #define NEZHA_OPT_DRAFT_FILTER 2
 #define NEZHA_OPT_FINAL_MASK 3
 #define NEZHA_OPT_LEVEL_FILTER 4
+#define NEZHA_OPT_ADAPTIVE_DRAFT 5
 nezha_status nezha_set_option(nezha_ctx* ctx, int32_t option, int32_t value);
 
 /* ---- stage-wise entry points (the same kernels as nezha_decode, one step at a time) ------------------- */

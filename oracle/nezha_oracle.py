@@ -511,7 +511,8 @@ def accepted_lengths(tuples: Sequence[Tuple[int, ...]], true_sets: List[List[Bea
 def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: int, valid: Optional[ValidSet],
                        drafts_round1: Optional[List[Tuple[int, ...]]] = None,
                        draft_tree_round1: Optional[List[List[Tuple[int, ...]]]] = None,
-                       use_drafts: bool = True, every_level: bool = False) -> Tuple[List[List[Beam]], SpecStats]:
+                       use_drafts: bool = True, every_level: bool = False,
+                       adaptive: bool = False) -> Tuple[List[List[Beam]], SpecStats]:
     """Algorithm 2 with the readings listed in the module header.
 
     B_1 comes from the prefill hidden state h_0.  Each round, with m levels settled (true beams B_m):
@@ -528,7 +529,9 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
       * accepted length of a drafted tuple = the largest i <= (level reached) whose i-prefix is a beam of B_i.
     Every B_j is computed from M_p's logits only, so the result equals ar_beam_search whatever the drafts.
     use_drafts=False gives L-1 rounds of plain autoregressive steps.  every_level: the validity filter at every level,
-    in the draft head's search and in the primary model's alike.
+    in the draft head's search and in the primary model's alike.  adaptive: a request stops drafting once a round has
+    gained nothing from its drafts -- it settled only the one level that the pass settles anyway -- and finishes with plain
+    autoregressive steps (an engine policy, not part of Algorithm 2; the result is Algorithm 1's either way).
     """
     s = model.s
     L = s.L
@@ -538,11 +541,12 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
                      valid if (L == 1 or every_level) else None)
     true_sets.append(B)
     m = 1
+    speculate = True
     while m < L:
         stats.rounds += 1
         # ---- draft (Algorithm 2, drafting step): tree[j - 1] = drafted nodes of level j
         tree: List[List[Tuple[int, ...]]] = [[] for _ in range(L)]
-        if not use_drafts:
+        if not use_drafts or not speculate:
             pass
         elif stats.rounds == 1 and draft_tree_round1 is not None:
             tree = [[tuple(int(c) for c in t) for t in lv] for lv in draft_tree_round1]
@@ -567,6 +571,8 @@ def speculative_decode(model: PrimaryModel, head: DraftHead, req: Request, K: in
         stats.primary_tokens += len(true_sets[m - 1]) + sum(nodes)
         stats.accepted_len.append(accepted_lengths(tree[L - 1], true_sets, j))
         stats.reject_level.append(j)
+        if adaptive:
+            speculate = j - m >= 2
         m = j
     return true_sets, stats
 

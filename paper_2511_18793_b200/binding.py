@@ -20,7 +20,7 @@ lib = C.CDLL(LIB_PATH)
 
 MAX_LEVELS = 8
 MODE_DRAFT, MODE_VERIFIED, MODE_AR = 0, 1, 2
-OPT_DRAFT_TRANSITION, OPT_DRAFT_INPUTS, OPT_DRAFT_FILTER, OPT_FINAL_MASK, OPT_LEVEL_FILTER = 0, 1, 2, 3, 4
+OPT_DRAFT_TRANSITION, OPT_DRAFT_INPUTS, OPT_DRAFT_FILTER, OPT_FINAL_MASK, OPT_LEVEL_FILTER, OPT_ADAPTIVE_DRAFT = 0, 1, 2, 3, 4, 5
 STATUS_NAMES = ["OK", "ERR_ARG", "ERR_STATE", "ERR_ARENA_TOO_SMALL", "ERR_CUDA", "ERR_HASH_FULL", "ERR_CATALOG",
                 "ERR_UNSUPPORTED"]
 

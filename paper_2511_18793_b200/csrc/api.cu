@@ -89,6 +89,7 @@ struct nezha_ctx {
   bool use_graphs;
   int opt_transition, opt_inputs, opt_filter;   // nezha_set_option (ablations of the draft head)
   int opt_mask;             // nezha_set_option: 0 = the primary model's last-level mask probes the hash set, 1 (default) = it reads the prefix map
+  int opt_adaptive;         // nezha_set_option: 1 = a request stops drafting after a round that gained nothing from its drafts
   int opt_level_filter;     // nezha_set_option: 1 = validity filter at every level (prefixes of valid IDs), 0 (default) = last level only
   int m_expected;           // tokens the current verify pass is expected to hold (0 = unknown); shapes GEMM tiling only
   int m_seen[kMaxLevels + 1];   // tokens each round of the last decode call processed, rounded up to a row tile
@@ -258,6 +259,7 @@ size_t carve(nezha_ctx* c) {
   e.tb_count = cv.take<int>((size_t)(c->L + 1) * c->Bmax);
   e.tb_anc = cv.take<int>(lbk * c->L); e.tb_self = cv.take<int>(lbk); e.tb_src = cv.take<int>(lbk);
   e.row_m = cv.take<int>(c->Bmax); e.row_cur = cv.take<int>(c->Bmax); e.row_P = cv.take<int>(c->Bmax);
+  e.row_m_start = cv.take<int>(c->Bmax); e.row_spec = cv.take<int>(c->Bmax);
   e.dw_codes = cv.take<int>(lbk * c->L); e.dw_score = cv.take<float>(lbk); e.dw_parent = cv.take<int>(lbk);
   e.dw_count = cv.take<int>((size_t)(c->L + 1) * c->Bmax);
   e.d_m = cv.take<int>(c->Bmax);
@@ -491,13 +493,16 @@ void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_le
 
 nezha_status pending_device_error(nezha_ctx* c) {
   int st = 0;
-  NZ_CUDA(c, cudaMemcpyAsync(c->host_counters + 8, c->es.status, sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  NZ_CUDA(c, cudaMemcpyAsync(c->host_counters + 8, c->es.status, 4 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   NZ_CUDA(c, cudaStreamSynchronize(c->st));
   st = c->host_counters[8];
-  if (st) NZ_CUDA(c, cudaMemsetAsync(c->es.status, 0, sizeof(int), c->st));
+  if (st) NZ_CUDA(c, cudaMemsetAsync(c->es.status, 0, 4 * sizeof(int), c->st));
   if (st & kStHashFull) return fail(c, NEZHA_ERR_HASH_FULL, "hash set insertion exhausted its probe bound");
   if (st & kStBadCode) return fail(c, NEZHA_ERR_CATALOG, "a code outside [0, T_l) was given");
-  if (st) return fail(c, NEZHA_ERR_CUDA, "a bounded device-side wait expired (kernel gave up and returned)");
+  if (st)      // a kernel that records where it gave up leaves three more words (0 if it does not)
+    return fail(c, NEZHA_ERR_CUDA, "a bounded device-side wait expired (kernel gave up and returned); where: " +
+                                       std::to_string(c->host_counters[9]) + " " + std::to_string(c->host_counters[10]) + " " +
+                                       std::to_string(c->host_counters[11]));
   return NEZHA_OK;
 }
 
@@ -559,7 +564,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
   const int R = L - 1;
   auto key_of = [&](int segment) {
     std::array<uintptr_t, 16> k{};
-    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20 | (is_tree ? 1 : 0) << 24 | c->opt_level_filter << 25);
+    k[0] = (uintptr_t)segment; k[1] = (uintptr_t)batch; k[2] = (uintptr_t)K; k[3] = (uintptr_t)(mode | c->opt_transition << 8 | c->opt_inputs << 12 | c->opt_filter << 16 | c->opt_mask << 20 | (is_tree ? 1 : 0) << 24 | c->opt_level_filter << 25 | c->opt_adaptive << 26);
     k[4] = (uintptr_t)drafts; k[5] = (uintptr_t)n_draft; k[6] = (uintptr_t)out_codes; k[7] = (uintptr_t)out_scores;
     k[8] = (uintptr_t)out_count; k[9] = (uintptr_t)tr.drafts; k[10] = (uintptr_t)tr.n_draft; k[11] = (uintptr_t)tr.accepted_len;
     k[12] = (uintptr_t)tr.level_reached; k[13] = (uintptr_t)tr.beams ^ ((uintptr_t)tr.tree_codes << 1);
@@ -630,7 +635,7 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
         s.out_count = e.tb_count + (size_t)(n + 1) * c->Bmax;
         launch_select_advance(s, e, n, K, out_codes, out_scores, out_count, c->st);
       }
-      launch_round_end(e, batch, K, round, tr, c->st);
+      launch_round_end(e, batch, K, round, tr, mode == NEZHA_MODE_VERIFIED ? c->opt_adaptive : 0, c->st);
       cudaMemcpyAsync(c->host_counters + 16 + 8 * round, e.counters, 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st);
     });
     c->m_expected = 0;
@@ -694,7 +699,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
   c->chains_now = 0;
-  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 1; c->opt_level_filter = 0;
+  c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 1; c->opt_level_filter = 0; c->opt_adaptive = 0;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
   c->arena = (char*)arena; c->arena_bytes = arena_bytes;
@@ -878,6 +883,9 @@ nezha_status nezha_set_option(nezha_ctx* c, int32_t option, int32_t value) {
     case NEZHA_OPT_FINAL_MASK:
       if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: final mask must be 0 or 1");
       c->opt_mask = value; break;
+    case NEZHA_OPT_ADAPTIVE_DRAFT:
+      if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: adaptive drafting must be 0 or 1");
+      c->opt_adaptive = value; break;
     case NEZHA_OPT_LEVEL_FILTER:
       if (value != 0 && value != 1) return fail(c, NEZHA_ERR_ARG, "nezha_set_option: level filter must be 0 or 1");
       c->opt_level_filter = value; break;

@@ -17,6 +17,7 @@
 // same loop; a row masks them with the bit set of the positions it may see (its own tuple's codes).  At the end each
 // thread normalises and stores its row.  Every mbarrier wait is bounded (abort flag, error status, TMEM freed).
 #include <math.h>
+#include <stdlib.h>
 
 #include "gemm_epilogue.cuh"
 
@@ -33,25 +34,51 @@ constexpr int kRingU = 2;          // K tiles in flight, and V tiles in flight (
 constexpr int kThreadsU = 192;     // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: softmax (one thread per row)
 constexpr float kRaise = 8.f;      // the reference maximum follows the true one only in steps larger than this (log2 units)
 
-template <int HD> struct UmmaCfg {
+// PT ("P in TMEM"): the softmax threads write P straight back into the TMEM columns its scores came from (bf16 pairs, the
+// A operand of the second product read from TMEM) instead of through a shared-memory buffer, and S is double-buffered:
+// S_{j+2} = Q K_{j+2}^T is issued right behind P_j V_j, the softmax of tile j + 1 never waits for the P V product of tile
+// j, and the 16 KB that P took hold a third V slot.  Without PT: one S, one P buffer in shared memory (three CTAs per SM
+// at hd = 64, where TMEM is what limits the PT form to two).
+template <int HD, bool PT> struct UmmaCfg {
+  static constexpr int kKRing = kRingU, kVRing = PT ? 3 : kRingU;
   static constexpr int kQBytes = kRowsU * HD * 2;
-  static constexpr int kPBytes = kRowsU * kPosU * 2;
+  static constexpr int kPBytes = PT ? 0 : kRowsU * kPosU * 2;
   static constexpr int kTileBytes = kPosU * HD * 2;            // one K (or V) tile
-  // One S accumulator, one P buffer, two K and two V slots: 65 KB (hd 64) / 113 KB (hd 128) per CTA, so that three /
-  // two CTAs share an SM.  A CTA is a chain (S -> softmax -> P V per tile) whose softmax takes most of the tile's time;
-  // the S product of the next tile still runs under it (the scores leave TMEM at the start of the softmax), and
-  // concurrency comes from the CTAs that share the SM rather than from second buffers.
   // Two CTAs of the hd = 128 shape fit an SM only if each stays below (228 KB - 2 x 1 KB reserved) / 2 = 113 KB: the tiles
-  // alone are 112 KB, so the barriers get 128 bytes and the alignment slack 512 (the dynamic array is declared with the
+  // alone are 112 KB, so the barriers get 192 bytes and the alignment slack 512 (the dynamic array is declared with the
   // tiles' 1024-byte alignment; the kernel checks the slack it really needs and reports instead of overrunning).
-  static constexpr int kBarBytes = 128, kSlack = 512;
-  static constexpr int kTilesBytes = kQBytes + kPBytes + 2 * kRingU * kTileBytes;
+  static constexpr int kBarBytes = 192, kSlack = 512;
+  static constexpr int kTilesBytes = kQBytes + kPBytes + (kKRing + kVRing) * kTileBytes;
   static constexpr int kSmemBytes = kTilesBytes + kBarBytes + kSlack;
-  static constexpr int kTmemCols = HD == 64 ? 128 : 256;       // S: 64 columns, O: HD columns; a power of two
+  // TMEM columns.  Plain: S at 0 (64), O at 64 (HD).  PT: S_0 / P_0 at 0, S_1 / P_1 at 64, O at 128.
+  static constexpr int kTmemCols = PT ? 256 : (HD == 64 ? 128 : 256);
+  static constexpr uint32_t kColO = PT ? 128 : 64;
+  static constexpr int kCtasPerSm = PT ? 2 : (HD == 64 ? 3 : 2);
   static constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kPosU >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
   static constexpr uint32_t kIdescPV =
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) /* B is N-major */ | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(kRowsU >> 4) << 24);
 };
+
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (128 rows = lanes, K along the columns, two bf16 per 32-bit cell) is read
+// from tensor memory.
+__device__ __forceinline__ void tc_mma_a_tmem(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_st32_bits(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 
 // N-major (MN-major) operand tile with the 128-byte swizzle: rows of 64 elements along N, 8-row groups along K 1024 B
 // apart (SBO), 64-element groups along N `lbo` bytes apart (LBO).
@@ -101,16 +128,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return r;
 }
 
-template <int HD>
-__global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
+template <int HD, bool PT>
+__global__ void __launch_bounds__(kThreadsU, UmmaCfg<HD, PT>::kCtasPerSm) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
                                                              const __grid_constant__ CUtensorMap tmV,
                                                              const __grid_constant__ CUtensorMap tmKx,
                                                              const __grid_constant__ CUtensorMap tmVx, AttnArgs a, int* status) {
-  using C = UmmaCfg<HD>;
-  constexpr int S = kRingU;
+  using C = UmmaCfg<HD, PT>;
+  constexpr int SK = C::kKRing, SV = C::kVRing;     // K and V ring lengths
   constexpr int NH = HD / 64;                       // 64-column sub-tiles of a K / V / Q tile
   constexpr int KS = HD / 16;                       // k-steps of Q K^T
-  constexpr uint32_t kColS = 0, kColO = 64;         // TMEM columns: S at 0, O at 64
+  constexpr uint32_t kColO = C::kColO;              // TMEM columns: S (and P) buffer b at 64 b, O behind them
 
   pdl_wait();                                       // before the first global read and before any exit
   pdl_launch();
@@ -143,21 +170,41 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
     return;
   }
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_base = base, p_base = base + C::kQBytes, k_base = p_base + C::kPBytes, v_base = k_base + S * C::kTileBytes;
-  const uint32_t bar_base = v_base + S * C::kTileBytes;
+  const uint32_t q_base = base, p_base = base + C::kQBytes, k_base = p_base + C::kPBytes, v_base = k_base + SK * C::kTileBytes;
+  const uint32_t bar_base = v_base + SV * C::kTileBytes;
   auto k_full = [&](int s) { return bar_base + 8u * s; };
-  auto k_empty = [&](int s) { return bar_base + 8u * (S + s); };
-  auto v_full = [&](int s) { return bar_base + 8u * (2 * S + s); };
-  auto v_empty = [&](int s) { return bar_base + 8u * (3 * S + s); };
-  // one phase per tile on each of these: tile j completes phase j (parity j & 1)
-  const uint32_t s_full = bar_base + 8u * (4 * S), s_free = s_full + 8u, p_full = s_full + 16u, pv_done = s_full + 24u;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - base) + 8 * (4 * S + 4));
+  auto k_empty = [&](int s) { return bar_base + 8u * (SK + s); };
+  auto v_full = [&](int s) { return bar_base + 8u * (2 * SK + s); };
+  auto v_empty = [&](int s) { return bar_base + 8u * (2 * SK + SV + s); };
+  // Plain: one phase per tile on each of s_full(0), s_free, p_full(0), pv_done (tile j completes phase j).  PT: s_full(b)
+  // and p_full(b) belong to S / P buffer b = j & 1 (tile j completes phase j >> 1 of them); s_free is not used.
+  const uint32_t bar_misc = bar_base + 8u * (2 * SK + 2 * SV);
+  auto s_full = [&](int b) { return bar_misc + 8u * b; };
+  auto p_full = [&](int b) { return bar_misc + 16u + 8u * b; };
+  const uint32_t s_free = bar_misc + 32u;
+  // "P_j V_j is complete".  Plain: one barrier, one phase per tile, every softmax warp waits for every phase.  PT: the
+  // softmax warps wait for it only before a rescale of O and at the end, and may then be up to two products ahead of or
+  // behind the tensor core -- more than a parity can tell apart on one barrier -- so the products alternate between two
+  // barriers (tile j completes phase j >> 1 of barrier j & 1), on each of which a waiter is never more than one phase off.
+  auto pv_done = [&](int j) { return bar_misc + 40u + (PT ? 8u * (uint32_t)(j & 1) : 0u); };
+  auto pv_parity = [&](int j) { return (uint32_t)(PT ? (j >> 1) : j) & 1u; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_misc - base) + 56);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  static_assert(8 * (2 * C::kKRing + 2 * C::kVRing) + 56 + 8 <= C::kBarBytes, "barrier area");
+  // where a bounded wait gave up (first one wins): status[1] = wait site, tile and warp; status[2] = the CTA; status[3] = its sizes
+  auto gave_up = [&](int site, int j) {
+    if (atomicCAS(status + 1, 0, site * 100000 + j * 100 + (int)(threadIdx.x >> 5) * 10 + (PT ? 1 : 0)) == 0) {
+      status[2] = (int)(blockIdx.x + 100 * blockIdx.y + 10000 * blockIdx.z) + 1;
+      status[3] = NT * 100000 + R;
+    }
+  };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
-    mbar_init(s_full, 1); mbar_init(s_free, 4); mbar_init(p_full, 4); mbar_init(pv_done, 1);
+    for (int s = 0; s < SK; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
+    for (int s = 0; s < SV; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 4); }
+    mbar_init(s_free, 4); mbar_init(pv_done(0), 1); mbar_init(pv_done(1), 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -197,61 +244,68 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
       int t = 0, k_issued = 0, v_issued = 0;
       bool ok = true;
       for (; t < NT; ++t) {
-        const int s = t % S;
-        const uint32_t par = (uint32_t)((t / S) - 1) & 1u;
+        const int sk = t % SK, sv = t % SV;
         const bool ctx_tile = t < n_tiles;
         const int y = ctx_tile ? kv_row0 + t * kPosU : request * a.ext_positions + (t - n_tiles) * kPosU;
         const int x0 = ctx_tile ? 0 : kvh * HD;      // the draft cache is [positions, kv heads * hd]: this head's columns
-        if (t >= S && !mbar_wait_or_abort(k_empty(s), par, abort_flag)) { ok = false; break; }
-        mbar_expect_tx(k_full(s), C::kTileBytes);
+        if (t >= SK && !mbar_wait_or_abort(k_empty(sk), (uint32_t)((t / SK) - 1) & 1u, abort_flag)) { gave_up(1, t); ok = false; break; }
+        mbar_expect_tx(k_full(sk), C::kTileBytes);
 #pragma unroll
         for (int h = 0; h < NH; ++h)
-          tma_load_2d(k_base + s * C::kTileBytes + h * (kPosU * 128), ctx_tile ? &tmK : &tmKx, x0 + h * 64, y, k_full(s));
+          tma_load_2d(k_base + sk * C::kTileBytes + h * (kPosU * 128), ctx_tile ? &tmK : &tmKx, x0 + h * 64, y, k_full(sk));
         ++k_issued;
-        if (t >= S && !mbar_wait_or_abort(v_empty(s), par, abort_flag)) { ok = false; break; }
-        mbar_expect_tx(v_full(s), C::kTileBytes);
+        if (t >= SV && !mbar_wait_or_abort(v_empty(sv), (uint32_t)((t / SV) - 1) & 1u, abort_flag)) { gave_up(2, t); ok = false; break; }
+        mbar_expect_tx(v_full(sv), C::kTileBytes);
 #pragma unroll
         for (int h = 0; h < NH; ++h)
-          tma_load_2d(v_base + s * C::kTileBytes + h * (kPosU * 128), ctx_tile ? &tmV : &tmVx, x0 + h * 64, y, v_full(s));
+          tma_load_2d(v_base + sv * C::kTileBytes + h * (kPosU * 128), ctx_tile ? &tmV : &tmVx, x0 + h * 64, y, v_full(sv));
         ++v_issued;
       }
       if (!ok) {                                     // drain the copies still in flight before the CTA's memory goes away
         *abort_flag = 1;
-        for (int j = max(0, k_issued - S); j < k_issued; ++j) mbar_wait(k_full(j % S), (j / S) & 1);
-        for (int j = max(0, v_issued - S); j < v_issued; ++j) mbar_wait(v_full(j % S), (j / S) & 1);
+        for (int j = max(0, k_issued - SK); j < k_issued; ++j) mbar_wait(k_full(j % SK), (j / SK) & 1);
+        for (int j = max(0, v_issued - SV); j < v_issued; ++j) mbar_wait(v_full(j % SV), (j / SV) & 1);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = true;
-      auto issue_s = [&](int j) {                    // S_j = Q K_j^T (the one S accumulator)
-        const int s = j % S;
-        if (!mbar_wait_or_abort(k_full(s), (uint32_t)(j / S) & 1u, abort_flag)) return false;
-        if (j >= 1 && !mbar_wait_or_abort(s_free, (uint32_t)(j - 1) & 1u, abort_flag)) return false;   // scores of tile j - 1 are in registers
+      auto issue_s = [&](int j) {                    // S_j = Q K_j^T into S buffer (PT ? j & 1 : 0)
+        const int s = j % SK, b = PT ? (j & 1) : 0;
+        if (!mbar_wait_or_abort(k_full(s), (uint32_t)(j / SK) & 1u, abort_flag)) { gave_up(3, j); return false; }
+        // plain: the scores of tile j - 1 must be in registers.  PT: buffer b last held S_{j-2} / P_{j-2}, whose P V product
+        // was issued before this one, and the tensor core runs a CTA's products in issue order: nothing to wait for.
+        if (!PT && j >= 1 && !mbar_wait_or_abort(s_free, (uint32_t)(j - 1) & 1u, abort_flag)) { gave_up(4, j); return false; }
         tc_fence_after();
         const uint32_t kt = k_base + s * C::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks)
-          tc_mma(tmem_base + kColS, smem_desc(q_base + (ks >> 2) * (kRowsU * 128) + (ks & 3) * 32),
+          tc_mma(tmem_base + 64u * b, smem_desc(q_base + (ks >> 2) * (kRowsU * 128) + (ks & 3) * 32),
                  smem_desc(kt + (ks >> 2) * (kPosU * 128) + (ks & 3) * 32), C::kIdescS, ks > 0 ? 1u : 0u);
         tc_commit(k_empty(s));                       // K_j may be overwritten
-        tc_commit(s_full);
+        tc_commit(s_full(b));
         return true;
       };
       if (NT > 0) ok = issue_s(0);
+      if (PT && ok && NT > 1) ok = issue_s(1);
       for (int j = 0; j < NT && ok; ++j) {
-        if (j + 1 < NT && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
-        if (!mbar_wait_or_abort(p_full, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
-        if (!mbar_wait_or_abort(v_full(j % S), (uint32_t)(j / S) & 1u, abort_flag)) { ok = false; break; }
+        if (!PT && j + 1 < NT && !issue_s(j + 1)) { ok = false; break; }   // runs under the softmax of tile j
+        const int b = PT ? (j & 1) : 0;
+        if (!mbar_wait_or_abort(p_full(b), (uint32_t)(PT ? (j >> 1) : j) & 1u, abort_flag)) { gave_up(5, j); ok = false; break; }
+        if (!mbar_wait_or_abort(v_full(j % SV), (uint32_t)(j / SV) & 1u, abort_flag)) { gave_up(6, j); ok = false; break; }
         tc_fence_after();
-        const uint32_t vt = v_base + (j % S) * C::kTileBytes;
+        const uint32_t vt = v_base + (j % SV) * C::kTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < kPosU / 16; ++ks)
-          tc_mma(tmem_base + kColO, smem_desc(p_base + ks * 32), smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128), C::kIdescPV,
-                 (j > 0 || ks > 0) ? 1u : 0u);
-        tc_commit(v_empty(j % S));                   // V_j may be overwritten
-        tc_commit(pv_done);                          // O holds tiles 0..j, and P may be overwritten
+        for (int ks = 0; ks < kPosU / 16; ++ks) {
+          const uint64_t dv = smem_desc_nmajor(vt + ks * (16 * 128), kPosU * 128);
+          const uint32_t acc = (j > 0 || ks > 0) ? 1u : 0u;
+          if (PT) tc_mma_a_tmem(tmem_base + kColO, tmem_base + 64u * b + 8u * ks, dv, C::kIdescPV, acc);
+          else tc_mma(tmem_base + kColO, smem_desc(p_base + ks * 32), dv, C::kIdescPV, acc);
+        }
+        tc_commit(v_empty(j % SV));                  // V_j may be overwritten
+        tc_commit(pv_done(j));                       // O holds tiles 0..j (and, plain, P may be overwritten)
+        if (PT && j + 2 < NT && !issue_s(j + 2)) { ok = false; break; }   // behind P_j V_j, into the buffer it has just read
       }
       if (!ok) *abort_flag = 1;
     }
@@ -270,25 +324,29 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
       xpos[e] = off >= 0 ? (int)((off - (long long)request * a.ext_req_stride) / a.ext_pos_stride) : -1;
     }
     for (int j = 0; j < NT; ++j) {
-      const uint32_t par = (uint32_t)j & 1u, par_prev = par ^ 1u;
-      ok = warp_wait(s_full, par, abort_flag, lane);
-      if (!ok) break;
+      const int sb = PT ? (j & 1) : 0;               // S / P buffer of this tile
+      const uint32_t par = (uint32_t)(PT ? (j >> 1) : j) & 1u;
+      const uint32_t col_s = 64u * sb;
+      ok = warp_wait(s_full(sb), par, abort_flag, lane);
+      if (!ok) { if (lane == 0) gave_up(7, j); break; }
       if (warp_dead) {                               // (its P rows stay whatever they are: O rows nobody reads)
-        if (lane == 0) mbar_arrive(s_free);
-        if (j >= 1) {
-          ok = warp_wait(pv_done, par_prev, abort_flag, lane);
-          if (!ok) break;
+        if (!PT) {
+          if (lane == 0) mbar_arrive(s_free);
+          if (j >= 1) {
+            ok = warp_wait(pv_done(j - 1), pv_parity(j - 1), abort_flag, lane);
+            if (!ok) { if (lane == 0) gave_up(8, j); break; }
+          }
         }
-        if (lane == 0) mbar_arrive(p_full);
+        if (lane == 0) mbar_arrive(p_full(sb));
         continue;
       }
       tc_fence_after();
       float sv[kPosU];
-      tmem_ld32(tmem_base + lane_addr + kColS, sv);
-      tmem_ld32(tmem_base + lane_addr + kColS + 32u, sv + 32);
+      tmem_ld32(tmem_base + lane_addr + col_s, sv);
+      tmem_ld32(tmem_base + lane_addr + col_s + 32u, sv + 32);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(s_free);            // the scores are in registers: S may take tile j + 1
+      if (!PT && lane == 0) mbar_arrive(s_free);     // the scores are in registers: S may take tile j + 1
       if (j >= n_tiles) {                            // a tile of draft positions: the row's own mask
         unsigned long long mk = 0ull;
 #pragma unroll
@@ -330,11 +388,14 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
       const float rs = rs_lo + rs_hi;
       l_run = l_run * corr + rs;
       m_ref = m_new;
-      if (j >= 1) {                                  // the PV product of tile j - 1 is done: P is free, O holds every earlier tile
-        ok = warp_wait(pv_done, par_prev, abort_flag, lane);
-        if (!ok) break;
+      // Plain: the P V product of tile j - 1 must be done before P is overwritten.  PT: P_j has a buffer of its own (last
+      // read by P_{j-2} V_{j-2}, which completed before S_j did); only a rescale of O has to wait for P_{j-1} V_{j-1}.
+      const bool rescale = j > 0 && __any_sync(0xffffffffu, raise);
+      if (j >= 1 && (!PT || rescale)) {
+        ok = warp_wait(pv_done(j - 1), pv_parity(j - 1), abort_flag, lane);
+        if (!ok) { if (lane == 0) gave_up(9, j); break; }
       }
-      if (j > 0 && __any_sync(0xffffffffu, raise)) { // rescale O
+      if (rescale) {                                 // rescale O
         tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < HD / 32; ++c) {
@@ -345,17 +406,22 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
           tmem_st32(tmem_base + lane_addr + kColO + (uint32_t)(c * 32), ov);
         }
       }
+      if (PT) {                                      // P over the first half of the columns its scores came from
+        tmem_st32_bits(tmem_base + lane_addr + col_s, pk);
+      } else {
 #pragma unroll
-      for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(gen_base + (p_base - base) + row * 128 + ((c ^ (row & 7)) << 4)) =
-            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-      fence_async_smem();
+        for (int c = 0; c < 8; ++c)
+          *reinterpret_cast<uint4*>(gen_base + (p_base - base) + row * 128 + ((c ^ (row & 7)) << 4)) =
+              make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        fence_async_smem();
+      }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full);
+      if (lane == 0) mbar_arrive(p_full(sb));
     }
     if (ok && NT > 0) {
-      ok = warp_wait(pv_done, (uint32_t)(NT - 1) & 1u, abort_flag, lane);
+      ok = warp_wait(pv_done(NT - 1), pv_parity(NT - 1), abort_flag, lane);
+      if (!ok && lane == 0) gave_up(10, NT);
       tc_fence_after();
     }
     if (!ok) { if (lane == 0) *abort_flag = 1; }
@@ -392,12 +458,12 @@ __global__ void __launch_bounds__(kThreadsU, HD == 64 ? 3 : 2) attn_umma_kernel(
   if (threadIdx.x == 0 && *abort_flag) atomicOr(status, kStInternal);
 }
 
-template <int HD>
+template <int HD, bool PT>
 void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a, cudaStream_t st) {
-  using C = UmmaCfg<HD>;
+  using C = UmmaCfg<HD, PT>;
   static PerDeviceOnce configured;
   configured.run([] {
-    cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    cudaFuncSetAttribute(attn_umma_kernel<HD, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   });
   const int G = a.Hq / a.Hkv;
   dim3 grid(a.Hkv, (a.max_tokens_per_row * G + kRowsU - 1) / kRowsU, a.n_rows);
@@ -411,15 +477,24 @@ void launch_umma(const CUtensorMap* tk, const CUtensorMap* tv, const AttnArgs& a
       return;
     }
   }
-  launch_pdl(attn_umma_kernel<HD>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, tkx, tvx, a, a.status);
+  launch_pdl(attn_umma_kernel<HD, PT>, grid, dim3(kThreadsU), C::kSmemBytes, st, *tk, *tv, tkx, tvx, a, a.status);
 }
 
 }  // namespace
 
 // tk / tv: tensor maps of the layer's context K and V caches with boxes of 64 positions x 64 columns.
 void launch_attention_umma(const AttnArgs& a, const CUtensorMap* tk, const CUtensorMap* tv, cudaStream_t st) {
-  if (a.hd == 64) launch_umma<64>(tk, tv, a, st);
-  else launch_umma<128>(tk, tv, a, st);
+  // P through TMEM with two S buffers pays where the CTA's chain S -> softmax -> P V is the bound: several row tiles per
+  // (request, KV head) at hd = 128 (measured: -7 % on the 7B shape's 240-row passes, -6.5 % on the 1.5B shape).  One-tile
+  // passes of the 7B shape are bound by HBM and lose 20 % with it (the two-slot K ring then has to run two tiles ahead);
+  // at hd = 64 it costs the third CTA per SM for nothing.  NEZHA_ATTN_PT = 0 / 1 forces it off / on.
+  static const int pt = getenv("NEZHA_ATTN_PT") ? atoi(getenv("NEZHA_ATTN_PT")) : 2;
+  const int G = a.Hq / a.Hkv;
+  const long long r_bound = (long long)a.max_tokens_per_row * G;
+  const long long r = a.rows_expected > 0 && a.rows_expected < r_bound ? a.rows_expected : r_bound;
+  const bool use_pt = pt == 1 || (pt == 2 && a.hd == 128 && r > kRowsU);
+  if (a.hd == 64) { if (use_pt) launch_umma<64, true>(tk, tv, a, st); else launch_umma<64, false>(tk, tv, a, st); }
+  else { if (use_pt) launch_umma<128, true>(tk, tv, a, st); else launch_umma<128, false>(tk, tv, a, st); }
 }
 
 }  // namespace nz

@@ -372,6 +372,8 @@ __global__ void init_decode_kernel(EngineState e, int batch) {
   e.tb_src[lvl_bk(e, 0, b, 0)] = -1;
   e.row_m[b] = 0;
   e.row_cur[b] = -1;
+  e.row_spec[b] = 1;
+  e.row_m_start[b] = 0;
   e.d_m[b] = e.L;
   for (int l = 0; l <= e.L; ++l) e.dw_count[(long long)l * e.Bmax + b] = 0;     // no draft tree yet
 }
@@ -395,7 +397,11 @@ __global__ void draft_init_kernel(EngineState e, int batch, int from_scratch, __
     }
   }
   const int m = e.row_m[b];
-  if (m >= e.L) { if (threadIdx.x == 0) { e.d_m[b] = e.L; e.dw_count[(long long)e.L * e.Bmax + b] = 0; } return; }
+  if (m >= e.L || !e.row_spec[b]) {              // finished, or its drafting is switched off: an empty tree this round
+    if (threadIdx.x == 0) e.d_m[b] = e.L;
+    if ((int)threadIdx.x <= e.L) e.dw_count[(long long)threadIdx.x * e.Bmax + b] = 0;
+    return;
+  }
   const int mm = from_scratch ? 0 : m;
   const int cnt = e.tb_count[mm * e.Bmax + b];
   for (int k = threadIdx.x; k < e.Kmax; k += blockDim.x) {
@@ -673,6 +679,7 @@ __global__ void nodes_count_kernel(EngineState e, int batch) {
   if (threadIdx.x == 0) {
     e.row_tok_count[b] = nb + n_alive;
     e.row_cur[b] = m;
+    e.row_m_start[b] = m;
   }
 }
 
@@ -876,7 +883,9 @@ __global__ void __launch_bounds__(512) select_advance_kernel(SelectArgs a, Engin
 
 // End of a round: accepted length of every draft = the largest i <= (level reached) with D[k][0..i) in B_i;
 // trace outputs; counters for the host (unfinished requests, primary tokens, accepted levels).
-__global__ void round_end_kernel(EngineState e, int batch, int K, int round, nezha_trace tr, int m_before_unused) {
+// adaptive: a request whose round settled only the one level that the pass settles anyway gained nothing from its drafts
+// and stops drafting (its remaining rounds are plain autoregressive steps).
+__global__ void round_end_kernel(EngineState e, int batch, int K, int round, nezha_trace tr, int adaptive) {
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x;
@@ -924,6 +933,7 @@ __global__ void round_end_kernel(EngineState e, int batch, int K, int round, nez
   if (threadIdx.x == 0) {
     if (tr.n_draft) tr.n_draft[tro] = took_part ? nd : -1;
     if (tr.level_reached) tr.level_reached[tro] = took_part ? m_now : -1;
+    if (took_part && adaptive) e.row_spec[b] = (m_now - e.row_m_start[b] >= 2) ? 1 : 0;
     if (m_now < L) atomicAdd(&e.counters[0], 1);
     atomicAdd(&e.counters[1], e.row_tok_count[b]);
     atomicAdd(&e.counters[2], acc_sum);
@@ -1092,9 +1102,9 @@ void launch_select_advance(const SelectArgs& a, const EngineState& e, int n, int
   else if (a.T <= 512) launch_pdl(select_advance_kernel<16>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
   else launch_pdl(select_advance_kernel<32>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
 }
-void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, cudaStream_t st) {
+void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, int adaptive, cudaStream_t st) {
   LaunchScope ls(kcAccept, st);
-  launch_pdl(round_end_kernel, dim3(batch), dim3(64), 0, st, e, batch, K, round, tr, 0);
+  launch_pdl(round_end_kernel, dim3(batch), dim3(64), 0, st, e, batch, K, round, tr, adaptive);
 }
 void launch_write_out(const int* codes, const float* score, const int* count, int stride, int L, int batch, int K,
                       int* out_codes, float* out_score, int* out_count, cudaStream_t st) {

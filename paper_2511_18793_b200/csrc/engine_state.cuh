@@ -26,6 +26,8 @@ struct EngineState {
   int* row_m;       // [Bmax] levels settled (L = row finished)
   int* row_cur;     // [Bmax] level whose beams have logits in the current pass, -1 = row stopped this round
   int* row_P;       // [Bmax] context length of the row (BOS + history tokens)
+  int* row_m_start; // [Bmax] levels the row had settled when the current round began
+  int* row_spec;    // [Bmax] 1: the draft head drafts for the row in the next round (always 1 unless the adaptive policy is on)
 
   // The round's draft tree, [L+1][Bmax][Kmax]([L]): level l holds the drafted nodes with l codes (the draft head's beam
   // set of that level, or the distinct l-prefixes of caller-supplied tuples); dw_parent = slot of the node's parent in
@@ -100,7 +102,7 @@ void launch_nodes_from_prefixes(const EngineState& e, int batch, int n_beams, in
                                 cudaStream_t st);
 void launch_advance(const EngineState& e, int batch, int n, int K, int* out_codes, float* out_score, int* out_count,
                     cudaStream_t st);
-void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, cudaStream_t st);
+void launch_round_end(const EngineState& e, int batch, int K, int round, const nezha_trace& tr, int adaptive, cudaStream_t st);
 void launch_write_out(const int* codes, const float* score, const int* count, int stride, int L, int batch, int K,
                       int* out_codes, float* out_score, int* out_count, cudaStream_t st);
 void launch_copy_logits(const float* src, long long row_stride, int col_off, const int* row_index, int row_mul,

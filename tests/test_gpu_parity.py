@@ -482,6 +482,70 @@ def test_validity_filter_at_every_level(name):
     assert torch.equal(again["codes"], base[1]["codes"])
 
 
+@pytest.mark.parametrize("name", ["tiny", "small_cut"])
+def test_adaptive_drafting(name):
+    """NEZHA_OPT_ADAPTIVE_DRAFT = 1: a request stops drafting after a round that gained nothing.  Same items as without it
+    and as plain decoding; rounds, tokens and accepted lengths as the oracle's with the same policy (tiny: natural drafts
+    and seeded corrupted drafts); never more tokens than without it; the walk replayed from the trace."""
+    w = {"tiny": synth.WORKLOADS["tiny"],
+         "small_cut": synth.scaled(synth.WORKLOADS["small"], n_layers=2, n_items=100_000, batch=6, n_hist=20)}[name]
+    case = Case(w).prefill()
+    model, head, V = case.oracle
+    K = w.beam
+    plain = case.eng.decode(K, mode=1, trace=True)
+    ar = case.eng.decode(K, mode=2, trace=True)
+    case.eng.set_option(5, 1)
+    out = case.eng.decode(K, mode=1, trace=True)
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
+    assert out["stats"].primary_tokens <= plain["stats"].primary_tokens
+    check_walk_against_trace(out, w.batch, w.L)
+    tr = {k: v.cpu().numpy() for k, v in out["trace"].items()}
+    # the policy itself, from the trace: a round drafts (the draft head's tree has nodes) iff every earlier round of the
+    # request settled at least two levels
+    for b in range(w.batch):
+        spec, m = True, 1
+        for r in range(w.L - 1):
+            reached = int(tr["level_reached"][r, b])
+            if reached < 0:
+                break
+            drafted = bool((tr["tree_count"][r, :, b] > 0).any())
+            if not spec:
+                assert not drafted and int(tr["n_draft"][r, b]) == 0, (b, r)
+            spec = spec and (reached - m >= 2)
+            m = reached
+    if name == "tiny":
+        tot = 0
+        for b in range(w.batch):
+            sets, st = O.speculative_decode(model, head, case.req(b), K, V, adaptive=True)
+            for r in range(st.rounds):
+                n = len(st.accepted_len[r])
+                assert int(tr["n_draft"][r, b]) == n and list(tr["accepted_len"][r, b, :n]) == st.accepted_len[r]
+                assert int(tr["level_reached"][r, b]) == st.reject_level[r]
+            tot += st.primary_tokens
+        assert out["stats"].primary_tokens == tot
+        ar_codes = ar["codes"].cpu().numpy()
+        rng = np.random.default_rng(11)
+        drafts = ar_codes.copy()
+        n_draft = ar["count"].cpu().numpy().copy()
+        for b in range(w.batch):
+            for k in range(n_draft[b]):
+                if rng.random() < 0.6:
+                    lvl = int(rng.integers(0, w.L))
+                    drafts[b, k, lvl] = (drafts[b, k, lvl] + 1 + rng.integers(0, w.T[lvl] - 1)) % w.T[lvl]
+        got = case.eng.decode_with_drafts(K, torch.from_numpy(drafts).cuda(), torch.from_numpy(n_draft).cuda(), trace=True)
+        assert torch.equal(got["codes"], ar["codes"])
+        tot = 0
+        for b in range(w.batch):
+            D = [tuple(int(c) for c in drafts[b, k]) for k in range(n_draft[b])]
+            sets, st = O.speculative_decode(model, head, case.req(b), K, V, drafts_round1=D, adaptive=True)
+            assert [int(x) for x in got["trace"]["level_reached"][: st.rounds, b].cpu()] == st.reject_level
+            tot += st.primary_tokens
+        assert got["stats"].primary_tokens == tot
+    case.eng.set_option(5, 0)
+    again = case.eng.decode(K, mode=1)
+    assert again["stats"].primary_tokens == plain["stats"].primary_tokens
+
+
 def test_select_stage_with_prefix_filter(tiny):
     """One level of beam search on caller-supplied logits with the filter at an earlier level (level 1 of 3)."""
     w = tiny.w

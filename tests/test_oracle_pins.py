@@ -442,6 +442,50 @@ def test_speculative_walk_hand_worked_cases():
     assert codes_of(sp[-1]) == [(0, 0, 2), (0, 1, 1)]
 
 
+def test_adaptive_drafting_stops_after_a_round_without_gain():
+    """The engine policy on top of Algorithm 2: a round that settled only the one level the pass settles anyway turns the
+    request's drafting off.  Hand-worked on the zero-head case, and against plain drafting on random trees: same result,
+    never more tokens."""
+    cat = [(0, 0, 2), (0, 1, 1), (0, 1, 3), (1, 0, 0), (3, 3, 3)]
+    model, head, V, req = _zero_head_case(cat)
+    # first codes wrong: round 1 gains nothing (reaches level 2 = 1 + 1) -> round 2 drafts nothing: no drafted tuple, no
+    # tree node, B_2's 2 tokens only
+    sp, st = O.speculative_decode(model, head, req, 2, V, drafts_round1=[(2, 0, 0), (3, 3, 3)], adaptive=True)
+    assert codes_of(sp[-1]) == [(0, 0, 2), (0, 1, 1)]
+    assert (st.rounds, st.reject_level, st.accepted_len, st.primary_tokens, st.tree_nodes) == (2, [2, 3], [[0, 0], []], 4, [[0], []])
+    # the true tuples: one round, nothing to adapt
+    sp, st = O.speculative_decode(model, head, req, 2, V, drafts_round1=[(0, 0, 2), (0, 1, 1)], adaptive=True)
+    assert (st.rounds, st.accepted_len, st.primary_tokens) == (1, [[3, 3]], 4)
+    # four levels (T = 2 each, every tuple valid, zero heads, K = 2): B_1 = {0, 1}, B_2 = {00, 01}, B_3 = {000, 001},
+    # B_4 = {0000, 0001}.  Drafted tuples 0011 and 0100: tree level 2 = {00, 01} = B_2, level 3 = {001, 010} misses 000:
+    # round 1 settles levels 2 and 3 (a gain of two: keep drafting); the zero draft head continues from B_3 with the
+    # true level-4 set, round 2 finishes.
+    shape4 = synth.Workload("micro4", "fp32", 1, 16, 2, 1, 32, 4, (2, 2, 2, 2), 16, "uniform", 3, 2, 16, 5)
+    W4 = dict(synth.weights_to_numpy(synth.make_weights(shape4, std=0.5)))
+    W4["draft_logit"] = [np.zeros_like(a) for a in W4["draft_logit"]]
+    W4["lm_head"] = np.zeros_like(W4["lm_head"])
+    cat4 = np.asarray(list(itertools.product(range(2), repeat=4)), dtype=np.int32)
+    model4, head4, V4 = oracle_bundle(shape4, W4, cat4)
+    req4 = model4.prefill(synth.make_histories(shape4, None)[0])
+    sp, st = O.speculative_decode(model4, head4, req4, 2, V4, drafts_round1=[(0, 0, 1, 1), (0, 1, 0, 0)], adaptive=True)
+    assert [codes_of(x) for x in sp] == [[(0,), (1,)], [(0, 0), (0, 1)], [(0, 0, 0), (0, 0, 1)], [(0, 0, 0, 0), (0, 0, 0, 1)]]
+    assert (st.rounds, st.reject_level, st.accepted_len) == (2, [3, 4], [[3, 2], [4, 4]])
+    # one drafted tuple whose first code is a beam but whose second is not: its nodes (1,1) and (1,1,1) descend from the
+    # beam (1), so both are in round 1's pass (2 + 2 tokens), which gains nothing; rounds 2 and 3 are plain steps of 2 tokens
+    sp, st = O.speculative_decode(model4, head4, req4, 2, V4, drafts_round1=[(1, 1, 1, 1)], adaptive=True)
+    assert (st.rounds, st.reject_level, st.primary_tokens, st.accepted_len) == (3, [2, 3, 4], 4 + 2 + 2, [[1], [], []])
+    assert st.tree_nodes == [[1, 1], [0], []]
+    w, W, cat, model, head, V, hist = _micro()
+    rng = np.random.default_rng(9)
+    req = model.prefill(hist[0])
+    for trial in range(20):
+        tuples = [tuple(int(rng.integers(0, t)) for t in w.T) for _ in range(3)]
+        a = O.speculative_decode(model, head, req, 3, V, drafts_round1=tuples, adaptive=True)
+        p = O.speculative_decode(model, head, req, 3, V, drafts_round1=tuples)
+        assert [codes_of(x) for x in a[0]] == [codes_of(x) for x in p[0]]
+        assert a[1].primary_tokens <= p[1].primary_tokens and a[1].rounds >= p[1].rounds
+
+
 def test_tree_from_tuples_shares_prefixes():
     tree = O.tree_from_tuples([(1, 2, 3), (1, 2, 0), (1, 0, 3), (2, 2, 3), (1, 2, 3)], 3)
     assert tree == [[(1,), (2,)], [(1, 2), (1, 0), (2, 2)], [(1, 2, 3), (1, 2, 0), (1, 0, 3), (2, 2, 3)]]
