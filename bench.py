@@ -29,16 +29,29 @@ sys.path.insert(0, ROOT)
 sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 METRIC, UNIT = "items_per_s_decoded", "items/s"
-# bumped whenever a kernel of the class changes in a way that can change its DRAM traffic: a traffic figure taken
+# bumped whenever a kernel of the family changes in a way that can change its DRAM traffic: a traffic figure taken
 # from an older revision is reported as null
-KERNEL_REV = {"gemm": 6, "attention": 3, "probe": 2}
+KERNEL_REV = {"gemm": 7, "attention_tc": 3, "attention_umma": 5, "probe": 3}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the launches of the class in one decode step
-# (ncu, eager launches, L2 flushed before the step)
+# (ncu, eager launches, L2 flushed before the step); key = class @ workload
 NCU_TRAFFIC = {
-    "gemm@small": {"kernel_rev": 6, "dram_bytes_per_launch": 3.18e6, "source": "profiles/gemm_tc_kernel_ncu.md, section A2"},
-    "probe@0.5b@67108864": {"kernel_rev": 2, "dram_bytes_per_launch": 5.10e9, "source": "profiles/hs_probe_kernel.md"},
-    "attention@small": {"kernel_rev": 3, "dram_bytes_per_launch": 31.5e6, "source": "profiles/attn_tc_kernel_ncu.md, traffic section"},
+    # captured on a two-layer cut of the 7B shape (the full model under ncu is a 68 s step); a launch is the same at any
+    # depth, so the class average of the full model is rebuilt from the per-kernel figures: 12 layer launches per layer
+    # (three rounds) moved 1,371 MB, the 16 launches outside the layers 436 MB -> (32 x 1,371 + 436) / 400
+    "gemm@7b": {"family": "gemm", "kernel_rev": 7, "dram_bytes_per_launch": 110.8e6,
+                "source": "profiles/gemm_tc_kernel_ncu.md, section E (two-layer cut, scaled by launches per layer)"},
+    "gemm@small": {"family": "gemm", "kernel_rev": 6, "dram_bytes_per_launch": 3.18e6, "source": "profiles/gemm_tc_kernel_ncu.md, section A2"},
+    "probe@0.5b@67108864": {"family": "probe", "kernel_rev": 2, "dram_bytes_per_launch": 5.10e9, "source": "profiles/hs_probe_kernel.md"},
+    "attention@small": {"family": "attention_tc", "kernel_rev": 3, "dram_bytes_per_launch": 31.5e6,
+                        "source": "profiles/attn_tc_kernel_ncu.md, traffic section"},
 }
+
+
+def ncu_traffic(key):
+    rec = NCU_TRAFFIC.get(key)
+    if rec and rec["kernel_rev"] == KERNEL_REV.get(rec["family"]):
+        return rec
+    return None
 
 
 def whole_job_throughput(dist, local_ms: float, items_per_rank_step: int, steps: int, world: int, device="cpu"):
@@ -156,8 +169,8 @@ def probe_bench(args, w, eng, cat_dev, config, dev):
     ms = t0.elapsed_time(t1) / args.steps
     peaks = load_peaks()
     gbs = n * 41.0 / (ms / 1e3) / 1e9
-    rec = NCU_TRAFFIC.get(f"probe@{w.name}@{n}")
-    traffic = rec["dram_bytes_per_launch"] if rec and rec["kernel_rev"] == KERNEL_REV.get("probe") else None
+    rec = ncu_traffic(f"probe@{w.name}@{n}")
+    traffic = rec["dram_bytes_per_launch"] if rec else None
     slots = 4 * max(2, math.ceil(math.ceil(max(1, w.n_items) / w.load_factor) / 4))      # buckets of four 8-byte slots
     print(json.dumps({"metric": "hash_probes_per_s", "value": n / (ms / 1e3), "unit": "probes/s", "n_gpus": 1,
                       "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
@@ -263,10 +276,15 @@ def time_decode(ctx, mode, drafts, steps, warmup, flush, dist, world, dev, barri
         roof.update(bound="latency", note="dominant class is neither GEMM nor attention")
     # DRAM traffic of the dominant kernel from the ncu capture of that kernel in this workload (bytes per launch);
     # null when no capture matches the current kernel revision
-    rec = NCU_TRAFFIC.get(f"{dom}@{w.name}")
-    if rec and rec["kernel_rev"] == KERNEL_REV.get(dom):
+    rec = ncu_traffic(f"{dom}@{w.name}")
+    if rec:
         roof["traffic"] = rec["dram_bytes_per_launch"]
         roof["traffic_source"] = rec["source"]
+    if dom == "gemm":            # algorithmic bytes of an average launch of the class, to set beside `traffic`
+        esz = 4 if w.dtype == "fp32" else 2
+        act = (ptok / prof_steps) * (w.d_model * 4 + (w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim + w.n_q_heads * w.head_dim
+                                     + 3 * w.d_ffn) * esz * w.n_layers
+        roof["algorithmic_bytes_per_launch"] = (work["gemm_weight_bytes"] + act) / max(1.0, shares["gemm"]["launches_per_step"])
     # the whole step against its floor: per class the larger of (bytes / copy bandwidth) and (flops / tensor peak),
     # summed over the GEMM and attention classes (the rest moves kilobytes), divided by the measured step time
     if w.dtype == "bf16" and mode != 0:

@@ -259,7 +259,7 @@ size_t carve(nezha_ctx* c) {
   e.tb_count = cv.take<int>((size_t)(c->L + 1) * c->Bmax);
   e.tb_anc = cv.take<int>(lbk * c->L); e.tb_self = cv.take<int>(lbk); e.tb_src = cv.take<int>(lbk);
   e.row_m = cv.take<int>(c->Bmax); e.row_cur = cv.take<int>(c->Bmax); e.row_P = cv.take<int>(c->Bmax);
-  e.row_m_start = cv.take<int>(c->Bmax); e.row_spec = cv.take<int>(c->Bmax);
+  e.row_m_start = cv.take<int>(c->Bmax); e.row_spec = cv.take<int>(c->Bmax); e.draft_rows = cv.take<int>(1);
   e.dw_codes = cv.take<int>(lbk * c->L); e.dw_score = cv.take<float>(lbk); e.dw_parent = cv.take<int>(lbk);
   e.dw_count = cv.take<int>((size_t)(c->L + 1) * c->Bmax);
   e.d_m = cv.take<int>(c->Bmax);
@@ -447,10 +447,12 @@ SelectArgs select_base(nezha_ctx* c, int batch, int K) {
 bool draft_fast(const nezha_ctx* c) {
   return c->fused && c->opt_transition == 0 && c->opt_inputs == 0;
 }
-void draft_level_product(nezha_ctx* c, int batch, int l, bool with_state) {
+// in_round: inside a decode round, where the device knows whether any request still drafts (a round queued for nothing, or
+// one in which the adaptive policy has switched every request's drafting off, runs its products over zero rows)
+void draft_level_product(nezha_ctx* c, int batch, int l, bool with_state, bool in_round = false) {
   const int T = c->cfg.T[l - 1];
-  gemm(c, c->draft_sact, c->d, c->draft_wcat[l - 1], c->d, c->draft_g, c->Tmax + c->d, (long long)batch * c->Kmax, nullptr,
-       T + (with_state ? c->d : 0), c->d, kEpiStoreF32);
+  gemm(c, c->draft_sact, c->d, c->draft_wcat[l - 1], c->d, c->draft_g, c->Tmax + c->d, (long long)batch * c->Kmax,
+       in_round ? c->es.draft_rows : nullptr, T + (with_state ? c->d : 0), c->d, kEpiStoreF32);
 }
 void draft_level_step(nezha_ctx* c, int batch, int l) {
   launch_draft_step(c->es, batch, l, c->draft_g, c->Tmax + c->d, c->cfg.T[l - 1], c->draft_u, (const float*)c->draft_b_f32, c->draft_sact,
@@ -464,7 +466,7 @@ void draft_phase(nezha_ctx* c, int batch, int K, bool from_scratch, int first_le
   const bool fast = draft_fast(c);
   launch_draft_init(e, batch, from_scratch ? 1 : 0, fast ? c->draft_sact : nullptr, c->st);
   for (int l = 1; l <= c->L; ++l) {
-    if (fast && (l >= first_level || l < c->L)) draft_level_product(c, batch, l, l < c->L);
+    if (fast && (l >= first_level || l < c->L)) draft_level_product(c, batch, l, l < c->L, true);
     if (l >= first_level) {
       if (!fast) draft_logits_level(c, batch, l);
       SelectArgs s = select_base(c, batch, K);

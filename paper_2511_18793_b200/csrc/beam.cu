@@ -363,8 +363,10 @@ __global__ void init_decode_kernel(EngineState e, int batch) {
   pdl_wait();
   pdl_launch();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b == 0)
+  if (b == 0) {
     for (int i = 0; i < 8; ++i) e.counters[i] = 0;
+    *e.draft_rows = batch * e.Kmax;
+  }
   if (b >= batch) return;
   e.tb_count[0 * e.Bmax + b] = 1;
   e.tb_score[lvl_bk(e, 0, b, 0)] = 0.f;
@@ -647,6 +649,7 @@ __global__ void nodes_count_kernel(EngineState e, int batch) {
   const int L = e.L;
   __shared__ int n_alive;
   if (threadIdx.x == 0) n_alive = 0;
+  if (b == 0 && threadIdx.x == 0) *e.draft_rows = 0;     // this round's drafting is over; round_end raises it again if needed
   __syncthreads();
   if (m >= L) {
     if (threadIdx.x == 0) { e.row_tok_count[b] = 0; e.row_cur[b] = -1; e.req_info[b] = make_int4(0, 0, b, 0); }
@@ -934,6 +937,7 @@ __global__ void round_end_kernel(EngineState e, int batch, int K, int round, nez
     if (tr.n_draft) tr.n_draft[tro] = took_part ? nd : -1;
     if (tr.level_reached) tr.level_reached[tro] = took_part ? m_now : -1;
     if (took_part && adaptive) e.row_spec[b] = (m_now - e.row_m_start[b] >= 2) ? 1 : 0;
+    if (m_now < L && e.row_spec[b]) atomicMax(e.draft_rows, batch * Kmax);   // somebody drafts next round
     if (m_now < L) atomicAdd(&e.counters[0], 1);
     atomicAdd(&e.counters[1], e.row_tok_count[b]);
     atomicAdd(&e.counters[2], acc_sum);

@@ -27,6 +27,7 @@ struct EngineState {
   int* row_cur;     // [Bmax] level whose beams have logits in the current pass, -1 = row stopped this round
   int* row_P;       // [Bmax] context length of the row (BOS + history tokens)
   int* row_m_start; // [Bmax] levels the row had settled when the current round began
+  int* draft_rows;  // [1] rows of the draft head's products in the coming round: batch * Kmax, or 0 when no request drafts
   int* row_spec;    // [Bmax] 1: the draft head drafts for the row in the next round (always 1 unless the adaptive policy is on)
 
   // The round's draft tree, [L+1][Bmax][Kmax]([L]): level l holds the drafted nodes with l codes (the draft head's beam
