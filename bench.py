@@ -41,7 +41,7 @@ NCU_TRAFFIC = {
     "gemm@7b": {"family": "gemm", "kernel_rev": 7, "dram_bytes_per_launch": 110.8e6,
                 "source": "profiles/gemm_tc_kernel_ncu.md, section E (two-layer cut, scaled by launches per layer)"},
     "gemm@small": {"family": "gemm", "kernel_rev": 6, "dram_bytes_per_launch": 3.18e6, "source": "profiles/gemm_tc_kernel_ncu.md, section A2"},
-    "probe@0.5b@67108864": {"family": "probe", "kernel_rev": 2, "dram_bytes_per_launch": 5.10e9, "source": "profiles/hs_probe_kernel.md"},
+    "probe@0.5b@67108864": {"family": "probe", "kernel_rev": 3, "dram_bytes_per_launch": 5.10e9, "source": "profiles/hs_probe_kernel.md"},
     "attention@small": {"family": "attention_tc", "kernel_rev": 3, "dram_bytes_per_launch": 31.5e6,
                         "source": "profiles/attn_tc_kernel_ncu.md, traffic section"},
 }
