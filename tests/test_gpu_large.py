@@ -26,7 +26,17 @@ PLAN = {                       # workload -> (requests checked by the oracle, or
 def test_full_size_workload(name):
     w = synth.WORKLOADS[name]
     rows, odt = PLAN[name]
-    case = Case(w, oracle_dtype=odt).prefill()
+    # the launch configuration bench.py times: a stream of the engine's own, on which the library replays every round of a
+    # decode call as a CUDA graph from the third call on (first call eager, second captured)
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(st):
+        _full_size_checks(name, w, rows, odt, st)
+    torch.cuda.synchronize()
+
+
+def _full_size_checks(name, w, rows, odt, st):
+    case = Case(w, oracle_dtype=odt, stream=st).prefill()
     V = O.ValidSet(case.catalog, w.T)
     assert case.n_unique == w.n_items == len(V)
     # ---- hash set, bit exact
@@ -39,9 +49,18 @@ def test_full_size_workload(name):
     sib[:, -1] = np.tile(np.arange(w.T[-1]), len(pre))
     got = case.eng.probe(case.eng.pack(torch.from_numpy(sib.astype(np.int32)).cuda())).cpu().numpy().astype(bool)
     assert np.array_equal(got, V.contains(sib))
-    # ---- decode: invariants on every request
-    out = case.eng.decode(w.beam, mode=1, trace=True)
-    ar = case.eng.decode(w.beam, mode=2)
+    # ---- decode: invariants on every request (eager, captured and replayed calls must agree bit for bit)
+    outs = case.eng.alloc_outputs(w.batch, w.beam, trace=True)
+    first = {k: v.clone() for k, v in case.eng.decode(w.beam, mode=1, out=outs).items() if k in ("codes", "scores", "count")}
+    for call in range(4):       # the tiling follows the token counts of the call before: eager again, captured, replayed twice
+        out = case.eng.decode(w.beam, mode=1, out=outs)
+        st.synchronize()
+        for k, v in first.items():
+            assert torch.equal(out[k], v), (call, k)
+    ar_out = case.eng.alloc_outputs(w.batch, w.beam)
+    for call in range(4):
+        ar = case.eng.decode(w.beam, mode=2, out=ar_out)
+    st.synchronize()
     assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
     assert torch.allclose(out["scores"], ar["scores"], atol=1e-4)
     codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
