@@ -86,6 +86,37 @@ def test_error_paths(tiny):
     assert ei.value.status == 6
 
 
+def test_invalid_drafts_are_dropped_and_reported(tiny):
+    """Drafted tuples / tree nodes with a code outside [0, T_l) are no semantic IDs: the call reports NEZHA_ERR_CATALOG, the
+    tuple (node) takes no part, the items are Algorithm 1's all the same, and the next call is clean."""
+    b = tiny.binding
+    w = tiny.w
+    K = w.beam
+    ar = tiny.eng.decode(K, mode=2, trace=True)
+    drafts = ar["codes"].clone().clamp_(min=0)
+    drafts[:, 0, 1] = w.T[1]                                     # one bad tuple per request
+    out = tiny.eng.alloc_outputs(w.batch, K, trace=True)
+    with pytest.raises(b.NezhaError) as ei:
+        tiny.eng.decode_with_drafts(K, drafts, ar["count"].clone(), out=out)
+    assert ei.value.status == 6
+    assert torch.equal(out["codes"], ar["codes"]) and torch.equal(out["count"], ar["count"])
+    n_draft = out["trace"]["n_draft"][0].cpu().numpy()
+    assert np.array_equal(n_draft, np.maximum(ar["count"].cpu().numpy() - 1, 0))     # the bad tuple is not in the tree
+    beams = ar["trace"]["beams"].clone()
+    counts = (beams[:, :, :, 0] >= 0).sum(dim=2).to(torch.int32)
+    beams[1, :, 0, 0] = -5                                       # a bad node at level 2: it and its subtree are dead
+    with pytest.raises(b.NezhaError) as ei:
+        tiny.eng.decode_with_draft_tree(K, beams, counts, out=out)
+    assert ei.value.status == 6
+    assert torch.equal(out["codes"], ar["codes"])
+    check_walk_against_trace(tiny.eng.decode(K, mode=1, trace=True), w.batch, w.L)     # and the next call is clean
+    with pytest.raises(b.NezhaError) as ei:                       # null tree
+        b.lib.nezha_decode_with_draft_tree.argtypes
+        tiny.eng._check(b.lib.nezha_decode_with_draft_tree(tiny.eng._h, w.batch, K, None, None, out["codes"].data_ptr(),
+                                                            out["scores"].data_ptr(), out["count"].data_ptr(), None, None))
+    assert ei.value.status == 1
+
+
 # ---------------------------------------------------------------------------------------- stage-wise FP parity
 def test_prefill_hidden_states(tiny):
     h = tiny.eng.get_hidden().cpu().numpy()
