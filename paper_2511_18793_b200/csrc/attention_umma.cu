@@ -37,10 +37,10 @@ constexpr float kRaise = 8.f;      // the reference maximum follows the true one
 // PT ("P in TMEM"): the softmax threads write P straight back into the TMEM columns its scores came from (bf16 pairs, the
 // A operand of the second product read from TMEM) instead of through a shared-memory buffer, and S is double-buffered:
 // S_{j+2} = Q K_{j+2}^T is issued right behind P_j V_j, the softmax of tile j + 1 never waits for the P V product of tile
-// j, and the 16 KB that P took hold a third V slot.  Without PT: one S, one P buffer in shared memory (three CTAs per SM
+// j, and the 16 KB that P took hold a third K slot (S runs two tiles ahead).  Without PT: one S, one P buffer in shared memory (three CTAs per SM
 // at hd = 64, where TMEM is what limits the PT form to two).
 template <int HD, bool PT> struct UmmaCfg {
-  static constexpr int kKRing = kRingU, kVRing = PT ? 3 : kRingU;
+  static constexpr int kKRing = PT ? 3 : kRingU, kVRing = kRingU;
   static constexpr int kQBytes = kRowsU * HD * 2;
   static constexpr int kPBytes = PT ? 0 : kRowsU * kPosU * 2;
   static constexpr int kTileBytes = kPosU * HD * 2;            // one K (or V) tile
