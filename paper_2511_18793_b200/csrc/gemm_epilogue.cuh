@@ -201,6 +201,48 @@ __device__ __forceinline__ EpiRow epilogue_row(const GemmArgs& a, int row, int M
   return r;
 }
 
+// The epilogue proper on one staged 32 x 32 block (rows row0 .. row0 + 31, columns n_chunk .. n_chunk + 31) that sits in
+// the warp's transpose tile in the swizzled "8 lanes per row" image described above.  er = epilogue_row of row
+// row0 + lane; rows_here = how many of the 32 rows exist (> 0).  The caller has made the tile visible to the warp.
+template <int EPI>
+__device__ __forceinline__ void epilogue_block(const GemmArgs& a, float4* stg4, int lane, int row0, int rows_here, int n_chunk,
+                                               const EpiRow& er) {
+  const int k = lane & 7, rsub = lane >> 3;
+  const ChunkCtx cc = chunk_ctx<EPI>(a, n_chunk, k);
+  const int n = n_chunk + 4 * k;
+#pragma unroll
+  for (int it0 = 0; it0 < 8; it0 += 4) {
+    if (it0 * 4 >= rows_here) break;                           // warp-uniform
+    EpiAux aux[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = (it0 + u) * 4 + rsub;
+      const int p_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, er.pos, r) : 0;
+      if (r < rows_here) aux[u] = epi_prefetch<EPI>(a, cc, row0 + r, n, p_r);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = (it0 + u) * 4 + rsub;
+      const long long kv_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, er.kvd, r) : -1;
+      const float4 x = stg4[r * 8 + (k ^ (r & 7))];
+      const float4 back = epi_apply<EPI>(a, cc, r < rows_here, row0 + r, n, k, x, aux[u], kv_r);
+      if (EPI == kEpiAddNorm) stg4[r * 8 + (k ^ (r & 7))] = back;
+    }
+  }
+  __syncwarp();
+  if (EPI == kEpiAddNorm && lane < rows_here) {
+    // one partial sum of squares per 32-column group, added up in column order: the same bits whatever the tile width
+    float ssq = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float4 t = stg4[lane * 8 + (j ^ (lane & 7))];
+      ssq += t.x * t.x; ssq += t.y * t.y; ssq += t.z * t.z; ssq += t.w * t.w;
+    }
+    a.f.ss_out[(long long)(n_chunk >> 5) * a.f.ss_ld + row0 + lane] = ssq;
+  }
+  __syncwarp();
+}
+
 // One epilogue warp's share of a finished accumulator: TMEM lanes [32 q, 32 q + 32) (= rows m0 + 32 q ..) and the
 // 32-column groups half, half + 2, ... of the BN columns starting at TMEM column `tmem_acc`.  er = epilogue_row of
 // the lane's own row (lane = row while the block comes out of TMEM).
@@ -209,7 +251,6 @@ __device__ __forceinline__ EpiRow epilogue_row(const GemmArgs& a, int row, int M
 template <int BN, int EPI, int CHAINS = 1>
 __device__ __forceinline__ void drain_accumulator(const GemmArgs& a, uint32_t tmem_acc, int q, int half, int lane,
                                                   float4* stg4, int m0, int n0, int M, const EpiRow& er) {
-  const int row = m0 + q * 32 + lane;
   const int rows_here = min(32, M - (m0 + q * 32));          // rows of this quarter that exist (may be <= 0)
 #pragma unroll 1
   for (int c = half; c < BN / 32; c += 2) {
@@ -230,39 +271,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& a, uint32_t tm
       stg4[lane * 8 + (j ^ (lane & 7))] =
           make_float4(v[4 * j] * er.rs, v[4 * j + 1] * er.rs, v[4 * j + 2] * er.rs, v[4 * j + 3] * er.rs);
     __syncwarp();
-    const int k = lane & 7, rsub = lane >> 3;
-    const ChunkCtx cc = chunk_ctx<EPI>(a, n_chunk, k);
-    const int n = n_chunk + 4 * k;
-#pragma unroll
-    for (int it0 = 0; it0 < 8; it0 += 4) {
-      if (it0 * 4 >= rows_here) break;                           // warp-uniform
-      EpiAux aux[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int r = (it0 + u) * 4 + rsub;
-        const int p_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, er.pos, r) : 0;
-        if (r < rows_here) aux[u] = epi_prefetch<EPI>(a, cc, m0 + q * 32 + r, n, p_r);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int r = (it0 + u) * 4 + rsub;
-        const long long kv_r = (EPI == kEpiRopeKV) ? __shfl_sync(0xffffffffu, er.kvd, r) : -1;
-        const float4 x = stg4[r * 8 + (k ^ (r & 7))];
-        const float4 back = epi_apply<EPI>(a, cc, r < rows_here, m0 + q * 32 + r, n, k, x, aux[u], kv_r);
-        if (EPI == kEpiAddNorm) stg4[r * 8 + (k ^ (r & 7))] = back;
-      }
-    }
-    __syncwarp();
-    if (EPI == kEpiAddNorm && lane < rows_here) {
-      // one partial sum of squares per 32-column group, added up in column order: the same bits whatever the tile width
-      float ssq = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float4 t = stg4[lane * 8 + (j ^ (lane & 7))];
-        ssq += t.x * t.x; ssq += t.y * t.y; ssq += t.z * t.z; ssq += t.w * t.w;
-      }
-      a.f.ss_out[(long long)(n_chunk >> 5) * a.f.ss_ld + row] = ssq;
-    }
+    if (rows_here > 0) epilogue_block<EPI>(a, stg4, lane, m0 + q * 32, rows_here, n_chunk, er);
     __syncwarp();
   }
 }

@@ -278,9 +278,12 @@ bool gemm_tc_supported(const GemmArgs& a) {
 }
 
 void launch_gemm_tc_pair(const GemmArgs& a, int n_sm, cudaStream_t st);
+bool gemm_skinny_applies(const GemmArgs& a, int n_sm);
+void launch_gemm_skinny(const GemmArgs& a, int n_sm, cudaStream_t st);
 
 void launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
   LaunchScope ls(kcGemm, st);
+  if (gemm_skinny_applies(a, sm_count())) { launch_gemm_skinny(a, sm_count(), st); return; }
   const int m_plan = a.M_expected > 0 && a.M_expected < a.M ? a.M_expected : a.M;
   // Narrow outputs (N <= 1024) never fill a 256-wide tile well and their k-loops are bound by the MMA issue chain:
   // a caller that asks for two partial sums gets tiles of at most 128 columns with two issuers for them.  The rule

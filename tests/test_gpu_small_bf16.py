@@ -170,10 +170,12 @@ def test_bf16_shapes_ragged_histories(shape):
     check_walk_against_trace(out, w.batch, w.L)
 
 
-def test_paper_setting_three_levels_of_512_codes():
+@pytest.mark.parametrize("batch", [6, 3, 1])
+def test_paper_setting_three_levels_of_512_codes(batch):
     """L = 3 levels over codebooks of 512 (the paper's own setting), beam 10, short histories: every mode, all requests,
-    on a two-layer cut of the 1B-sized backbone."""
-    w = synth.scaled(synth.WORKLOADS["paper"], n_layers=2, batch=6)
+    on a two-layer cut of the 1B-sized backbone.  With 3 requests (60 rows per pass at most) and with 1 (20 rows) every
+    product of the decode calls runs in the weight-streaming kernel, on its 64-row and its 32-row tile."""
+    w = synth.scaled(synth.WORKLOADS["paper"], n_layers=2, batch=batch)
     case = Case(w).prefill()
     model, head, V = case.oracle
     assert case.n_unique == w.n_items
