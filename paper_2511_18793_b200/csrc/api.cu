@@ -96,9 +96,8 @@ struct nezha_ctx {
   int chains_now;           // GemmArgs::chains of the products being queued: 2 inside a decode call, 0 otherwise
   // Weight-streaming products: an engine none of whose decode passes can exceed kSkinnyRows rows runs every product of a
   // decode call through that kernel (the choice is per engine, so both decode modes compute the same bits).
-  SkinnyWork skinny_work;
   bool skinny_decode;
-  const SkinnyWork* skinny_now;   // GemmArgs::skinny of the products being queued
+  int skinny_now;           // GemmArgs::skinny of the products being queued
   int rounds_seen[3];       // rounds the last decode call of each mode needed: that many are launched without waiting
   int device;               // the GPU that was current at nezha_create
   int state;                // 0 created, 1 hash set built, 2 prefilled
@@ -246,11 +245,6 @@ size_t carve(nezha_ctx* c) {
   c->h_rows = cv.take<int>((size_t)c->Bmax * (c->L + 1));
   c->fused = c->bf16 && (c->hd == 64 || c->hd == 128) && c->d % 64 == 0 && c->F % 64 == 0;
   c->ss_a = c->ss_b = c->ss_e = nullptr;
-  c->skinny_work = SkinnyWork{nullptr, nullptr};
-  if (c->bf16) {
-    c->skinny_work.partials = cv.take<float>(kSkinnyPartialBytes / sizeof(float));
-    c->skinny_work.arrivals = cv.take<unsigned>(kSkinnyMaxTiles);
-  }
   c->draft_u = c->draft_hl = c->draft_g = nullptr; c->draft_sact = nullptr;
   for (int l = 0; l < kMaxLevels; ++l) c->draft_wcat[l] = nullptr;
   if (c->fused) {
@@ -514,9 +508,6 @@ nezha_status pending_device_error(nezha_ctx* c) {
   NZ_CUDA(c, cudaStreamSynchronize(c->st));
   st = c->host_counters[8];
   if (st) NZ_CUDA(c, cudaMemsetAsync(c->es.status, 0, 4 * sizeof(int), c->st));
-  // a weight-streaming product that gave up may have left arrivals counted
-  if ((st & kStInternal) && c->skinny_work.arrivals)
-    NZ_CUDA(c, cudaMemsetAsync(c->skinny_work.arrivals, 0, kSkinnyMaxTiles * sizeof(unsigned), c->st));
   if (st & kStHashFull) return fail(c, NEZHA_ERR_HASH_FULL, "hash set insertion exhausted its probe bound");
   if (st & kStBadCode) return fail(c, NEZHA_ERR_CATALOG, "a code outside [0, T_l) was given");
   if (st)      // a kernel that records where it gave up leaves three more words (0 if it does not)
@@ -577,9 +568,9 @@ nezha_status decode_impl(nezha_ctx* c, int batch, int K, int mode, const int* dr
     nezha_ctx* c;
     explicit ChainScope(nezha_ctx* c_) : c(c_) {
       c->chains_now = 2;
-      c->skinny_now = c->skinny_decode ? &c->skinny_work : nullptr;
+      c->skinny_now = c->skinny_decode ? 1 : 0;
     }
-    ~ChainScope() { c->chains_now = 0; c->skinny_now = nullptr; }
+    ~ChainScope() { c->chains_now = 0; c->skinny_now = 0; }
   } chain_scope(c);
   nezha_trace tr{};
   if (trace) tr = *trace;
@@ -722,7 +713,7 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
   for (int i = 0; i <= kMaxLevels; ++i) c->m_seen[i] = 0;
   for (int i = 0; i < 3; ++i) c->rounds_seen[i] = 0;
   c->chains_now = 0;
-  c->skinny_now = nullptr;
+  c->skinny_now = 0;
   c->opt_transition = 0; c->opt_inputs = 0; c->opt_filter = 1; c->opt_mask = 1; c->opt_level_filter = 0; c->opt_adaptive = 0;
   const size_t need = carve(c);
   if (need > arena_bytes) { delete c; return NEZHA_ERR_ARENA_TOO_SMALL; }
@@ -743,11 +734,9 @@ nezha_status nezha_create(const nezha_config* cfg, const nezha_weights* w, const
     return src && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   };
   bool ok = cudaMemsetAsync(c->es.status, 0, 8 * sizeof(int), st) == cudaSuccess;
-  if (c->skinny_work.arrivals)
-    ok = ok && cudaMemsetAsync(c->skinny_work.arrivals, 0, kSkinnyMaxTiles * sizeof(unsigned), st) == cudaSuccess;
   {
     const long long pass_rows = c->Mv_max > (long long)c->Bmax * c->Kmax ? c->Mv_max : (long long)c->Bmax * c->Kmax;
-    c->skinny_decode = c->fused && c->skinny_work.partials && pass_rows <= kSkinnyRows && !getenv("NEZHA_NO_SKINNY");
+    c->skinny_decode = c->fused && pass_rows <= kSkinnyRows && !getenv("NEZHA_NO_SKINNY");
   }
   // the caches start as zeros: tiles may overhang into never-written rows, whose (masked) values must be finite
   ok = ok && cudaMemsetAsync(c->k_ctx, 0, (size_t)c->nl * c->ctx_layer_elems * c->esz, st) == cudaSuccess &&
@@ -1020,9 +1009,9 @@ nezha_status nezha_gemm(nezha_ctx* c, const void* A, const void* W, void* C, int
   GemmArgs a{A, K, W, K, C, N, M, nullptr, N, K, epilogue, bias, c->es.status};
   a.chains = path == 3 ? 2 : 0;
   if (path == 4) {
-    if (M > kSkinnyRows || !c->skinny_work.partials)
+    if (M > kSkinnyRows || !c->bf16)
       return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: the weight-streaming kernel takes bf16 products of at most 64 rows");
-    a.skinny = &c->skinny_work;
+    a.skinny = 1;
   }
   const bool tc_ok = c->bf16 && gemm_tc_supported(a);
   if (path >= 2 && !tc_ok) return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: shape not covered by the tcgen05 kernel");

@@ -214,15 +214,7 @@ struct GemmFuse {
   int Hq, Hkv, hd;
 };
 
-// Work space of the weight-streaming kernel: room for one 128 x kSkinnyRows fp32 partial tile per CTA of its largest
-// grid, and one arrival counter per 128-column output tile (zero between launches: the last arriver resets its own).
-constexpr int kSkinnyRows = 64;
-constexpr int kSkinnyMaxCtas = 512, kSkinnyMaxTiles = 4096;
-struct SkinnyWork {
-  float* partials;       // [kSkinnyMaxCtas][128 * kSkinnyRows]
-  unsigned* arrivals;    // [kSkinnyMaxTiles]
-};
-constexpr size_t kSkinnyPartialBytes = (size_t)kSkinnyMaxCtas * 128 * kSkinnyRows * sizeof(float);
+constexpr int kSkinnyRows = 64;     // most rows a launch of the weight-streaming GEMM kernel takes
 
 struct GemmArgs {
   const void* A; long long lda;
@@ -241,12 +233,12 @@ struct GemmArgs {
   // differently: a caller that needs the same bits from launches of different sizes asks for the same value in all of
   // them (the tiling itself never changes the result).
   int chains;
-  // Non-null: a launch of at most kSkinnyRows rows may run as the weight-streaming kernel (weights as the 128-row MMA
-  // operand, the rows as its N, the K range split over CTAs whose partial tiles meet in this work space).  Its
-  // summation order differs from the other kernels' and depends on (N, K) and the device only: a caller that needs the
-  // same bits from two launches offers the work space to both or to neither.  W must be constant data (it is read
-  // before the launch's dependency on its predecessor is resolved).
-  const SkinnyWork* skinny;
+  // Non-zero: a launch of at most kSkinnyRows rows may run as the weight-streaming kernel (weights as the 128-row MMA
+  // operand, the rows as its N, the K range split over the CTAs of a cluster).  Its summation order differs from the
+  // other kernels' and depends on (N, K) and the device only: a caller that needs the same bits from two launches sets
+  // the flag in both or in neither.  W must be constant data (it is read before the launch's dependency on its
+  // predecessor is resolved).
+  int skinny;
 };
 
 void launch_gemm_simt(const GemmArgs& a, bool bf16, cudaStream_t st);

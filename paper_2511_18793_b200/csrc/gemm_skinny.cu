@@ -4,10 +4,10 @@
 // With a handful of rows the product is bound by reading W once from HBM.  The 128-row MMA operand is therefore a
 // 128 x 64 tile of W (16 KB per copy, the unit that has to be kept in flight), the rows of A are the MMA's N (MT = 32 or
 // 64), and the accumulator in TMEM is a 128 x MT block of C^T.  An output tile is 128 columns of C; the K range of a
-// tile is split over several CTAs so that every SM streams a share of W, whatever N.  Each CTA of a split tile writes
-// its partial block to a work space; the CTA that arrives last (an arrival counter per tile, no waiting) adds the
-// parts in split order -- the order of arrival never shows in the bits -- and runs the same fused epilogue as the
-// other tensor-core kernels.
+// tile is split over the CTAs of a thread-block cluster (up to 8) so that every SM streams a share of W, whatever N.
+// Each CTA leaves its partial block in its own shared memory; after a cluster barrier the 32 x 32 blocks of the tile are
+// dealt out to the cluster's CTAs, which add the parts in rank order, reading their peers' shared memory -- the bits
+// never depend on timing -- and run the same fused epilogue as the other tensor-core kernels.
 // A CTA issues the weight copies of its first ring round BEFORE the launch's dependency on the preceding kernel is
 // resolved (W is constant data), and the kernel is sized for two CTAs per SM, so the weight stream of a launch starts
 // while its predecessor is still draining.
@@ -40,32 +40,46 @@ template <int MT> struct SkinnyCfg {
   static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM");
 };
 
-__device__ __forceinline__ void epi_bar_sync(int n_threads) {
-  asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory");
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Every thread of every CTA of the cluster executes both halves, on every path.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 16 bytes of the shared memory of CTA `rank` of the cluster, at the address that `local` has in this CTA.
+__device__ __forceinline__ float4 ld_peer_f4(uint32_t local, uint32_t rank) {
+  uint32_t ra;
+  float4 v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local), "r"(rank));
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(ra) : "memory");
+  return v;
 }
 
-// grid = tiles x splits (blockIdx.x = tile * splits + split).  Warp 0: TMA producer; warp 1: TMEM owner and MMA issuer;
+// grid = tiles x splits, clusters of `splits` CTAs (blockIdx.x = tile * splits + split, split = rank in the cluster).  Warp 0: TMA producer; warp 1: TMEM owner and MMA issuer;
 // warps 2 ..: epilogue, warp w on TMEM lane quarter w % 4 (columns n0 + 32 q ..) and rows 32 c .. of A, c = (w - 2) / 4.
 template <int MT, int EPI>
 __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
     gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a,
-                       SkinnyWork work, int splits, int* status) {
+                       int splits, int* status) {
   using C = SkinnyCfg<MT>;
   constexpr int STAGES = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bar_base = base + STAGES * C::kStageBytes;
-  // barriers: full[STAGES], empty[STAGES], acc_full; then the TMEM slot, the abort flag and the "last arriver" flag
+  // barriers: full[STAGES], empty[STAGES], acc_full; then the TMEM slot and the abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   const uint32_t acc_full = bar_base + 8u * (2 * STAGES);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * C::kStageBytes + 8 * (2 * STAGES + 1));
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  volatile uint32_t* last_flag = tmem_slot + 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x / splits, split = blockIdx.x - tile * splits;
+  const int tile = blockIdx.x / splits, split = (int)cluster_rank();
   const int n0 = tile * 128;
   // this CTA's share of the k-steps: contiguous, the first (k_iters % splits) shares one step longer
   const int k_iters = a.K / BK;
@@ -77,7 +91,6 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(acc_full, 1);
     *abort_flag = 0;
-    *last_flag = 0;
     mbar_fence_init();
     tma_prefetch_map(&tmW);
     tma_prefetch_map(&tmX);
@@ -99,6 +112,7 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
   pdl_wait();
   pdl_launch();
   const int M = a.M_dev ? min(a.M, *a.M_dev) : a.M;
+  EpiRow er{1.f, 0, -1};                         // of the epilogue warps: the row the lane answers for in its block
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -143,71 +157,64 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
   } else {
     // ------------------------------------------------------------------ epilogue
     const int q = warp & 3, c = (warp - 2) >> 2, ew = warp - 2;
-    constexpr int kBlocks = 4 * (MT / 32);       // 32 x 32 blocks of a CTA's partial tile
     float4* stg4 = reinterpret_cast<float4*>(gen_base) + ew * (32 * 8);
     float* stg = reinterpret_cast<float*>(stg4);
     const int row0 = c * 32, n_chunk = n0 + q * 32;
     const int rows_here = min(32, M - row0);     // rows of this block that exist (may be <= 0)
     const bool have = rows_here > 0 && n_chunk < a.N;      // warp-uniform
-    const EpiRow er = epilogue_row<EPI>(a, row0 + lane, M);   // overlaps the main loop
+    if (splits == 1 || ew % splits == split) er = epilogue_row<EPI>(a, row0 + lane, M);   // overlaps the main loop
     bool ok = warp_wait(acc_full, 0, abort_flag, lane);
     tc_fence_after();
     float v[32];                                 // lane = column n_chunk + lane, v[j] = row row0 + j
     if (ok) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
-    if (splits == 1) {
+    if (splits > 1) {
+      // the partial block stays in this CTA's shared memory, in the "8 lanes per row" image; the cluster adds the parts below
       if (ok && have) {
-        // from lane = column to the "8 lanes per row" image: row j's 32 columns are one 128-byte line, chunks swizzled
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          stg[(j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3)] = v[j] * __shfl_sync(0xffffffffu, er.rs, j);
-        __syncwarp();
-        epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, er);
+        for (int j = 0; j < 32; ++j) stg[(j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3)] = v[j];
       }
-    } else {
-      // the partial block goes to the work space in the same image (every store of a warp is one 128-byte line)
-      if (ok && have) {
-        float* img = work.partials + ((size_t)blockIdx.x * kBlocks + (c * 4 + q)) * 1024;
+    } else if (ok && have) {
+      // from lane = column to the "8 lanes per row" image: row j's 32 columns are one 128-byte line, chunks swizzled
 #pragma unroll
-        for (int j = 0; j < 32; ++j) __stcg(img + (j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3), v[j]);
-        __threadfence();
-      }
-      if (!ok && lane == 0) *abort_flag = 1;
-      epi_bar_sync(32 * C::kEpiWarps);
-      if (ew == 0 && lane == 0 && !*abort_flag) {
-        __threadfence();                         // the other warps' parts, ordered before this thread by the barrier
-        const unsigned old = atomicAdd(work.arrivals + tile, 1u);
-        if (old == (unsigned)(splits - 1)) {
-          __threadfence();
-          work.arrivals[tile] = 0;               // every part has arrived: ready for the next launch
-          *last_flag = 1;
-        }
-      }
-      epi_bar_sync(32 * C::kEpiWarps);
-      if (*last_flag && have) {
-        __threadfence();
-        // lane's 8 chunks of the block image, summed over the parts in split order
-        const float4* src = reinterpret_cast<const float4*>(work.partials + ((size_t)(tile * splits) * kBlocks + (c * 4 + q)) * 1024);
+      for (int j = 0; j < 32; ++j)
+        stg[(j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3)] = v[j] * __shfl_sync(0xffffffffu, er.rs, j);
+      __syncwarp();
+      epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, er);
+    }
+    if (!ok && lane == 0) *abort_flag = 1;
+  }
+  if (splits > 1) {
+    // The cluster's CTAs are the splits of one tile (rank = split).  Block b of the tile is finished by CTA b mod
+    // splits: it adds the parts in rank order, reading its peers' shared memory, and runs the epilogue on the sum.
+    cluster_sync_all();                          // all parts are in place (or their CTA has raised its abort flag)
+    if (warp >= 2) {
+      const int q = warp & 3, c = (warp - 2) >> 2, ew = warp - 2;
+      float4* stg4 = reinterpret_cast<float4*>(gen_base) + ew * (32 * 8);
+      const int row0 = c * 32, n_chunk = n0 + q * 32;
+      const int rows_here = min(32, M - row0);
+      if (rows_here > 0 && n_chunk < a.N && !*abort_flag && ew % splits == split) {
+        const uint32_t img = base + (uint32_t)ew * 4096u + (uint32_t)lane * 16u;
         float4 acc[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = __ldcg(src + i * 32 + lane);
+        for (int i = 0; i < 8; ++i) acc[i] = ld_peer_f4(img + i * 512, 0);
         for (int sp = 1; sp < splits; ++sp) {
-          const float4* p = src + (size_t)sp * kBlocks * 256;
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float4 t = __ldcg(p + i * 32 + lane);
+            const float4 t = ld_peer_f4(img + i * 512, (uint32_t)sp);
             acc[i].x += t.x; acc[i].y += t.y; acc[i].z += t.z; acc[i].w += t.w;
           }
         }
+        __syncwarp();                            // (this CTA's own part is one of the sources)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float rs = __shfl_sync(0xffffffffu, er.rs, i * 4 + (lane >> 3));     // chunk i*32 + lane is of row i*4 + lane/8
+          const float rs = __shfl_sync(0xffffffffu, er.rs, i * 4 + (lane >> 3));
           stg4[i * 32 + lane] = make_float4(acc[i].x * rs, acc[i].y * rs, acc[i].z * rs, acc[i].w * rs);
         }
         __syncwarp();
         epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, er);
       }
     }
-    if (!ok && lane == 0) *abort_flag = 1;
+    cluster_sync_all();                          // no CTA leaves while a peer may still read its part
   }
   tc_fence_before();
   __syncthreads();
@@ -232,8 +239,15 @@ void launch(const GemmArgs& a, int tiles, int splits, cudaStream_t st) {
   configured.run([] {
     cudaFuncSetAttribute(gemm_skinny_kernel<MT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   });
-  launch_pdl(gemm_skinny_kernel<MT, EPI>, dim3(tiles * splits), dim3(C::kThreads), C::kSmemBytes, st, tw, tx, a, *a.skinny,
-             splits, a.status);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(tiles * splits); cfg.blockDim = dim3(C::kThreads); cfg.dynamicSmemBytes = C::kSmemBytes; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = splits; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  cudaLaunchKernelEx(&cfg, gemm_skinny_kernel<MT, EPI>, tw, tx, a, splits, a.status);
 }
 
 template <int MT>
@@ -252,8 +266,8 @@ void launch_mt(const GemmArgs& a, int tiles, int splits, cudaStream_t st) {
 
 }  // namespace
 
-// Number of CTAs a tile's K range is split over: as many as bring the grid to about `target` CTAs (one per SM unless
-// NEZHA_SKINNY_CTAS says otherwise), each with at least four k-steps (64 KB of W per 16 or 32 KB of partial tile).
+// Number of CTAs a tile's K range is split over (= the cluster size): as many as bring the grid to about one CTA per SM
+// (NEZHA_SKINNY_CTAS: another target), at most 8, each with at least four k-steps (64 KB of W per partial tile).
 // A function of N, K and the device only -- never of the row count -- so a product's bits do not depend on its rows.
 int gemm_skinny_splits(int N, int K, int n_sm) {
   static const int forced = getenv("NEZHA_SKINNY_CTAS") ? atoi(getenv("NEZHA_SKINNY_CTAS")) : 0;
@@ -261,14 +275,14 @@ int gemm_skinny_splits(int N, int K, int n_sm) {
   const int tiles = (N + 127) / 128, k_iters = K / BK;
   int s = target / tiles;
   if (s > k_iters / 4) s = k_iters / 4;
+  if (s > 8) s = 8;                              // the portable cluster size
   if (s < 1) s = 1;
-  while (s > 1 && (long long)tiles * s > kSkinnyMaxCtas) --s;
   return s;
 }
 
 bool gemm_skinny_applies(const GemmArgs& a, int n_sm) {
-  return a.skinny && a.skinny->partials && a.skinny->arrivals && a.M <= kSkinnyRows && (a.N + 127) / 128 <= kSkinnyMaxTiles &&
-         (long long)((a.N + 127) / 128) * gemm_skinny_splits(a.N, a.K, n_sm) <= kSkinnyMaxCtas;
+  (void)n_sm;
+  return a.skinny && a.M <= kSkinnyRows && (long long)((a.N + 127) / 128) * 8 <= 0x7fffffff;
 }
 
 void launch_gemm_skinny(const GemmArgs& a, int n_sm, cudaStream_t st) {

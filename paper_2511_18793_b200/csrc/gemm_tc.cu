@@ -30,7 +30,6 @@ template <int BN> struct Cfg {
   static constexpr int kStages = BN >= 192 ? 4 : BN == 160 ? 5 : BN == 128 ? 6 : 8;
   static constexpr int kSmemBytes =
       kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTransposeBytes;
-  static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;       // two accumulators; a power of two >= 32
   // kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128.
   static constexpr uint32_t kInstrDesc =
       (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
