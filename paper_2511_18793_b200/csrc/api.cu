@@ -841,6 +841,9 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
   for (int b0 = 0; b0 < batch; b0 += c->chunk_rows) {
     const int rows = (batch - b0 < c->chunk_rows) ? batch - b0 : c->chunk_rows;
     const long long M = (long long)rows * S_call;
+    // a prompt chunk of at most 64 tokens in an engine of the weight-streaming class (one short history): the same
+    // kernel as its decode passes.  The prefill is shared by all decode modes, so their equality is not touched.
+    c->skinny_now = c->skinny_decode && M <= kSkinnyRows ? 1 : 0;
     launch_prefill_tokens(e, hist_codes, n_hist, b0, rows, max_n, S_call, c->S, c->h_rows, c->st);
     if (c->fused) {
       launch_embed_norm(c->embed, e.tok_id, (int)M, nullptr, c->d, c->resid, c->layers[0].attn_norm, c->xn, c->ss_e, c->st);
@@ -858,6 +861,7 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
         gemm(c, (char*)c->h_act + (ho + (size_t)l * c->d) * c->esz, (long long)(c->L + 1) * c->d, c->draft_logit[l - 1], c->d,
              c->draft_hl + ((size_t)(l - 1) * c->Bmax + b0) * c->Tmax, c->Tmax, rows, nullptr, c->cfg.T[l - 1], c->d, kEpiStoreF32);
   }
+  c->skinny_now = 0;
   NZ_CUDA(c, cudaGetLastError());
   c->batch = batch;
   c->state = 2;
