@@ -193,14 +193,26 @@ def test_paper_setting_three_levels_of_512_codes(batch):
     live = np.arange(w.beam)[None, :] < count[:, None]
     assert V.contains(codes[live]).all()
     check_walk_against_trace(out, w.batch, w.L)
+    # the true beam sets as the draft tree: one round, the tokens of plain decoding, every tuple accepted in full
+    tb = out["trace"]["beams"]
+    counts = (tb[:, :, :, 0] >= 0).sum(dim=2).to(torch.int32)
+    pt = case.eng.decode_with_draft_tree(w.beam, tb, counts, trace=True)
+    assert torch.equal(pt["codes"], ar["codes"]) and torch.equal(pt["count"], ar["count"])
+    live_t = torch.from_numpy(live).cuda()                  # (one pass over all levels rounds differently from one per level)
+    assert (pt["scores"][live_t] - ar["scores"][live_t]).abs().max().item() <= tolerance(w) if live.any() else True
+    assert pt["stats"].rounds == 1 and pt["stats"].primary_tokens == int(counts[: w.L - 1].sum())
+    check_walk_against_trace(pt, w.batch, w.L)
 
 
-@pytest.mark.parametrize("name", ["tiny", "small"])
+@pytest.mark.parametrize("name", ["tiny", "small", "paper_batch1"])
 def test_graph_replay_equals_eager_launches(name):
     """On a stream of its own the library captures every round of a decode call into a CUDA graph after one eager
     run and replays it afterwards.  Eager, capturing and replaying calls must give the same bits as an engine on the
-    default stream (which never captures), in every mode, with and without trace outputs and with injected drafts."""
-    w = synth.WORKLOADS[name]
+    default stream (which never captures), in every mode, with and without trace outputs and with injected drafts.
+    (paper_batch1: one request of the paper's setting on a two-layer cut, whose products are cluster launches of the
+    weight-streaming kernel: those are captured and replayed too, and the drafts of the last part are the result
+    itself, so that call ends in one round.)"""
+    w = synth.scaled(synth.WORKLOADS["paper"], n_layers=2, batch=1) if name == "paper_batch1" else synth.WORKLOADS[name]
     ref = Case(w).prefill()
     st = torch.cuda.Stream()
     torch.cuda.synchronize()
