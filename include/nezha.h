@@ -256,7 +256,7 @@ nezha_status nezha_select(nezha_ctx* ctx, int32_t batch, int32_t n_beams, int32_
  *               is not covered: bf16 storage, K % 64 == 0, N % 32 == 0); 3: the tcgen05 kernel as the decode calls use
  *               it: for N <= 1024 the K range is accumulated in two interleaved partial sums (two MMA issuers), which
  *               rounds differently from path 2 in the last bits; 4: the weight-streaming tcgen05 kernel that the
- *               decode calls of an engine with at most 64 rows per pass use (M <= 64; W is the 128-row MMA operand,
+ *               decode calls of an engine with at most 128 rows per pass use (M <= 128; W is the 128-row MMA operand,
  *               the K range is split over CTAs and the parts are added in a fixed order that depends on N, K and
  *               the device only; W must not be written by work still in flight on the stream)
  * Used by every projection of the primary model (Algorithm 1's model call), the LM head and the draft head

@@ -841,7 +841,7 @@ nezha_status nezha_prefill(nezha_ctx* c, const int32_t* hist_codes, const int32_
   for (int b0 = 0; b0 < batch; b0 += c->chunk_rows) {
     const int rows = (batch - b0 < c->chunk_rows) ? batch - b0 : c->chunk_rows;
     const long long M = (long long)rows * S_call;
-    // a prompt chunk of at most 64 tokens in an engine of the weight-streaming class (one short history): the same
+    // a prompt chunk of at most kSkinnyRows tokens in an engine of the weight-streaming class (one short history): the same
     // kernel as its decode passes.  The prefill is shared by all decode modes, so their equality is not touched.
     c->skinny_now = c->skinny_decode && M <= kSkinnyRows ? 1 : 0;
     launch_prefill_tokens(e, hist_codes, n_hist, b0, rows, max_n, S_call, c->S, c->h_rows, c->st);
@@ -1014,7 +1014,7 @@ nezha_status nezha_gemm(nezha_ctx* c, const void* A, const void* W, void* C, int
   a.chains = path == 3 ? 2 : 0;
   if (path == 4) {
     if (M > kSkinnyRows || !c->bf16)
-      return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: the weight-streaming kernel takes bf16 products of at most 64 rows");
+      return fail(c, NEZHA_ERR_UNSUPPORTED, "nezha_gemm: the weight-streaming kernel takes bf16 products of at most 128 rows");
     a.skinny = 1;
   }
   const bool tc_ok = c->bf16 && gemm_tc_supported(a);

@@ -214,7 +214,7 @@ struct GemmFuse {
   int Hq, Hkv, hd;
 };
 
-constexpr int kSkinnyRows = 64;     // most rows a launch of the weight-streaming GEMM kernel takes
+constexpr int kSkinnyRows = 128;    // most rows a launch of the weight-streaming GEMM kernel takes
 
 struct GemmArgs {
   const void* A; long long lda;

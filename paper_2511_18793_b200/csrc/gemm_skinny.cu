@@ -1,9 +1,9 @@
-// Weight-streaming GEMM for launches of at most 64 rows:  C[M,N] (op)= A[M,K] * W[N,K]^T  with the operands' roles
+// Weight-streaming GEMM for launches of at most 128 rows:  C[M,N] (op)= A[M,K] * W[N,K]^T  with the operands' roles
 // swapped on the tensor core.
 //
 // With a handful of rows the product is bound by reading W once from HBM.  The 128-row MMA operand is therefore a
-// 128 x 64 tile of W (16 KB per copy, the unit that has to be kept in flight), the rows of A are the MMA's N (MT = 32 or
-// 64), and the accumulator in TMEM is a 128 x MT block of C^T.  An output tile is 128 columns of C; the K range of a
+// 128 x 64 tile of W (16 KB per copy, the unit that has to be kept in flight), the rows of A are the MMA's N (MT = 32, 64
+// or 128), and the accumulator in TMEM is a 128 x MT block of C^T.  An output tile is 128 columns of C; the K range of a
 // tile is split over the CTAs of a thread-block cluster (up to 8) so that every SM streams a share of W, whatever N.
 // Each CTA leaves its partial block in its own shared memory; after a cluster barrier the 32 x 32 blocks of the tile are
 // dealt out to the cluster's CTAs, which add the parts in rank order, reading their peers' shared memory -- the bits
@@ -26,8 +26,10 @@ template <int MT> struct SkinnyCfg {
   static constexpr int kTileBytesW = 128 * BK * 2;
   static constexpr int kTileBytesX = MT * BK * 2;
   static constexpr int kStageBytes = kTileBytesW + kTileBytesX;
-  static constexpr int kStages = MT == 32 ? 5 : 4;
-  static constexpr int kEpiWarps = 4 * (MT / 32);            // one per (TMEM lane quarter, block of 32 rows of A)
+  static constexpr int kStages = MT == 32 ? 5 : MT == 64 ? 4 : 3;
+  static constexpr int kBlocks = 4 * (MT / 32);              // 32 x 32 blocks of the tile: (TMEM lane quarter, 32 rows of A)
+  static constexpr int kEpiWarps = MT == 32 ? 4 : 8;         // warp w: lane quarter w % 4, every (kEpiWarps / 4)-th row block
+  static constexpr int kBlocksPerWarp = kBlocks / kEpiWarps;
   static constexpr int kThreads = 64 + 32 * kEpiWarps;
   static constexpr int kBarBytes = 128;
   // (the epilogue's transpose tiles reuse the ring: a CTA has one tile, and the ring is idle once it is accumulated)
@@ -36,7 +38,7 @@ template <int MT> struct SkinnyCfg {
   // kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N = MT, M = 128.
   static constexpr uint32_t kInstrDesc =
       (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-  static_assert(kEpiWarps * 4096 <= kStages * kStageBytes, "transpose tiles do not fit in the ring");
+  static_assert(kBlocks * 4096 <= kStages * kStageBytes, "transpose tiles do not fit in the ring");
   static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM");
 };
 
@@ -60,7 +62,7 @@ __device__ __forceinline__ float4 ld_peer_f4(uint32_t local, uint32_t rank) {
 }
 
 // grid = tiles x splits, clusters of `splits` CTAs (blockIdx.x = tile * splits + split, split = rank in the cluster).  Warp 0: TMA producer; warp 1: TMEM owner and MMA issuer;
-// warps 2 ..: epilogue, warp w on TMEM lane quarter w % 4 (columns n0 + 32 q ..) and rows 32 c .. of A, c = (w - 2) / 4.
+// warps 2 ..: epilogue, warp w on TMEM lane quarter w % 4 (columns n0 + 32 q ..) and the 32-row blocks c = (w - 2) / 4, + 1 or 2, .. of A.
 template <int MT, int EPI>
 __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
     gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a,
@@ -112,7 +114,10 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
   pdl_wait();
   pdl_launch();
   const int M = a.M_dev ? min(a.M, *a.M_dev) : a.M;
-  EpiRow er{1.f, 0, -1};                         // of the epilogue warps: the row the lane answers for in its block
+  constexpr int BPW = C::kBlocksPerWarp, CSTEP = C::kEpiWarps / 4;
+  EpiRow er[BPW];                                // of the epilogue warps: the row the lane answers for in each of its blocks
+#pragma unroll
+  for (int bi = 0; bi < BPW; ++bi) er[bi] = EpiRow{1.f, 0, -1};
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -156,30 +161,38 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int q = warp & 3, c = (warp - 2) >> 2, ew = warp - 2;
-    float4* stg4 = reinterpret_cast<float4*>(gen_base) + ew * (32 * 8);
-    float* stg = reinterpret_cast<float*>(stg4);
-    const int row0 = c * 32, n_chunk = n0 + q * 32;
-    const int rows_here = min(32, M - row0);     // rows of this block that exist (may be <= 0)
-    const bool have = rows_here > 0 && n_chunk < a.N;      // warp-uniform
-    if (splits == 1 || ew % splits == split) er = epilogue_row<EPI>(a, row0 + lane, M);   // overlaps the main loop
-    bool ok = warp_wait(acc_full, 0, abort_flag, lane);
+    // block b = 4 c + q of the tile: columns n0 + 32 q .., rows 32 c .. of A; its transpose tile is slot b of the (idle) ring
+    const int q = warp & 3, c0 = (warp - 2) >> 2;
+    const int n_chunk = n0 + q * 32;
+#pragma unroll
+    for (int bi = 0; bi < BPW; ++bi) {             // overlaps the main loop
+      const int c = c0 + bi * CSTEP;
+      if (splits == 1 || (c * 4 + q) % splits == split) er[bi] = epilogue_row<EPI>(a, c * 32 + lane, M);
+    }
+    const bool ok = warp_wait(acc_full, 0, abort_flag, lane);
     tc_fence_after();
-    float v[32];                                 // lane = column n_chunk + lane, v[j] = row row0 + j
-    if (ok) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
-    if (splits > 1) {
-      // the partial block stays in this CTA's shared memory, in the "8 lanes per row" image; the cluster adds the parts below
-      if (ok && have) {
+#pragma unroll 1
+    for (int bi = 0; bi < BPW && ok; ++bi) {
+      const int c = c0 + bi * CSTEP, blk = c * 4 + q;
+      const int row0 = c * 32, rows_here = min(32, M - row0);   // rows of this block that exist (may be <= 0)
+      if (rows_here <= 0 || n_chunk >= a.N) continue;        // warp-uniform
+      float4* stg4 = reinterpret_cast<float4*>(gen_base) + blk * (32 * 8);
+      float* stg = reinterpret_cast<float*>(stg4);
+      float v[32];                               // lane = column n_chunk + lane, v[j] = row row0 + j
+      tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+      if (splits > 1) {
+        // the partial block stays in this CTA's shared memory, in the "8 lanes per row" image; the cluster adds the parts below
 #pragma unroll
         for (int j = 0; j < 32; ++j) stg[(j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3)] = v[j];
-      }
-    } else if (ok && have) {
-      // from lane = column to the "8 lanes per row" image: row j's 32 columns are one 128-byte line, chunks swizzled
+      } else {
+        // from lane = column to the "8 lanes per row" image: row j's 32 columns are one 128-byte line, chunks swizzled
+        const float rs_mine = bi == 0 ? er[0].rs : er[BPW - 1].rs;
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        stg[(j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3)] = v[j] * __shfl_sync(0xffffffffu, er.rs, j);
-      __syncwarp();
-      epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, er);
+        for (int j = 0; j < 32; ++j)
+          stg[(j * 8 + ((lane >> 2) ^ (j & 7))) * 4 + (lane & 3)] = v[j] * __shfl_sync(0xffffffffu, rs_mine, j);
+        __syncwarp();
+        epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, bi == 0 ? er[0] : er[BPW - 1]);
+      }
     }
     if (!ok && lane == 0) *abort_flag = 1;
   }
@@ -187,13 +200,17 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
     // The cluster's CTAs are the splits of one tile (rank = split).  Block b of the tile is finished by CTA b mod
     // splits: it adds the parts in rank order, reading its peers' shared memory, and runs the epilogue on the sum.
     cluster_sync_all();                          // all parts are in place (or their CTA has raised its abort flag)
-    if (warp >= 2) {
-      const int q = warp & 3, c = (warp - 2) >> 2, ew = warp - 2;
-      float4* stg4 = reinterpret_cast<float4*>(gen_base) + ew * (32 * 8);
-      const int row0 = c * 32, n_chunk = n0 + q * 32;
-      const int rows_here = min(32, M - row0);
-      if (rows_here > 0 && n_chunk < a.N && !*abort_flag && ew % splits == split) {
-        const uint32_t img = base + (uint32_t)ew * 4096u + (uint32_t)lane * 16u;
+    if (warp >= 2 && !*abort_flag) {
+      const int q = warp & 3, c0 = (warp - 2) >> 2;
+      const int n_chunk = n0 + q * 32;
+#pragma unroll 1
+      for (int bi = 0; bi < BPW; ++bi) {
+        const int c = c0 + bi * CSTEP, blk = c * 4 + q;
+        const int row0 = c * 32, rows_here = min(32, M - row0);
+        if (rows_here <= 0 || n_chunk >= a.N || blk % splits != split) continue;
+        const EpiRow& erb = bi == 0 ? er[0] : er[BPW - 1];
+        float4* stg4 = reinterpret_cast<float4*>(gen_base) + blk * (32 * 8);
+        const uint32_t img = base + (uint32_t)blk * 4096u + (uint32_t)lane * 16u;
         float4 acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = ld_peer_f4(img + i * 512, 0);
@@ -207,11 +224,11 @@ __global__ void __launch_bounds__(SkinnyCfg<MT>::kThreads, 2)
         __syncwarp();                            // (this CTA's own part is one of the sources)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float rs = __shfl_sync(0xffffffffu, er.rs, i * 4 + (lane >> 3));
+          const float rs = __shfl_sync(0xffffffffu, erb.rs, i * 4 + (lane >> 3));
           stg4[i * 32 + lane] = make_float4(acc[i].x * rs, acc[i].y * rs, acc[i].z * rs, acc[i].w * rs);
         }
         __syncwarp();
-        epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, er);
+        epilogue_block<EPI>(a, stg4, lane, row0, rows_here, n_chunk, erb);
       }
     }
     cluster_sync_all();                          // no CTA leaves while a peer may still read its part
@@ -288,7 +305,8 @@ bool gemm_skinny_applies(const GemmArgs& a, int n_sm) {
 void launch_gemm_skinny(const GemmArgs& a, int n_sm, cudaStream_t st) {
   const int tiles = (a.N + 127) / 128, splits = gemm_skinny_splits(a.N, a.K, n_sm);
   if (a.M <= 32) launch_mt<32>(a, tiles, splits, st);      // (the bound, not the expected count: no row may be dropped)
-  else launch_mt<64>(a, tiles, splits, st);
+  else if (a.M <= 64) launch_mt<64>(a, tiles, splits, st);
+  else launch_mt<128>(a, tiles, splits, st);
 }
 
 }  // namespace nz

@@ -46,6 +46,16 @@ def e2e_tolerance(w, std=0.02):
     return max(tolerance(w), 4.0 * std * np.sqrt(w.d_model) * 1.6e-3 * np.sqrt(8.0 * w.n_layers))
 
 
+def wide_tolerance(w, std=0.02):
+    """Logits (and log-probabilities) of a shallow cut of a WIDE model, whole pipeline: the final hidden state is off by
+    about 0.0074 rms per layer (measured on the two-layer cuts; the model above gives 0.0045-0.0071), a logit inherits
+    ||row|| = std * sqrt(d) times that, and the largest of the few thousand values a test compares is held to 5 sigma.
+    At d = 512 this stays below the plain 2e-2; at d = 2048 and one layer it is 3.3e-2."""
+    if w.dtype == "fp32":
+        return tolerance(w)
+    return max(tolerance(w), 5.0 * std * np.sqrt(w.d_model) * 0.0074 * np.sqrt(w.n_layers))
+
+
 class Case:
     """Engine + oracle on one workload.  Weights are drawn once and handed to both sides as the same bytes."""
 

@@ -97,19 +97,19 @@ def test_gemm_odd_number_of_k_steps_many_tiles_per_cta(ctx, N, K, path):
 
 @pytest.mark.parametrize("N,K", [(512, 512), (3072, 2048), (2048, 8192), (2080, 2048), (16384, 2048), (32, 64), (256, 192)])
 def test_weight_streaming_gemm(ctx, N, K):
-    """The kernel for launches of at most 64 rows (weights as the 128-row MMA operand, K split over CTAs): every epilogue
-    against the fp64 product, for row counts on both sides of its 32-row tile; a row's bits depend neither on the
+    """The kernel for launches of at most 128 rows (weights as the 128-row MMA operand, K split over CTAs): every epilogue
+    against the fp64 product, for row counts in each of its three accumulator widths (32, 64, 128); a row's bits depend neither on the
     number of rows nor on the order in which the CTAs of a tile arrive (run twice)."""
     g = torch.Generator(device="cuda"); g.manual_seed(N * 11 + K)
-    A64 = (torch.randn(64, K, generator=g, device="cuda") * 0.5).bfloat16()
+    A64 = (torch.randn(128, K, generator=g, device="cuda") * 0.5).bfloat16()
     W = (torch.randn(N, K, generator=g, device="cuda") * 0.05).bfloat16()
     bias = torch.randn(N, generator=g, device="cuda")
-    res64 = torch.randn(64, N, generator=g, device="cuda")
+    res64 = torch.randn(128, N, generator=g, device="cuda")
     ref64 = _ref(A64, W)                                    # (also a device synchronisation: W is at rest from here on)
     scale = np.abs(ref64).max()
-    full = torch.empty(64, N, dtype=torch.float32, device="cuda")
+    full = torch.empty(128, N, dtype=torch.float32, device="cuda")
     ctx.eng.gemm(A64, W, full, epilogue=1, path=4)
-    for M in (1, 7, 20, 32, 33, 50, 64):
+    for M in (1, 7, 20, 32, 33, 50, 64, 65, 97, 128):
         A, ref = A64[:M].contiguous(), ref64[:M]
         out = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
         ctx.eng.gemm(A, W, out, epilogue=1, path=4)
@@ -130,10 +130,10 @@ def test_weight_streaming_gemm(ctx, N, K):
     ctx.eng.sync()
 
 
-def test_weight_streaming_gemm_takes_at_most_64_rows(ctx):
-    A = torch.zeros(65, 64, dtype=torch.bfloat16, device="cuda")
+def test_weight_streaming_gemm_takes_at_most_128_rows(ctx):
+    A = torch.zeros(129, 64, dtype=torch.bfloat16, device="cuda")
     W = torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")
-    out = torch.zeros(65, 128, dtype=torch.float32, device="cuda")
+    out = torch.zeros(129, 128, dtype=torch.float32, device="cuda")
     with pytest.raises(ctx.binding.NezhaError) as ei:
         ctx.eng.gemm(A, W, out, epilogue=1, path=4)
     assert ei.value.status == 7

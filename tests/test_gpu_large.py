@@ -11,7 +11,7 @@ import torch
 
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
-from gpu_helpers import Case, check_levels, check_walk_against_trace, e2e_tolerance, hidden_rms_bound, hidden_tolerance, stage_tolerance
+from gpu_helpers import Case, wide_tolerance, check_levels, check_walk_against_trace, e2e_tolerance, hidden_rms_bound, hidden_tolerance, stage_tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -122,7 +122,7 @@ def test_two_layer_cut_at_full_width(name):
     w = synth.scaled(synth.WORKLOADS[name], n_layers=2, batch=4, n_items=200_000)
     case = Case(w).prefill()
     model, head, V = case.oracle
-    tol = max(2e-2, 5.0 * 0.02 * np.sqrt(w.d_model) * 0.0074 * np.sqrt(2.0))
+    tol = wide_tolerance(w)
     h = case.eng.get_hidden().cpu().numpy()
     for b in range(w.batch):
         dh = h[b] - case.req(b).h

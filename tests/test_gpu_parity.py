@@ -6,7 +6,7 @@ import torch
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
 from helpers import codes_of
-from gpu_helpers import Case, assert_topk_matches, check_levels, check_walk_against_trace, tolerance
+from gpu_helpers import Case, assert_topk_matches, check_levels, check_walk_against_trace, tolerance, wide_tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -496,7 +496,8 @@ def test_validity_filter_at_every_level(name):
     beams, scores = out["trace"]["beams"].cpu().numpy(), out["trace"]["beam_scores"].cpu().numpy()
     dcodes, dscores, dcount = (dr[k].cpu().numpy() for k in ("codes", "scores", "count"))
     for b in range(w.batch):
-        check_levels(case, b, beams[:, b], scores[:, b], w.beam, every_level=True)
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam, every_level=True,
+                     tol=wide_tolerance(w) if name == "t512" else None)      # d = 2048: see wide_tolerance
         for n in range(w.L):
             cnt = int((beams[n, b, :, 0] >= 0).sum())
             assert V.contains_prefix(beams[n, b, :cnt, : n + 1]).all()

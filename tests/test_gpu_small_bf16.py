@@ -9,7 +9,7 @@ import torch
 
 from oracle import nezha_oracle as O
 from paper_2511_18793_b200 import synth
-from gpu_helpers import Case, assert_topk_matches, check_levels, check_walk_against_trace, tolerance
+from gpu_helpers import Case, assert_topk_matches, check_levels, check_walk_against_trace, tolerance, wide_tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -170,11 +170,12 @@ def test_bf16_shapes_ragged_histories(shape):
     check_walk_against_trace(out, w.batch, w.L)
 
 
-@pytest.mark.parametrize("batch", [6, 3, 1])
+@pytest.mark.parametrize("batch", [7, 6, 3, 1])
 def test_paper_setting_three_levels_of_512_codes(batch):
     """L = 3 levels over codebooks of 512 (the paper's own setting), beam 10, short histories: every mode, all requests,
-    on a two-layer cut of the 1B-sized backbone.  With 3 requests (60 rows per pass at most) and with 1 (20 rows) every
-    product of the decode calls runs in the weight-streaming kernel, on its 64-row and its 32-row tile."""
+    on a two-layer cut of the 1B-sized backbone.  With 6 requests (120 rows per pass at most), 3 (60 rows) and 1 (20 rows)
+    every product of the decode calls runs in the weight-streaming kernel, on its 128-, 64- and 32-row accumulator; with
+    7 requests in the general kernels."""
     w = synth.scaled(synth.WORKLOADS["paper"], n_layers=2, batch=batch)
     case = Case(w).prefill()
     model, head, V = case.oracle
@@ -186,7 +187,7 @@ def test_paper_setting_three_levels_of_512_codes(batch):
     dr = case.eng.decode(w.beam, mode=0)
     dcodes, dscores, dcount = (dr[k].cpu().numpy() for k in ("codes", "scores", "count"))
     for b in range(w.batch):
-        check_levels(case, b, beams[:, b], scores[:, b], w.beam)
+        check_levels(case, b, beams[:, b], scores[:, b], w.beam, tol=wide_tolerance(w))     # d = 2048, two layers
         ref = O.nezha_draft(head, case.req(b), w.beam, V)[-1]
         assert_topk_matches(dcodes[b], dscores[b], dcount[b], ref, w.beam, tolerance(w))
     codes, count = out["codes"].cpu().numpy(), out["count"].cpu().numpy()
