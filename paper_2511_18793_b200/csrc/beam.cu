@@ -66,6 +66,14 @@ __device__ __forceinline__ void sort_desc(unsigned long long (&v)[N]) {
 // dependent steps on a few warps, so its time is the sum of their latencies: loads whose address needs no other load
 // go out together at the top; each lane keeps its keys sorted, so one survivor costs two redux and a shift; small
 // merges are a rank count with no serial loop at all.
+// Codebooks of more than 256 codes keep 16 or 32 keys per lane in registers (sorted 64-bit keys besides the scores): those
+// variants run with at most 8 warps so that a thread may use up to 255 registers instead of spilling its sort.
+__host__ __device__ constexpr int select_max_threads(int vpl) { return vpl >= 16 ? 256 : 512; }
+inline int select_warps(const SelectArgs& a) {
+  const int cap = a.T > 256 ? 8 : 16;
+  return a.in_stride < 8 ? 8 : a.in_stride > cap ? cap : a.in_stride;
+}
+
 template <int VPL>
 __device__ __forceinline__ void select_body(const SelectArgs& a) {
   const int b = blockIdx.x;
@@ -297,7 +305,7 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
 }
 
 template <int VPL>
-__global__ void __launch_bounds__(512) select_kernel(SelectArgs a) {
+__global__ void __launch_bounds__(select_max_threads(VPL)) select_kernel(SelectArgs a) {
   pdl_wait();
   pdl_launch();
   select_body<VPL>(a);
@@ -332,7 +340,7 @@ void launch_select(const SelectArgs& a, cudaStream_t st) {
   if (a.batch <= 0) return;
   const size_t smem = select_smem_bytes(a.in_stride, a.K);
   LaunchScope ls(kcSelect, st);
-  const int warps = a.in_stride < 8 ? 8 : a.in_stride > 16 ? 16 : a.in_stride;   // a warp per beam where that fits
+  const int warps = select_warps(a);   // a warp per beam where that fits
   const dim3 block(32 * warps);
   if (a.T <= 32) launch_pdl(select_kernel<1>, dim3(a.batch), block, smem, st, a);
   else if (a.T <= 256) launch_pdl(select_kernel<8>, dim3(a.batch), block, smem, st, a);
@@ -612,7 +620,7 @@ __global__ void draft_step_kernel(EngineState e, int batch, int l, const float* 
 // The selection of draft level l and the state update that follows it, in one launch: a block selects its request's
 // beams (or skips that when the request's level is already settled) and then advances the states of its own slots.
 template <int VPL>
-__global__ void __launch_bounds__(512) select_step_kernel(SelectArgs a, EngineState e, int l, const float* __restrict__ G,
+__global__ void __launch_bounds__(select_max_threads(VPL)) select_step_kernel(SelectArgs a, EngineState e, int l, const float* __restrict__ G,
                                                           long long g_stride, int t_cols, const float* __restrict__ U,
                                                           const float* __restrict__ bias, __nv_bfloat16* s_act) {
   pdl_wait();
@@ -875,7 +883,7 @@ __global__ void advance_kernel(EngineState e, int batch, int n, int K, int* out_
 }
 // The selection of B_{n+1} and the step above in one launch (both act on the requests whose current level is n).
 template <int VPL>
-__global__ void __launch_bounds__(512) select_advance_kernel(SelectArgs a, EngineState e, int n, int K, int* out_codes,
+__global__ void __launch_bounds__(select_max_threads(VPL)) select_advance_kernel(SelectArgs a, EngineState e, int n, int K, int* out_codes,
                                                              float* out_score, int* out_count) {
   pdl_wait();
   pdl_launch();
@@ -1065,7 +1073,7 @@ void launch_select_step(const SelectArgs& a, const EngineState& e, int l, const 
   if (a.batch <= 0) return;
   const size_t smem = select_smem_bytes(a.in_stride, a.K);
   LaunchScope ls(kcSelect, st);
-  const int warps = a.in_stride < 8 ? 8 : a.in_stride > 16 ? 16 : a.in_stride;
+  const int warps = select_warps(a);
   const dim3 block(32 * warps), grid(a.batch);
   __nv_bfloat16* s = (__nv_bfloat16*)s_act;
   if (a.T <= 32) launch_pdl(select_step_kernel<1>, grid, block, smem, st, a, e, l, G, g_stride, t_cols, U, bias, s);
@@ -1099,7 +1107,7 @@ void launch_select_advance(const SelectArgs& a, const EngineState& e, int n, int
   if (a.batch <= 0) return;
   const size_t smem = select_smem_bytes(a.in_stride, a.K);
   LaunchScope ls(kcSelect, st);
-  const int warps = a.in_stride < 8 ? 8 : a.in_stride > 16 ? 16 : a.in_stride;
+  const int warps = select_warps(a);
   const dim3 block(32 * warps), grid(a.batch);
   if (a.T <= 32) launch_pdl(select_advance_kernel<1>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
   else if (a.T <= 256) launch_pdl(select_advance_kernel<8>, grid, block, smem, st, a, e, n, K, out_codes, out_score, out_count);
