@@ -66,11 +66,11 @@ __device__ __forceinline__ void sort_desc(unsigned long long (&v)[N]) {
 // dependent steps on a few warps, so its time is the sum of their latencies: loads whose address needs no other load
 // go out together at the top; each lane keeps its keys sorted, so one survivor costs two redux and a shift; small
 // merges are a rank count with no serial loop at all.
-// Codebooks of more than 256 codes keep 16 or 32 keys per lane in registers (sorted 64-bit keys besides the scores): those
-// variants run with at most 8 warps so that a thread may use up to 255 registers instead of spilling its sort.
-__host__ __device__ constexpr int select_max_threads(int vpl) { return vpl >= 16 ? 256 : 512; }
+// Codebooks of more than 512 codes keep 32 keys per lane in registers besides the scores: that variant runs with at most
+// 8 warps so that a thread may use up to 255 registers.
+__host__ __device__ constexpr int select_max_threads(int vpl) { return vpl >= 32 ? 256 : 512; }
 inline int select_warps(const SelectArgs& a) {
-  const int cap = a.T > 256 ? 8 : 16;
+  const int cap = a.T > 512 ? 8 : 16;
   return a.in_stride < 8 ? 8 : a.in_stride > cap ? cap : a.in_stride;
 }
 
@@ -172,30 +172,71 @@ __device__ __forceinline__ void select_body(const SelectArgs& a) {
           if (want_probe[j] && !ok[j]) key[j0 + j] = -INFINITY;
       }
     }
-    // this lane's keys in descending order: (ordered score bits, then the smaller code first); 0 = used up
-    unsigned long long sk[VPL];
-#pragma unroll
-    for (int j = 0; j < VPL; ++j) sk[j] = ((unsigned long long)ordered_bits(key[j]) << 32) | (unsigned)(VPL - 1 - j);
-    sort_desc<VPL>(sk);
-    // ordered extraction: the warp's best head (ties go to the smaller code), whose lane then shifts its list
     int cnt = 0;
-    for (int it = 0; it < want; ++it) {
-      const unsigned ho = (unsigned)(sk[0] >> 32);
-      const int ht = lane + 32 * (VPL - 1 - (int)(unsigned)sk[0]);
-      const unsigned mo = __reduce_max_sync(0xffffffffu, ho);
-      if (mo <= kOrderedNegInf) break;
-      const int bt = (int)__reduce_min_sync(0xffffffffu, ho == mo ? (unsigned)ht : 0x7fffffffu);
-      if ((bt & 31) == lane) {
+    if constexpr (VPL >= 16) {
+      // Wide codebooks: no per-lane sort.  A sorting network of 16 or 32 keys is kilobytes of straight-line code that a
+      // warp runs once, and fetching it costs more than it saves (12.6 us per beam at T = 512 against 3.2 at T = 256;
+      // 6 us with this loop).  With many survivors per beam (K = 50) the sorted lists below are the cheaper form.
+      // Each round every lane finds its best remaining key (four independent scans, so the chain is VPL / 4 long), the
+      // warp picks the best of those (ties go to the smaller code), and the owner retires it: a short loop body.
+      unsigned ob[VPL];                                  // ordered score bits; 0 = used up
 #pragma unroll
-        for (int j = 0; j + 1 < VPL; ++j) sk[j] = sk[j + 1];
-        sk[VPL - 1] = 0ull;
+      for (int j = 0; j < VPL; ++j) ob[j] = ordered_bits(key[j]);
+#pragma unroll 1
+      for (int it = 0; it < want; ++it) {
+        unsigned qo[4]; int qj[4];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          qo[q4] = 0u; qj[q4] = q4 * (VPL / 4);
+#pragma unroll
+          for (int j = q4 * (VPL / 4); j < (q4 + 1) * (VPL / 4); ++j)
+            if (ob[j] > qo[q4]) { qo[q4] = ob[j]; qj[q4] = j; }
+        }
+        unsigned ho = qo[0]; int hj = qj[0];
+#pragma unroll
+        for (int q4 = 1; q4 < 4; ++q4)
+          if (qo[q4] > ho) { ho = qo[q4]; hj = qj[q4]; }     // strict: the smaller code wins a tie
+        const int ht = lane + 32 * hj;
+        const unsigned mo = __reduce_max_sync(0xffffffffu, ho);
+        if (mo <= kOrderedNegInf) break;
+        const int bt = (int)__reduce_min_sync(0xffffffffu, ho == mo ? (unsigned)ht : 0x7fffffffu);
+        if ((bt & 31) == lane) {
+#pragma unroll
+          for (int j = 0; j < VPL; ++j)
+            if (j == (bt >> 5)) ob[j] = 0u;
+        }
+        if (lane == 0) {
+          const float bv = from_ordered_bits(mo);
+          l_score[(size_t)r * a.K + cnt] = all_codes ? bv : base + bv;
+          l_tok[(size_t)r * a.K + cnt] = bt;
+        }
+        ++cnt;
       }
-      if (lane == 0) {
-        const float bv = from_ordered_bits(mo);
-        l_score[(size_t)r * a.K + cnt] = all_codes ? bv : base + bv;
-        l_tok[(size_t)r * a.K + cnt] = bt;
+    } else {
+      // this lane's keys in descending order: (ordered score bits, then the smaller code first); 0 = used up
+      unsigned long long sk[VPL];
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) sk[j] = ((unsigned long long)ordered_bits(key[j]) << 32) | (unsigned)(VPL - 1 - j);
+      sort_desc<VPL>(sk);
+      // ordered extraction: the warp's best head (ties go to the smaller code), whose lane then shifts its list
+      for (int it = 0; it < want; ++it) {
+        const unsigned ho = (unsigned)(sk[0] >> 32);
+        const int ht = lane + 32 * (VPL - 1 - (int)(unsigned)sk[0]);
+        const unsigned mo = __reduce_max_sync(0xffffffffu, ho);
+        if (mo <= kOrderedNegInf) break;
+        const int bt = (int)__reduce_min_sync(0xffffffffu, ho == mo ? (unsigned)ht : 0x7fffffffu);
+        if ((bt & 31) == lane) {
+#pragma unroll
+          for (int j = 0; j + 1 < VPL; ++j) sk[j] = sk[j + 1];
+          sk[VPL - 1] = 0ull;
+        }
+        if (lane == 0) {
+          const float bv = from_ordered_bits(mo);
+          l_score[(size_t)r * a.K + cnt] = all_codes ? bv : base + bv;
+          l_tok[(size_t)r * a.K + cnt] = bt;
+        }
+        ++cnt;
       }
-      ++cnt;
     }
     __syncwarp();
     if (!all_codes && (a.filter || a.prefix_filter)) {   // filter the chosen codes, keep their order
