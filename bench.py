@@ -31,7 +31,7 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 METRIC, UNIT = "items_per_s_decoded", "items/s"
 # bumped whenever a kernel of the family changes in a way that can change its DRAM traffic: a traffic figure taken
 # from an older revision is reported as null
-KERNEL_REV = {"gemm": 7, "attention_tc": 3, "attention_umma": 5, "probe": 3}
+KERNEL_REV = {"gemm": 7, "gemm_skinny": 2, "attention_tc": 3, "attention_umma": 5, "probe": 3}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the launches of the class in one decode step
 # (ncu, eager launches, L2 flushed before the step); key = class @ workload
 NCU_TRAFFIC = {
@@ -40,6 +40,11 @@ NCU_TRAFFIC = {
     # (three rounds) moved 1,371 MB, the 16 launches outside the layers 436 MB -> (32 x 1,371 + 436) / 400
     "gemm@7b": {"family": "gemm", "kernel_rev": 7, "dram_bytes_per_launch": 110.8e6,
                 "source": "profiles/gemm_tc_kernel_ncu.md, section E (two-layer cut, scaled by launches per layer)"},
+    # the weight-streaming kernel, captured on a two-layer cut of the paper-shaped backbone (same widths): the four
+    # projections of a layer read 8.61 + 67.25 + 34.02 + 12.75 MB, the LM-head rows 4.33 MB; a plain decode step of the
+    # 16-layer model is 2 x (64 layer launches + 1) + 1 launches -> (2 x (16 x 122.63 + 4.33) + 2.1) / 131
+    "gemm@paper": {"family": "gemm_skinny", "kernel_rev": 2, "dram_bytes_per_launch": 30.0e6,
+                   "source": "profiles/gemm_skinny_kernel_ncu.md (two-layer cut, scaled by launches per layer)"},
     "gemm@small": {"family": "gemm", "kernel_rev": 6, "dram_bytes_per_launch": 3.18e6, "source": "profiles/gemm_tc_kernel_ncu.md, section A2"},
     "probe@0.5b@67108864": {"family": "probe", "kernel_rev": 3, "dram_bytes_per_launch": 5.10e9, "source": "profiles/hs_probe_kernel.md"},
     "attention@small": {"family": "attention_tc", "kernel_rev": 3, "dram_bytes_per_launch": 31.5e6,
@@ -283,6 +288,8 @@ def time_decode(ctx, mode, drafts, steps, warmup, flush, dist, world, dev, barri
     # DRAM traffic of the dominant kernel from the ncu capture of that kernel in this workload (bytes per launch);
     # null when no capture matches the current kernel revision
     rec = ncu_traffic(f"{dom}@{w.name}")
+    if rec and rec["family"] == "gemm_skinny" and w.batch * w.beam * max(1, w.L - 1) > 128:
+        rec = None                     # that capture is of the weight-streaming kernel: engines of at most 128 rows per pass
     if rec:
         roof["traffic"] = rec["dram_bytes_per_launch"]
         roof["traffic_source"] = rec["source"]
